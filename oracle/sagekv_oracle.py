@@ -1,0 +1,283 @@
+"""Plain CPU oracle for the SAGE-KV hot path (arXiv 2503.08879, Section 2).
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, obviously-correct statement
+of what the four steps compute.  It is imported by the tests, by the smoke
+check and by the benchmark's CPU-baseline leg, and by nothing else; the CUDA
+library never calls it and shares no code, tables or helpers with it.
+
+Everything is numpy in float64.  bf16 tensors arrive as uint16 bit patterns and
+are widened exactly (a bf16 is the top half of an fp32).  One call handles one
+batch element and one layer.  Nothing here is blocked, fused or reordered
+beyond what the definitions below say.
+
+Notation (Section 2, Step 1, and Appendix A.2):
+  N    context length, the last token included
+  S    sink / initial tokens          (n_init)
+  R    recent tokens                  (n_recent)
+  E    eviction-region length,  E = N - 1 - S - R
+  H_q, H_kv   query / key-value head counts,  G = H_q / H_kv
+  k    tokens each query head keeps   (k_q in the C interface)
+  L    reduced-cache length per KV head,  L = S + G*k + R + 1
+
+Positions are 0-based here: sink [0,S), eviction region [S,S+E), recent window
+[S+E, N-1), last token N-1  (the paper's P_{1:S}, P_{S+1:S+E}, P_{S+E+1:N-1}, P_N).
+
+Pins (tests/test_oracle_pins.py): budget_split <- the numbers Appendix A.2
+prints; score <- closed forms (uniform keys, one planted key), row sums, a
+library softmax; select <- exhaustive subset search on tiny rows, library
+argmax / top-k on distinct values; compact <- row-by-row source identity;
+decode_step <- library scaled-dot-product attention for k = E, masked full
+attention for any k, sink+recent attention for k = 0, ring contents after
+t appends.  What is NOT pinned: that this heuristic reproduces the paper's
+LongBench accuracy ("parity unpinned" for the method as a whole: it needs
+the benchmark data and trained weights, neither of which is available).
+"""
+
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "bf16_bits_to_f64",
+    "f64_to_bf16_bits",
+    "budget_split",
+    "partition",
+    "score",
+    "select",
+    "compact",
+    "decode_step",
+    "full_attention",
+]
+
+
+# --------------------------------------------------------------------------
+# bf16 <-> float64 (storage format only; no arithmetic of the method)
+# --------------------------------------------------------------------------
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns (uint16) to float64."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def f64_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even narrowing of finite float64 values to bf16 bits."""
+    f = np.asarray(x, dtype=np.float64).astype(np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    rounded = u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))
+    return (rounded >> np.uint64(16)).astype(np.uint16)
+
+
+# --------------------------------------------------------------------------
+# Appendix A.2: how a token budget B is divided
+# --------------------------------------------------------------------------
+
+def budget_split(B: int, G: int) -> tuple[int, int, int]:
+    """(sink, k, recent) for token budget B and query-group number G.
+
+    Appendix A.2: sink window B/4, k = B/(2G), recent window B/4.  When 2G
+    does not divide B the appendix's own Qwen example (G = 7, B = 8192) takes
+    k = 512 and gives every slot that is left to the recent window
+    (8192 - 2048 - 7*512 = 2560).  Reading used here for the non-divisible
+    case: k is the largest power of two not above B/(2G); the recent window is
+    always B - sink - G*k.  In the divisible case this is the plain rule.
+    """
+    if B < 4 or G < 1:
+        raise ValueError("budget_split needs B >= 4 and G >= 1")
+    sink = B // 4
+    if B % (2 * G) == 0:
+        k = B // (2 * G)
+    else:
+        k = 1
+        while 2 * k * 2 * G <= B:
+            k *= 2
+    recent = B - sink - G * k
+    return sink, k, recent
+
+
+# --------------------------------------------------------------------------
+# Step 1: partition of the full cache
+# --------------------------------------------------------------------------
+
+def partition(N: int, S: int, R: int) -> dict:
+    """Index ranges of the four parts (Step 1).  Half-open, 0-based."""
+    E = N - 1 - S - R
+    if S < 0 or R < 0 or E < 0:
+        raise ValueError("need S >= 0, R >= 0 and S + R + 1 <= N")
+    return {
+        "E": E,
+        "sink": (0, S),
+        "evict": (S, S + E),
+        "recent": (S + E, N - 1),
+        "last": N - 1,
+    }
+
+
+# --------------------------------------------------------------------------
+# Step 2a: attention scores of the last token over the eviction region
+# --------------------------------------------------------------------------
+
+def score(q_last_bits: np.ndarray, K_bits: np.ndarray, S: int, R: int,
+          scale: float | None = None) -> np.ndarray:
+    """Softmax attention of the last token's query over the evicted tokens.
+
+    q_last_bits [H_q, d] and K_bits [H_kv, N, d] are bf16 bit patterns.  Query
+    head h reads KV head h // G.  Returns p [H_q, E] in float64 with
+        s[h, i] = scale * sum_c q[h, c] * K[h // G, S + i, c]
+        p[h, i] = exp(s[h, i] - max_j s[h, j]) / sum_j exp(s[h, j] - max_j s[h, j])
+    where j runs over the eviction region only (Step 2; scale = 1/sqrt(d)).
+    """
+    q = bf16_bits_to_f64(q_last_bits)
+    H_q, d = q.shape
+    H_kv, N, d2 = K_bits.shape
+    assert d == d2 and H_q % H_kv == 0
+    G = H_q // H_kv
+    part = partition(N, S, R)
+    E = part["E"]
+    lo, hi = part["evict"]
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    p = np.zeros((H_q, E), dtype=np.float64)
+    if E == 0:
+        return p
+    for g in range(H_kv):
+        Kev = bf16_bits_to_f64(K_bits[g, lo:hi])          # [E, d]
+        for j in range(G):
+            h = g * G + j
+            s = (Kev @ q[h]) * scale                      # [E]
+            m = np.max(s)
+            e = np.exp(s - m)
+            p[h] = e / np.sum(e)
+    return p
+
+
+# --------------------------------------------------------------------------
+# Step 2b: per-head top-k
+# --------------------------------------------------------------------------
+
+def select(p: np.ndarray, k: int, S: int) -> np.ndarray:
+    """Top-k of every score row, the lower position winning a tie.
+
+    p [H_q, E] in any float dtype; comparisons are made in that dtype.  Each
+    row is ordered by (score descending, position ascending); the first
+    min(k, E) entries are kept and re-ordered by position ascending (the
+    reduced cache keeps token order, Appendix A.2).  Returns absolute token
+    positions, int32 [H_q, min(k, E)], each in [S, S+E).
+    """
+    H_q, E = p.shape
+    kk = min(int(k), E)
+    out = np.zeros((H_q, kk), dtype=np.int32)
+    pos = np.arange(E)
+    for h in range(H_q):
+        order = np.lexsort((pos, -p[h]))      # last key is the primary one
+        out[h] = np.sort(order[:kk]) + S
+    return out
+
+
+# --------------------------------------------------------------------------
+# Step 3: reduced cache C = Concat(S, E_topk, R, P_N)
+# --------------------------------------------------------------------------
+
+def compact(K_bits: np.ndarray, V_bits: np.ndarray, idx: np.ndarray,
+            S: int, R: int) -> tuple[np.ndarray, np.ndarray]:
+    """Reduced cache per KV head (Step 3).
+
+    idx [H_q, k] are absolute positions chosen per query head.  "This yields
+    H_q groups of the top-k" (Step 2) and the budget counts G*k selected slots
+    per KV head (Appendix A.2), so the G lists of a KV head's query heads are
+    laid side by side, duplicates kept:
+        rows(g) = [0..S) ++ idx[g*G] ++ ... ++ idx[g*G+G-1] ++ [S+E..N-1) ++ [N-1]
+    Returns (Kc, Vc) uint16 [H_kv, L, d] with L = S + G*k + R + 1; pure copies.
+    """
+    H_kv, N, d = K_bits.shape
+    H_q, k = idx.shape
+    G = H_q // H_kv
+    E = partition(N, S, R)["E"]
+    L = S + G * k + R + 1
+    Kc = np.zeros((H_kv, L, d), dtype=np.uint16)
+    Vc = np.zeros((H_kv, L, d), dtype=np.uint16)
+    for g in range(H_kv):
+        rows = list(range(0, S))
+        for j in range(G):
+            rows.extend(int(t) for t in idx[g * G + j])
+        rows.extend(range(S + E, N - 1))
+        rows.append(N - 1)
+        assert len(rows) == L
+        for r, t in enumerate(rows):
+            Kc[g, r] = K_bits[g, t]
+            Vc[g, r] = V_bits[g, t]
+    return Kc, Vc
+
+
+# --------------------------------------------------------------------------
+# Plain softmax attention (the FullAttention baseline of Section 3.1)
+# --------------------------------------------------------------------------
+
+def full_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray,
+                   keep: np.ndarray | None = None,
+                   scale: float | None = None) -> tuple[np.ndarray, np.ndarray]:
+    """softmax(q K^T * scale) V for grouped heads, float64 in and out.
+
+    q [H_q, d]; K, V [H_kv, n, d]; keep [H_q, n] bool (False = logit -inf).
+    Returns (o [H_q, d], lse [H_q]) with lse the log of the softmax denominator.
+    """
+    H_q, d = q.shape
+    H_kv, n, _ = K.shape
+    G = H_q // H_kv
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    o = np.zeros((H_q, d), dtype=np.float64)
+    lse = np.full((H_q,), -np.inf, dtype=np.float64)
+    for h in range(H_q):
+        g = h // G
+        s = (K[g] @ q[h]) * scale
+        if keep is not None:
+            s = np.where(keep[h], s, -np.inf)
+        m = np.max(s)
+        if not np.isfinite(m):
+            continue
+        e = np.exp(s - m)
+        z = np.sum(e)
+        o[h] = (e / z) @ V[g]
+        lse[h] = m + np.log(z)
+    return o, lse
+
+
+# --------------------------------------------------------------------------
+# Step 4: one decode step on the reduced cache
+# --------------------------------------------------------------------------
+
+def decode_step(q_bits: np.ndarray, k_new_bits, v_new_bits,
+                Kc: np.ndarray, Vc: np.ndarray, step: int,
+                S: int, k: int, R: int,
+                scale: float | None = None) -> tuple[np.ndarray, np.ndarray, int]:
+    """Append one token to the recent window, then attend (Step 4).
+
+    The reduced cache of a KV head is [sink S | G segments of k | window R+1],
+    the window being the R recent tokens followed by the last token, oldest
+    first.  Appending token number `step` (0, 1, ...) overwrites window slot
+    step mod (R+1): the oldest entry leaves, the size stays (Step 4).  With
+    k_new_bits None nothing is appended.  Query head h = g*G + j then attends
+    to the sink, to ITS OWN segment j and to the window, i.e. to S + k + R + 1
+    entries, the length Step 3 states.  Kc, Vc are updated in place.
+    Returns (o [H_q, d] float64, lse [H_q], step after the call).
+    """
+    H_kv, L, d = Kc.shape
+    H_q = q_bits.shape[0]
+    G = H_q // H_kv
+    assert L == S + G * k + R + 1
+    if k_new_bits is not None:
+        slot = S + G * k + (step % (R + 1))
+        for g in range(H_kv):
+            Kc[g, slot] = k_new_bits[g]
+            Vc[g, slot] = v_new_bits[g]
+        step = step + 1
+    keep = np.zeros((H_q, L), dtype=bool)
+    for h in range(H_q):
+        j = h % G
+        keep[h, 0:S] = True
+        keep[h, S + j * k: S + (j + 1) * k] = True
+        keep[h, S + G * k: L] = True
+    o, lse = full_attention(bf16_bits_to_f64(q_bits), bf16_bits_to_f64(Kc),
+                            bf16_bits_to_f64(Vc), keep=keep, scale=scale)
+    return o, lse, step
