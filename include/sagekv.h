@@ -1,0 +1,162 @@
+/*
+ * sagekv.h -- C interface of the SAGE-KV hot path (arXiv 2503.08879, Section 2)
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The method, per transformer layer, after the prompt has been prefilled:
+ *   Step 1  split the KV cache of N tokens into  sink [0,S) | eviction region
+ *           [S,S+E) | recent window [S+E,N-1) | last token N-1,  E = N-1-S-R;
+ *   Step 2  score the eviction region with the last token's query and keep,
+ *           for every query head, the k best-scoring tokens;
+ *   Step 3  build the reduced cache  C = Concat(sink, selected, recent, last);
+ *   Step 4  decode on C; every new token's (k,v) enters the recent window and
+ *           the oldest entry of the window leaves.
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer unless its comment says "host".
+ *     The library never takes ownership of a caller's buffer.
+ *   - bf16 tensors are passed as `void*` / `const void*` (16-bit elements);
+ *     head_dim is innermost and contiguous; head_dim must be 128.
+ *   - `sagekv_strides` are in ELEMENTS.  Base pointers must be 16-byte aligned
+ *     and every stride a multiple of 8 elements.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL
+ *     is the default stream).  No call synchronises, and none of the three hot
+ *     calls allocates.  Calls that share a context must be issued on one stream
+ *     (or otherwise ordered): they share the context's scratch memory.
+ *   - Return value: SAGEKV_OK (0) or a negative SAGEKV_ERR_* code.  Argument
+ *     errors are found on the host before anything is launched.
+ *   - A query head h reads KV head h / G, G = n_q_heads / n_kv_heads <= 8.
+ */
+#ifndef SAGEKV_H_
+#define SAGEKV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  SAGEKV_OK = 0,
+  SAGEKV_ERR_INVALID = -1,     /* null pointer, negative size, S+R+1 > N, k % G != 0 ... */
+  SAGEKV_ERR_ALIGN = -2,       /* pointer or stride breaks the alignment rules above     */
+  SAGEKV_ERR_UNSUPPORTED = -3, /* head_dim != 128, G > 8, size beyond the context's max  */
+  SAGEKV_ERR_CUDA = -4,        /* a CUDA runtime call failed (see sagekv_last_cuda_error) */
+  SAGEKV_ERR_NOMEM = -5        /* scratch allocation failed in sagekv_create             */
+};
+
+typedef struct sagekv_ctx sagekv_ctx; /* opaque; owns only its scratch memory */
+
+typedef struct {
+  int32_t n_q_heads;    /* H_q                                              */
+  int32_t n_kv_heads;   /* H_kv, divides H_q                                */
+  int32_t head_dim;     /* d_h, must be 128                                 */
+  int32_t batch;        /* independent sequences per call                   */
+  float softmax_scale;  /* 0 => 1/sqrt(head_dim)                            */
+} sagekv_shape;
+
+typedef struct {
+  int64_t batch_stride; /* elements between consecutive batch entries       */
+  int64_t head_stride;  /* elements between consecutive KV heads            */
+  int64_t token_stride; /* elements between consecutive tokens (>= head_dim)*/
+} sagekv_strides;
+
+/* Description of one layer's reduced cache.  Filled by sagekv_select_compact,
+ * read by sagekv_decode_attn.  Host struct; `d_step` is a device pointer to one
+ * int32 owned by the caller: the number of tokens appended so far. */
+typedef struct {
+  int32_t n_init;    /* S                                                    */
+  int32_t k_q;       /* tokens kept per query head (after clamping to E)     */
+  int32_t n_sel;     /* G * k_q selected slots per KV head                   */
+  int32_t n_recent;  /* R                                                    */
+  int32_t ring_len;  /* R + 1: the recent tokens and the last token          */
+  int32_t len;       /* L = S + n_sel + R + 1 rows per KV head               */
+  int32_t *d_step;   /* device int32, reset to 0 by sagekv_select_compact    */
+} sagekv_cache_state;
+
+/* Create / destroy a context for one shape.  `max_ctx` bounds N, `max_len`
+ * bounds the reduced-cache length L of later calls; scratch for the score
+ * partials and the split-K partials is allocated here (cudaMalloc on the
+ * current device) and freed by sagekv_destroy.  Errors: INVALID, UNSUPPORTED,
+ * NOMEM.  `*out` is NULL on failure. */
+int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, int32_t max_len);
+int sagekv_destroy(sagekv_ctx *ctx);
+
+/* Appendix A.2, "Hyper-parameter settings": token budget B and query-group
+ * number G give sink window B/4, k = B/(2G) kept tokens per query head and
+ * recent window B/4.  When 2G does not divide B (the appendix's Qwen2.5 case,
+ * G = 7: k = 512, recent = 8192 - 2048 - 7*512 = 2560) k is the largest power
+ * of two not above B/(2G) and the slots left over go to the recent window:
+ * n_recent = B - n_init - G*k_q always.  Host-only; outputs are host pointers.
+ * Errors: INVALID for B < 4, G < 1 or a null pointer. */
+int sagekv_budget_split(int32_t B, int32_t G, int32_t *n_init, int32_t *k_q, int32_t *n_recent);
+
+/* Step 2, first half ("attention scores between the last token of the input
+ * sequence and the evicted tokens").  For every batch entry b, query head h and
+ * eviction-region offset i in [0,E):
+ *     s = scale * <q_last[b,h,:], K[b, h/G, S+i, :]>
+ *     scores[b,h,i] = exp(s - max_j s_j) / sum_j exp(s_j - max_j s_j),  j in [0,E)
+ * (a softmax over the eviction region only; every row sums to 1).
+ *   q_last  bf16 [batch, H_q, 128], contiguous.
+ *   K       bf16 [batch, H_kv, n_ctx, 128] addressed through `ks`.
+ *   scores  fp32 [batch*H_q rows], row r at scores + r*scores_row_stride;
+ *           scores_row_stride >= E and a multiple of 4, base 16-byte aligned.
+ * bf16 products are accumulated in fp32.  E == 0 writes nothing.
+ * Errors: INVALID (null, n_init+n_recent+1 > n_ctx, stride < E), ALIGN,
+ * UNSUPPORTED (n_ctx above the context's max_ctx), CUDA. */
+int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_strides ks,
+                 int64_t n_ctx, int32_t n_init, int32_t n_recent,
+                 float *scores, int64_t scores_row_stride, void *stream);
+
+/* Step 2, second half, and Step 3.  `k` is the number of selected slots per KV
+ * head; it must be a multiple of G and every query head keeps k_q = min(k/G, E)
+ * tokens ("this yields H_q groups of the top-k"; Appendix A.2 counts G*k
+ * selected slots in the budget).  Per score row the k_q largest scores are
+ * kept; of equal scores the lower position wins; the kept positions are written
+ * in ascending order (token order is maintained, Appendix A.2).
+ *   idx     int32 [batch, H_q, k_q] contiguous: absolute positions in [S,S+E).
+ *   Kc, Vc  bf16 [batch, H_kv, >= L, 128] through `cs`; row layout per KV head g
+ *           [0,S) sink | G segments of k_q rows, segment j = idx of head g*G+j |
+ *           R recent tokens | last token,     L = S + G*k_q + R + 1
+ *           (Step 3: C = Concat(S, E_topk, R, P_N)).  Rows are bit-exact copies.
+ *   state   host struct, filled on return; state->d_step must already point to
+ *           a device int32, which is set to 0 on the stream.
+ * Comparisons are made on the fp32 bit patterns given; scores must not be NaN.
+ * Errors: INVALID (null, k < 0, k % G != 0, bad partition), ALIGN,
+ * UNSUPPORTED (L above the context's max_len), CUDA. */
+int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_row_stride,
+                          const void *K, const void *V, sagekv_strides ks,
+                          int64_t n_ctx, int32_t n_init, int32_t n_recent, int32_t k,
+                          int32_t *idx, void *Kc, void *Vc, sagekv_strides cs,
+                          sagekv_cache_state *state, void *stream);
+
+/* Step 4 ("each new token's KV pair is added to the recent window R, evicting
+ * the oldest entry in R to maintain its size").  With t = *state->d_step:
+ * if k_new / v_new are non-NULL they overwrite row S + n_sel + (t mod ring_len)
+ * of every KV head (row S + n_sel is the oldest recent token after compaction)
+ * and *d_step becomes t+1; with both NULL nothing is appended.  Then
+ *     out[b,h,:] = softmax(scale * q[b,h,:] . Kview^T) . Vview
+ * where the view of head h = g*G+j is sink + segment j + window, i.e.
+ * S + k_q + R + 1 rows, the reduced-cache length Step 3 states.
+ *   q       bf16 [batch, H_q, 128];  k_new, v_new  bf16 [batch, H_kv, 128]
+ *   out     bf16 [batch, H_q, 128];  lse  fp32 [batch, H_q] or NULL (natural-log
+ *           of the softmax denominator, max included)
+ * The cache is streamed once in split-K partitions whose partial results are
+ * merged by log-sum-exp inside the same launch; products and sums are fp32,
+ * softmax weights are rounded to bf16 before they multiply V.
+ * Errors: INVALID (null, exactly one of k_new/v_new NULL), ALIGN,
+ * UNSUPPORTED (state->len above the context's max_len), CUDA. */
+int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                       void *Kc, void *Vc, sagekv_strides cs, const sagekv_cache_state *state,
+                       void *out, float *lse, void *stream);
+
+/* Text for a return code; never NULL.  Static storage. */
+const char *sagekv_strerror(int code);
+
+/* The cudaError_t value of the most recent failing CUDA call made through
+ * `ctx` (0 if none), for diagnosing SAGEKV_ERR_CUDA. */
+int sagekv_last_cuda_error(const sagekv_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAGEKV_H_ */

@@ -1,0 +1,132 @@
+// Shared device helpers and the internal launch interface of the SAGE-KV kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sagekv.h"
+
+namespace sagekv {
+
+constexpr int kHeadDim = 128;             // elements per row; a bf16 row is 256 bytes
+constexpr int kMaxGroup = 8;              // G <= 8: one mma tile dimension holds a KV head's query heads
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ---- score ---------------------------------------------------------------
+constexpr int kScoreWarps = 8;
+constexpr int kScoreTokPerWarp = 32;      // two 16-token mma tiles in flight per warp
+constexpr int kScoreChunk = kScoreWarps * kScoreTokPerWarp;   // tokens per CTA
+
+struct ScoreParams {
+  const uint16_t *q;       // [B, H_q, 128]
+  const uint16_t *K;       // [B, H_kv, N, 128] through ks
+  sagekv_strides ks;
+  float *scores;           // [B*H_q rows]
+  int64_t row_stride;
+  float2 *partials;        // [B*H_q, n_chunks] (max, sum) in log2 units
+  int n_chunks;
+  int E, S, G, H_q, H_kv, B;
+  float scale_log2;        // softmax scale * log2(e)
+};
+cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream);
+
+// ---- select + compact ------------------------------------------------------
+struct SelectParams {
+  const float *scores;
+  int64_t row_stride;
+  const uint16_t *K, *V;
+  sagekv_strides ks;
+  uint16_t *Kc, *Vc;
+  sagekv_strides cs;
+  int32_t *idx;            // [B, H_q, k_q]
+  int32_t *d_step;
+  int E, S, R, N, k_q, G, H_q, H_kv, B;
+};
+cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t stream);
+cudaError_t select_compact_setup();   // one-time function attributes
+
+// ---- decode attention ------------------------------------------------------
+constexpr int kDecodeWarps = 4;
+constexpr int kDecodeTile = kDecodeWarps * 16;                         // tokens per CTA iteration
+constexpr int kPartialStride = kMaxGroup * kHeadDim + 2 * kMaxGroup;   // floats per split partial: O[8][128], m[8], l[8]
+
+struct DecodeParams {
+  const uint16_t *q;       // [B, H_q, 128]
+  const uint16_t *k_new;   // [B, H_kv, 128] or null
+  const uint16_t *v_new;
+  uint16_t *Kc, *Vc;
+  sagekv_strides cs;
+  uint16_t *out;           // [B, H_q, 128]
+  float *lse;              // [B, H_q] or null
+  float *partials;         // [B*H_kv, n_splits, kPartialStride]
+  int32_t *tickets;        // [B*H_kv] arrival counters + [1] finished-heads counter, all 0 between launches
+  int32_t *d_step;
+  int n_splits, iters;     // every split covers iters * kDecodeTile rows
+  int S, k_q, n_sel, ring_len, L, G, H_q, H_kv, B;
+  float scale_log2;
+};
+cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream);
+
+// ---- device helpers --------------------------------------------------------
+#if defined(__CUDACC__)
+
+// 16-byte read-only load that does not linger in L1: cache rows are streamed once.
+__device__ __forceinline__ uint4 ld_stream_v4(const void *ptr) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(ptr));
+  return v;
+}
+
+// plain 16-byte load (for rows another kernel on the stream may have just written)
+__device__ __forceinline__ uint4 ld_v4(const void *ptr) {
+  uint4 v;
+  asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(ptr));
+  return v;
+}
+
+__device__ __forceinline__ void st_v4(void *ptr, uint4 v) {
+  asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+}
+
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float &d0, float &d1, float &d2, float &d3, uint32_t a0, uint32_t a1,
+                                               uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// two fp32 -> packed bf16x2 (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// merge two (max, sum) pairs of a running softmax kept in log2 units
+__device__ __forceinline__ void merge_ml(float &m, float &l, float m2, float l2) {
+  const float M = fmaxf(m, m2);
+  if (M == -INFINITY) {
+    l = 0.f;
+  } else {
+    l = l * fast_exp2(m - M) + l2 * fast_exp2(m2 - M);
+  }
+  m = M;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace sagekv

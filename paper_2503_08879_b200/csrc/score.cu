@@ -1,0 +1,163 @@
+// Step 2 (first half): softmax attention of the last token's query over the eviction region.
+//
+// Pass 1 (score_logits_kernel) streams the K rows of the eviction region once.  A warp takes 16 tokens
+// per tensor-core tile: token rows are the M dimension, the KV head's G query heads (padded to 8) the
+// N dimension, head_dim the contraction.  Every lane loads 16-byte pieces of "its" two token rows
+// straight from global memory into the A fragment; because a dot product does not care in which order
+// the 128 products are summed, the fragment's k slots are filled with whatever columns those 16 bytes
+// hold and the query (B fragment) is loaded with the same permutation.  The kernel writes the scaled
+// logits (log2 units) and one (max, sum-of-exp2) pair per CTA and head.
+// Pass 2 (score_finalize_kernel) merges those pairs per row and normalises the row in place; the
+// logits were written a few microseconds earlier and are still in L2.
+#include "common.cuh"
+
+namespace sagekv {
+
+__global__ void __launch_bounds__(kScoreWarps * 32) score_logits_kernel(const ScoreParams p) {
+  const int chunk = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, c = lane & 3;
+
+  // B fragments: query head (kvh*G + g) for n = g, zero padding for n >= G
+  uint4 qf[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) qf[j] = make_uint4(0u, 0u, 0u, 0u);
+  if (g < p.G) {
+    const uint16_t *qrow = p.q + ((int64_t)b * p.H_q + kvh * p.G + g) * kHeadDim;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) qf[j] = *reinterpret_cast<const uint4 *>(qrow + j * 32 + c * 8);
+  }
+
+  const uint16_t *Kbase = p.K + (int64_t)b * p.ks.batch_stride + (int64_t)kvh * p.ks.head_stride +
+                          (int64_t)p.S * p.ks.token_stride;
+  const int tok_base = chunk * kScoreChunk + warp * kScoreTokPerWarp;
+  const int last = p.E - 1;
+
+  // lane (g, c) holds, of token rows g and g+8 of each tile, the 16-byte pieces at columns j*32 + c*8
+  uint4 ka[2][4], kb[2][4];
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int r0 = min(tok_base + t * 16 + g, last);
+    const int r1 = min(tok_base + t * 16 + g + 8, last);
+    const char *pa = reinterpret_cast<const char *>(Kbase + (int64_t)r0 * p.ks.token_stride) + c * 16;
+    const char *pb = reinterpret_cast<const char *>(Kbase + (int64_t)r1 * p.ks.token_stride) + c * 16;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      ka[t][j] = ld_stream_v4(pa + j * 64);
+      kb[t][j] = ld_stream_v4(pb + j * 64);
+    }
+  }
+
+  // running softmax statistics of heads 2c and 2c+1 over the rows this lane sees
+  float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
+  const int h0 = 2 * c, h1 = 2 * c + 1;
+  float *row0 = p.scores + ((int64_t)b * p.H_q + kvh * p.G + h0) * p.row_stride;
+  float *row1 = row0 + p.row_stride;
+
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      mma_bf16_16816(a0, a1, a2, a3, ka[t][j].x, kb[t][j].x, ka[t][j].y, kb[t][j].y, qf[j].x, qf[j].y);
+      mma_bf16_16816(a0, a1, a2, a3, ka[t][j].z, kb[t][j].z, ka[t][j].w, kb[t][j].w, qf[j].z, qf[j].w);
+    }
+    const int r0 = tok_base + t * 16 + g, r1 = r0 + 8;
+    const float s00 = a0 * p.scale_log2, s01 = a1 * p.scale_log2;   // (r0,h0) (r0,h1)
+    const float s10 = a2 * p.scale_log2, s11 = a3 * p.scale_log2;   // (r1,h0) (r1,h1)
+    const bool v0 = r0 < p.E, v1 = r1 < p.E;
+    if (h0 < p.G) {
+      if (v0) row0[r0] = s00;
+      if (v1) row0[r1] = s10;
+      const float x0 = v0 ? s00 : -INFINITY, x1 = v1 ? s10 : -INFINITY;
+      const float M = fmaxf(m0, fmaxf(x0, x1));
+      if (M != -INFINITY) l0 = l0 * fast_exp2(m0 - M) + fast_exp2(x0 - M) + fast_exp2(x1 - M);
+      m0 = M;
+    }
+    if (h1 < p.G) {
+      if (v0) row1[r0] = s01;
+      if (v1) row1[r1] = s11;
+      const float x0 = v0 ? s01 : -INFINITY, x1 = v1 ? s11 : -INFINITY;
+      const float M = fmaxf(m1, fmaxf(x0, x1));
+      if (M != -INFINITY) l1 = l1 * fast_exp2(m1 - M) + fast_exp2(x0 - M) + fast_exp2(x1 - M);
+      m1 = M;
+    }
+  }
+
+  // over the 8 row groups of the warp (lanes with equal c)
+#pragma unroll
+  for (int off = 4; off < 32; off <<= 1) {
+    merge_ml(m0, l0, __shfl_xor_sync(0xffffffffu, m0, off), __shfl_xor_sync(0xffffffffu, l0, off));
+    merge_ml(m1, l1, __shfl_xor_sync(0xffffffffu, m1, off), __shfl_xor_sync(0xffffffffu, l1, off));
+  }
+  __shared__ float sm_m[kScoreWarps][kMaxGroup], sm_l[kScoreWarps][kMaxGroup];
+  if (g == 0) {
+    sm_m[warp][h0] = m0; sm_l[warp][h0] = l0;
+    sm_m[warp][h1] = m1; sm_l[warp][h1] = l1;
+  }
+  __syncthreads();
+  if (threadIdx.x < p.G) {
+    const int h = threadIdx.x;
+    float m = sm_m[0][h], l = sm_l[0][h];
+#pragma unroll
+    for (int w = 1; w < kScoreWarps; ++w) merge_ml(m, l, sm_m[w][h], sm_l[w][h]);
+    p.partials[((int64_t)b * p.H_q + kvh * p.G + h) * p.n_chunks + chunk] = make_float2(m, l);
+  }
+}
+
+constexpr int kFinalizeThreads = 256;
+
+__global__ void __launch_bounds__(kFinalizeThreads) score_finalize_kernel(const ScoreParams p, int per_slice) {
+  const int row = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float m = -INFINITY, l = 0.f;
+  const float2 *part = p.partials + (int64_t)row * p.n_chunks;
+  for (int i = threadIdx.x; i < p.n_chunks; i += kFinalizeThreads) {
+    const float2 v = part[i];
+    merge_ml(m, l, v.x, v.y);
+  }
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1)
+    merge_ml(m, l, __shfl_xor_sync(0xffffffffu, m, off), __shfl_xor_sync(0xffffffffu, l, off));
+  __shared__ float sm_m[kFinalizeThreads / 32], sm_l[kFinalizeThreads / 32];
+  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+  __syncthreads();
+  m = sm_m[0]; l = sm_l[0];
+#pragma unroll
+  for (int w = 1; w < kFinalizeThreads / 32; ++w) merge_ml(m, l, sm_m[w], sm_l[w]);
+  const float inv = 1.f / l;
+
+  float *rowp = p.scores + (int64_t)row * p.row_stride;
+  const int lo = blockIdx.x * per_slice;            // per_slice is a multiple of 4
+  const int hi = min(p.E, lo + per_slice);
+  for (int i = lo + threadIdx.x * 4; i < hi; i += kFinalizeThreads * 4) {
+    if (i + 3 < hi) {
+      float4 v = *reinterpret_cast<float4 *>(rowp + i);
+      v.x = fast_exp2(v.x - m) * inv; v.y = fast_exp2(v.y - m) * inv;
+      v.z = fast_exp2(v.z - m) * inv; v.w = fast_exp2(v.w - m) * inv;
+      *reinterpret_cast<float4 *>(rowp + i) = v;
+    } else {
+      for (int e = i; e < hi; ++e) rowp[e] = fast_exp2(rowp[e] - m) * inv;
+    }
+  }
+}
+
+cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream) {
+  if (p.E <= 0) return cudaSuccess;
+  dim3 grid(p.n_chunks, p.H_kv, p.B);
+  score_logits_kernel<<<grid, kScoreWarps * 32, 0, stream>>>(p);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  const int rows = p.B * p.H_q;
+  int slices = (n_sm * 4 + rows - 1) / rows;
+  const int max_slices = (p.E + 1023) / 1024;
+  if (slices > max_slices) slices = max_slices;
+  if (slices < 1) slices = 1;
+  int per_slice = (p.E + slices - 1) / slices;
+  per_slice = (per_slice + 3) & ~3;
+  slices = (p.E + per_slice - 1) / per_slice;
+  score_finalize_kernel<<<dim3(slices, rows), kFinalizeThreads, 0, stream>>>(p, per_slice);
+  return cudaGetLastError();
+}
+
+}  // namespace sagekv
