@@ -1,0 +1,252 @@
+// The C interface (include/sagekv.h): argument checks on the host, then the kernel launches.
+#include <math.h>
+#include <new>
+
+#include "common.cuh"
+
+using namespace sagekv;
+
+struct sagekv_ctx {
+  sagekv_shape shape;
+  int G;
+  int64_t max_ctx;
+  int32_t max_len;
+  int n_sm;
+  float scale;
+  float2 *score_partials;   // [B*H_q, ceil(max_ctx / kScoreChunk)]
+  int max_chunks;
+  float *decode_partials;   // [B*H_kv, max_splits, kPartialStride]
+  int max_splits;
+  int32_t *tickets;         // [B*H_kv + 1], zero between launches
+  int last_cuda_error;
+};
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool strides_ok(const sagekv_strides &s) {
+  return s.batch_stride % 8 == 0 && s.head_stride % 8 == 0 && s.token_stride % 8 == 0;
+}
+int cuda_fail(sagekv_ctx *ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda_error = (int)e;
+  return SAGEKV_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, int32_t max_len) {
+  if (out == nullptr) return SAGEKV_ERR_INVALID;
+  *out = nullptr;
+  if (shape == nullptr || shape->n_q_heads < 1 || shape->n_kv_heads < 1 || shape->batch < 1 || max_ctx < 1 ||
+      max_len < 1 || shape->n_q_heads % shape->n_kv_heads != 0 || !(shape->softmax_scale >= 0.f))
+    return SAGEKV_ERR_INVALID;
+  if (shape->head_dim != kHeadDim || shape->n_q_heads / shape->n_kv_heads > kMaxGroup ||
+      max_ctx > (int64_t)1 << 30 || (int64_t)shape->batch * shape->n_q_heads > 65535)
+    return SAGEKV_ERR_UNSUPPORTED;
+  sagekv_ctx *ctx = new (std::nothrow) sagekv_ctx();
+  if (ctx == nullptr) return SAGEKV_ERR_NOMEM;
+  ctx->shape = *shape;
+  ctx->G = shape->n_q_heads / shape->n_kv_heads;
+  ctx->max_ctx = max_ctx;
+  ctx->max_len = max_len;
+  ctx->scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.0f / sqrtf((float)shape->head_dim);
+  ctx->last_cuda_error = 0;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    delete ctx;
+    return SAGEKV_ERR_CUDA;
+  }
+  ctx->n_sm = prop.multiProcessorCount;
+  ctx->max_chunks = (int)((max_ctx + kScoreChunk - 1) / kScoreChunk);
+  ctx->max_splits = (max_len + kDecodeTile - 1) / kDecodeTile;
+  const size_t n_rows = (size_t)shape->batch * shape->n_q_heads;
+  const size_t n_heads = (size_t)shape->batch * shape->n_kv_heads;
+  cudaError_t e = cudaMalloc(&ctx->score_partials, n_rows * ctx->max_chunks * sizeof(float2));
+  if (e == cudaSuccess)
+    e = cudaMalloc(&ctx->decode_partials, n_heads * ctx->max_splits * kPartialStride * sizeof(float));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->tickets, (n_heads + 1) * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(ctx->tickets, 0, (n_heads + 1) * sizeof(int32_t));
+  if (e == cudaSuccess) e = select_compact_setup();
+  if (e != cudaSuccess) {
+    cudaFree(ctx->score_partials);
+    cudaFree(ctx->decode_partials);
+    cudaFree(ctx->tickets);
+    delete ctx;
+    cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? SAGEKV_ERR_NOMEM : SAGEKV_ERR_CUDA;
+  }
+  *out = ctx;
+  return SAGEKV_OK;
+}
+
+int sagekv_destroy(sagekv_ctx *ctx) {
+  if (ctx == nullptr) return SAGEKV_ERR_INVALID;
+  cudaFree(ctx->score_partials);
+  cudaFree(ctx->decode_partials);
+  cudaFree(ctx->tickets);
+  delete ctx;
+  return SAGEKV_OK;
+}
+
+int sagekv_budget_split(int32_t B, int32_t G, int32_t *n_init, int32_t *k_q, int32_t *n_recent) {
+  if (B < 4 || G < 1 || n_init == nullptr || k_q == nullptr || n_recent == nullptr) return SAGEKV_ERR_INVALID;
+  const int32_t sink = B / 4;
+  int32_t k;
+  if (B % (2 * G) == 0) {
+    k = B / (2 * G);
+  } else {
+    k = 1;
+    while ((int64_t)4 * k * G <= B) k *= 2;   // largest power of two with 2*G*k <= B
+  }
+  *n_init = sink;
+  *k_q = k;
+  *n_recent = B - sink - G * k;
+  return SAGEKV_OK;
+}
+
+int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_strides ks, int64_t n_ctx, int32_t n_init,
+                 int32_t n_recent, float *scores, int64_t scores_row_stride, void *stream) {
+  if (ctx == nullptr || q_last == nullptr || K == nullptr || scores == nullptr) return SAGEKV_ERR_INVALID;
+  if (n_init < 0 || n_recent < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx) return SAGEKV_ERR_INVALID;
+  if (n_ctx > ctx->max_ctx) return SAGEKV_ERR_UNSUPPORTED;
+  const int64_t E = n_ctx - 1 - n_init - n_recent;
+  if (scores_row_stride < E || ks.token_stride < kHeadDim) return SAGEKV_ERR_INVALID;
+  if (!aligned16(q_last) || !aligned16(K) || !aligned16(scores) || !strides_ok(ks) || scores_row_stride % 4 != 0)
+    return SAGEKV_ERR_ALIGN;
+  ScoreParams p;
+  p.q = static_cast<const uint16_t *>(q_last);
+  p.K = static_cast<const uint16_t *>(K);
+  p.ks = ks;
+  p.scores = scores;
+  p.row_stride = scores_row_stride;
+  p.partials = ctx->score_partials;
+  p.n_chunks = (int)((E + kScoreChunk - 1) / kScoreChunk);
+  p.E = (int)E;
+  p.S = n_init;
+  p.G = ctx->G;
+  p.H_q = ctx->shape.n_q_heads;
+  p.H_kv = ctx->shape.n_kv_heads;
+  p.B = ctx->shape.batch;
+  p.scale_log2 = ctx->scale * kLog2e;
+  const cudaError_t e = launch_score(p, ctx->n_sm, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
+}
+
+int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_row_stride, const void *K,
+                          const void *V, sagekv_strides ks, int64_t n_ctx, int32_t n_init, int32_t n_recent,
+                          int32_t k, int32_t *idx, void *Kc, void *Vc, sagekv_strides cs, sagekv_cache_state *state,
+                          void *stream) {
+  if (ctx == nullptr || K == nullptr || V == nullptr || Kc == nullptr || Vc == nullptr || state == nullptr ||
+      state->d_step == nullptr)
+    return SAGEKV_ERR_INVALID;
+  if (n_init < 0 || n_recent < 0 || k < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx ||
+      k % ctx->G != 0)
+    return SAGEKV_ERR_INVALID;
+  if (n_ctx > ctx->max_ctx) return SAGEKV_ERR_UNSUPPORTED;
+  const int64_t E = n_ctx - 1 - n_init - n_recent;
+  int64_t k_q = k / ctx->G;
+  if (k_q > E) k_q = E;
+  if (k_q > 0 && (scores == nullptr || idx == nullptr || scores_row_stride < E)) return SAGEKV_ERR_INVALID;
+  if (ks.token_stride < kHeadDim || cs.token_stride < kHeadDim) return SAGEKV_ERR_INVALID;
+  const int64_t L = (int64_t)n_init + ctx->G * k_q + n_recent + 1;
+  if (L > ctx->max_len) return SAGEKV_ERR_UNSUPPORTED;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !strides_ok(ks) || !strides_ok(cs) ||
+      (k_q > 0 && (!aligned16(scores) || scores_row_stride % 4 != 0)))
+    return SAGEKV_ERR_ALIGN;
+  SelectParams p;
+  p.scores = scores;
+  p.row_stride = scores_row_stride;
+  p.K = static_cast<const uint16_t *>(K);
+  p.V = static_cast<const uint16_t *>(V);
+  p.ks = ks;
+  p.Kc = static_cast<uint16_t *>(Kc);
+  p.Vc = static_cast<uint16_t *>(Vc);
+  p.cs = cs;
+  p.idx = idx;
+  p.d_step = state->d_step;
+  p.E = (int)E;
+  p.S = n_init;
+  p.R = n_recent;
+  p.N = (int)n_ctx;
+  p.k_q = (int)k_q;
+  p.G = ctx->G;
+  p.H_q = ctx->shape.n_q_heads;
+  p.H_kv = ctx->shape.n_kv_heads;
+  p.B = ctx->shape.batch;
+  const cudaError_t e = launch_select_compact(p, ctx->n_sm, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  state->n_init = n_init;
+  state->k_q = (int32_t)k_q;
+  state->n_sel = (int32_t)(ctx->G * k_q);
+  state->n_recent = n_recent;
+  state->ring_len = n_recent + 1;
+  state->len = (int32_t)L;
+  return SAGEKV_OK;
+}
+
+int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *Kc, void *Vc,
+                       sagekv_strides cs, const sagekv_cache_state *state, void *out, float *lse, void *stream) {
+  if (ctx == nullptr || q == nullptr || Kc == nullptr || Vc == nullptr || state == nullptr || out == nullptr)
+    return SAGEKV_ERR_INVALID;
+  if ((k_new == nullptr) != (v_new == nullptr)) return SAGEKV_ERR_INVALID;
+  if (k_new != nullptr && state->d_step == nullptr) return SAGEKV_ERR_INVALID;
+  if (state->n_init < 0 || state->k_q < 0 || state->n_recent < 0 || state->n_sel != ctx->G * state->k_q ||
+      state->ring_len != state->n_recent + 1 || state->len != state->n_init + state->n_sel + state->ring_len ||
+      cs.token_stride < kHeadDim)
+    return SAGEKV_ERR_INVALID;
+  if (state->len > ctx->max_len) return SAGEKV_ERR_UNSUPPORTED;
+  if (!aligned16(q) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(out) || !strides_ok(cs) ||
+      (k_new != nullptr && (!aligned16(k_new) || !aligned16(v_new))))
+    return SAGEKV_ERR_ALIGN;
+  DecodeParams p;
+  p.q = static_cast<const uint16_t *>(q);
+  p.k_new = static_cast<const uint16_t *>(k_new);
+  p.v_new = static_cast<const uint16_t *>(v_new);
+  p.Kc = static_cast<uint16_t *>(Kc);
+  p.Vc = static_cast<uint16_t *>(Vc);
+  p.cs = cs;
+  p.out = static_cast<uint16_t *>(out);
+  p.lse = lse;
+  p.partials = ctx->decode_partials;
+  p.tickets = ctx->tickets;
+  p.d_step = state->d_step;
+  p.S = state->n_init;
+  p.k_q = state->k_q;
+  p.n_sel = state->n_sel;
+  p.ring_len = state->ring_len;
+  p.L = state->len;
+  p.G = ctx->G;
+  p.H_q = ctx->shape.n_q_heads;
+  p.H_kv = ctx->shape.n_kv_heads;
+  p.B = ctx->shape.batch;
+  p.scale_log2 = ctx->scale * kLog2e;
+  // partitions of iters*64 rows: as many CTAs as keep about two per SM busy
+  const int heads = p.B * p.H_kv;
+  int iters = 1;
+  while (((p.L + iters * kDecodeTile - 1) / (iters * kDecodeTile)) * heads > 2 * ctx->n_sm &&
+         iters * kDecodeTile < p.L)
+    ++iters;
+  p.iters = iters;
+  p.n_splits = (p.L + iters * kDecodeTile - 1) / (iters * kDecodeTile);
+  const cudaError_t e = launch_decode(p, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
+}
+
+const char *sagekv_strerror(int code) {
+  switch (code) {
+    case SAGEKV_OK: return "ok";
+    case SAGEKV_ERR_INVALID: return "invalid argument";
+    case SAGEKV_ERR_ALIGN: return "pointer or stride not aligned";
+    case SAGEKV_ERR_UNSUPPORTED: return "unsupported shape or size";
+    case SAGEKV_ERR_CUDA: return "CUDA runtime error";
+    case SAGEKV_ERR_NOMEM: return "out of memory";
+    default: return "unknown error code";
+  }
+}
+
+int sagekv_last_cuda_error(const sagekv_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+}  // extern "C"

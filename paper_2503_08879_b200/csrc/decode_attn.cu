@@ -226,8 +226,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_attn_kernel(const Decod
         __syncthreads();
       }
       const float outv = lsum > 0.f ? o_cta[0] / lsum : 0.f;
-      reinterpret_cast<__nv_bfloat16_raw *>(p.out)[((int64_t)b * p.H_q + kvh * p.G + h) * kHeadDim + d].x =
-          (unsigned short)(pack_bf16x2(outv, 0.f) & 0xffffu);
+      p.out[((int64_t)b * p.H_q + kvh * p.G + h) * kHeadDim + d] = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
       if (p.lse != nullptr && d == 0)
         p.lse[(int64_t)b * p.H_q + kvh * p.G + h] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
     }

@@ -35,7 +35,7 @@ struct SelShared {
   int scan_tmp[kSelWarps];
   int found[2];
   int list_count;
-  int pad_[3];
+  int pad_[1];
 };
 static_assert(sizeof(SelShared) % 16 == 0, "staged scores must stay 16-byte aligned");
 
