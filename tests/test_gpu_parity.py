@@ -1,0 +1,204 @@
+"""CUDA path vs the CPU oracle, element by element, through the C-ABI binding.
+
+Tolerances (written out once, used everywhere below):
+  scores            |gpu - ref| <= 1e-3 * |ref|            (bf16 products, fp32 sums, approximate exp2)
+  selected indices  bit-exact against the oracle's select run on the GPU's own scores; against the
+                    oracle's select on the oracle's scores the sets may differ only in tokens whose
+                    oracle score is within 1e-3 (relative) of the k-th score
+  gathered K, V     bit-exact given the indices
+  attention output  |gpu - ref| <= 1e-2 + 1e-2 * |ref|     (bf16 output, bf16 softmax weights)
+"""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import sagekv_oracle as O
+from paper_2503_08879_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+SCORE_RTOL = 1e-3
+TIE_BAND = 1e-3
+OUT_ATOL, OUT_RTOL = 1e-2, 1e-2
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2503_08879_b200 import binding
+    return binding
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().contiguous().view(torch.uint16).numpy()
+
+
+def check_scores(gpu_scores, lay, w, b):
+    ref = O.score(bits(lay["q_last"][b]), bits(lay["K"][b]), w.n_init, w.n_recent)
+    got = gpu_scores.view(w.batch, w.n_q_heads, -1)[b, :, : w.E].cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(got, ref, rtol=SCORE_RTOL, atol=1e-30)
+    if w.E > 0:
+        np.testing.assert_allclose(got.sum(axis=1), 1.0, atol=1e-4)
+    return ref, got
+
+
+def check_select(idx_gpu, got_scores, ref_scores, w, k_q):
+    S = w.n_init
+    # (i) same scores in, same indices out
+    want = O.select(got_scores.astype(np.float32), k_q, S)
+    assert np.array_equal(idx_gpu, want)
+    # (ii) against the oracle's own scores: differences only inside the tie band
+    ref_idx = O.select(ref_scores.astype(np.float32), k_q, S)
+    for h in range(idx_gpu.shape[0]):
+        a, r = set(idx_gpu[h].tolist()), set(ref_idx[h].tolist())
+        if a == r:
+            continue
+        kth = np.sort(ref_scores[h])[::-1][k_q - 1]
+        for t in a ^ r:
+            assert abs(ref_scores[h, t - S] - kth) <= TIE_BAND * kth, (h, t)
+    assert np.all(np.diff(idx_gpu, axis=1) > 0)
+
+
+def check_compact(layer, lay, idx_gpu, w, b):
+    Kc_ref, Vc_ref = O.compact(bits(lay["K"][b]), bits(lay["V"][b]), idx_gpu, w.n_init, w.n_recent)
+    Kc, Vc = layer.cache()
+    assert np.array_equal(bits(Kc[b]), Kc_ref) and np.array_equal(bits(Vc[b]), Vc_ref)
+    return Kc_ref, Vc_ref
+
+
+def check_out(out, ref):
+    got = out.float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref)
+    assert np.all(err <= OUT_ATOL + OUT_RTOL * np.abs(ref)), float(err.max())
+
+
+def run_pipeline(B, w, n_decode, device="cuda", strided=False):
+    """All four steps on one layer of workload `w`, every result checked against the oracle."""
+    lay = synth.make_layer(w, 0, device)
+    K, V = lay["K"], lay["V"]
+    if strided:   # token stride 136 and a gap between heads: exercises the stride arguments
+        Kp = torch.zeros(w.batch, w.n_kv_heads, w.n_ctx + 3, 136, dtype=torch.bfloat16, device=device)
+        Vp = torch.zeros_like(Kp)
+        Kp[:, :, : w.n_ctx, :128] = K
+        Vp[:, :, : w.n_ctx, :128] = V
+        K, V = Kp[:, :, : w.n_ctx, :128], Vp[:, :, : w.n_ctx, :128]
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    scores = sk.score(lay["q_last"], K, w.n_init, w.n_recent)
+    layer = sk.select_compact(scores, K, V, w.n_init, w.n_recent, w.n_sel)
+    torch.cuda.synchronize()
+    st = layer.state
+    k_q = min(w.k_q, w.E)
+    assert (st.n_init, st.k_q, st.n_sel, st.n_recent, st.ring_len, st.len) == (
+        w.n_init, k_q, w.G * k_q, w.n_recent, w.n_recent + 1, w.n_init + w.G * k_q + w.n_recent + 1)
+    assert int(layer.step.item()) == 0
+    caches = []
+    for b in range(w.batch):
+        ref_scores, got_scores = check_scores(scores, lay, w, b)
+        idx_gpu = layer.indices()[b].cpu().numpy()
+        if k_q > 0:
+            check_select(idx_gpu, got_scores, ref_scores, w, k_q)
+        caches.append(list(check_compact(layer, lay, idx_gpu, w, b)))
+    # attention with the last token's query and no append, then decode steps with appends
+    lse = torch.empty(w.batch, w.n_q_heads, dtype=torch.float32, device=device)
+    out = sk.decode_attn(lay["q_last"], None, None, layer, lse=lse)
+    torch.cuda.synchronize()
+    for b in range(w.batch):
+        ref, ref_lse, _ = O.decode_step(bits(lay["q_last"][b]), None, None, caches[b][0], caches[b][1], 0,
+                                        w.n_init, k_q, w.n_recent)
+        check_out(out[b], ref)
+        np.testing.assert_allclose(lse[b].cpu().numpy(), ref_lse, rtol=1e-3, atol=1e-3)
+    steps = [0] * w.batch
+    for t in range(n_decode):
+        d = synth.make_decode_inputs(w, 0, t, device)
+        out = sk.decode_attn(d["q"], d["k_new"], d["v_new"], layer)
+        torch.cuda.synchronize()
+        assert int(layer.step.item()) == t + 1
+        for b in range(w.batch):
+            ref, _, steps[b] = O.decode_step(bits(d["q"][b]), bits(d["k_new"][b]), bits(d["v_new"][b]),
+                                             caches[b][0], caches[b][1], steps[b], w.n_init, k_q, w.n_recent)
+            check_out(out[b], ref)
+    Kc, Vc = layer.cache()
+    for b in range(w.batch):   # the window rolled the same way on both sides
+        assert np.array_equal(bits(Kc[b]), caches[b][0]) and np.array_equal(bits(Vc[b]), caches[b][1])
+    sk.close()
+    return lay, layer
+
+
+def test_c1_full_config(B):
+    w = synth.workload("C1")
+    run_pipeline(B, w, n_decode=w.decode_steps)
+
+
+@pytest.mark.parametrize("name,kw,n_decode", [
+    # several score chunks, several cluster CTAs, ragged tails everywhere
+    ("C2", dict(n_ctx=20011), 5),
+    # window shorter than the number of decode steps: the ring wraps twice
+    ("C1", dict(n_ctx=3001, budget=128, n_recent_min=8), 21),
+    # G = 7 with the non-divisible budget split, near-duplicate keys (ties at the threshold), batch 2
+    ("C4-b1", dict(n_ctx=9000, batch=2), 4),
+    # clustered heavy tokens: one CTA of the cluster owns most of the kept rows
+    ("C5-4096", dict(n_ctx=30000, budget=1024, n_recent_min=64), 3),
+    # reduced cache longer than one partition pass: several tiles per CTA in decode
+    ("C3-4096", dict(n_ctx=40000), 3),
+])
+def test_scaled_configs(B, name, kw, n_decode):
+    w = synth.workload(name).with_(n_layers=1, **kw)
+    run_pipeline(B, w, n_decode)
+
+
+def test_strided_cache(B):
+    w = synth.workload("C1").with_(n_ctx=5000)
+    run_pipeline(B, w, 3, strided=True)
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (16, 2), (8, 1)])
+def test_group_sizes(B, hq, hkv):
+    w = synth.workload("C1").with_(n_q_heads=hq, n_kv_heads=hkv, n_ctx=2500, budget=4 + 8 * (hq // hkv) + 16,
+                                   n_recent_min=16)
+    run_pipeline(B, w, 3)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(n_ctx=70, budget=72, n_init=4, n_recent_min=64),      # E = 1, k_q = 1
+    dict(n_ctx=69, budget=72, n_init=4, n_recent_min=64),      # E = 0: the cache is everything
+    dict(n_ctx=100, budget=228, n_init=4, n_recent_min=64),    # k_q = 40 > E = 31: clamped, k_q = E
+    dict(n_ctx=300, budget=24, n_init=4, n_recent_min=20),     # k = 0: sink + recent only
+    dict(n_ctx=300, budget=36, n_init=0, n_recent_min=0),      # no sink, no recent window (ring of 1)
+    dict(n_ctx=2, budget=1, n_init=0, n_recent_min=1),         # two tokens
+])
+def test_degenerate_partitions(B, kw):
+    w = synth.workload("C1").with_(**kw)
+    run_pipeline(B, w, 3)
+
+
+def test_full_size_128k_one_layer(B):
+    """C3 at budget 2048, one layer, the launch configuration the benchmark times."""
+    w = synth.workload("C3-2048")
+    run_pipeline(B, w, 2)
+
+
+def test_full_size_qwen_128k_batch4_sampled(B):
+    """C4 at batch 4: scores and indices checked for one batch entry, caches and outputs for all."""
+    w = synth.workload("C4-b4")
+    dev = "cuda"
+    lay = synth.make_layer(w, 0, dev)
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    scores = sk.score(lay["q_last"], lay["K"], w.n_init, w.n_recent)
+    layer = sk.select_compact(scores, lay["K"], lay["V"], w.n_init, w.n_recent, w.n_sel)
+    d = synth.make_decode_inputs(w, 0, 0, dev)
+    out = sk.decode_attn(d["q"], d["k_new"], d["v_new"], layer)
+    torch.cuda.synchronize()
+    for b in range(w.batch):
+        idx_gpu = layer.indices()[b].cpu().numpy()
+        got = scores.view(w.batch, w.n_q_heads, -1)[b, :, : w.E].cpu().numpy()
+        assert np.array_equal(idx_gpu, O.select(got, w.k_q, w.n_init))
+        if b == 3:
+            ref_scores, got_scores = check_scores(scores, lay, w, b)
+            check_select(idx_gpu, got_scores, ref_scores, w, w.k_q)
+        Kc_ref, Vc_ref = O.compact(bits(lay["K"][b]), bits(lay["V"][b]), idx_gpu, w.n_init, w.n_recent)
+        ref, _, _ = O.decode_step(bits(d["q"][b]), bits(d["k_new"][b]), bits(d["v_new"][b]), Kc_ref, Vc_ref, 0,
+                                  w.n_init, w.k_q, w.n_recent)
+        check_out(out[b], ref)
+        Kc, Vc = layer.cache()
+        assert np.array_equal(bits(Kc[b]), Kc_ref) and np.array_equal(bits(Vc[b]), Vc_ref)
+    sk.close()

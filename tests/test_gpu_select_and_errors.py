@@ -1,0 +1,140 @@
+"""Select on hand-made score rows (ties, constants, negative values, guard bands) and the
+argument-error matrix of the C interface.  Nothing here relies on the score kernel."""
+
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import sagekv_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2503_08879_b200 import binding
+    return binding
+
+
+def bits(t):
+    return t.detach().cpu().contiguous().view(torch.uint16).numpy()
+
+
+def run_select(B, rows: np.ndarray, k_q: int, S=3, R=5, H_kv=None, pad=8):
+    """rows [H_q, E] fp32 -> (idx [H_q, k_q], Kc, Vc, K, V) with random K/V and guard bands checked."""
+    H_q, E = rows.shape
+    H_kv = H_kv or H_q
+    G = H_q // H_kv
+    N = S + E + R + 1
+    g = torch.Generator(device="cuda").manual_seed(1234 + E)
+    K = torch.randn(1, H_kv, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    V = torch.randn(1, H_kv, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    stride = (E + 3) // 4 * 4 + pad
+    buf = torch.full((H_q, stride), 7.5, dtype=torch.float32, device="cuda")
+    buf[:, :E] = torch.from_numpy(rows).cuda()
+    sk = B.SageKV(H_q, H_kv, 128, 1, max_ctx=N, max_len=S + G * k_q + R + 1)
+    layer = sk.new_layer(S, R, G * k_q)
+    canary = 0x5A5A
+    layer.Kc.view(torch.int16).fill_(canary)
+    layer.Vc.view(torch.int16).fill_(canary)
+    layer.idx.fill_(-77)
+    before = buf.clone()
+    sk.select_compact(buf, K, V, S, R, G * k_q, layer)
+    torch.cuda.synchronize()
+    assert torch.equal(before, buf)                       # scores are read-only, padding untouched
+    kk = min(k_q, E)
+    idx = layer.indices()[0].cpu().numpy()
+    assert layer.idx.flatten()[H_q * kk:].eq(-77).all()   # nothing written past the used part
+    Kc_ref, Vc_ref = O.compact(bits(K[0]), bits(V[0]), idx, S, R)
+    Kc, Vc = layer.cache()
+    assert np.array_equal(bits(Kc[0]), Kc_ref) and np.array_equal(bits(Vc[0]), Vc_ref)
+    sk.close()
+    return idx
+
+
+@pytest.mark.parametrize("E,k_q", [(1, 1), (5, 2), (33, 33), (600, 7), (2049, 100), (5000, 64), (16385, 479),
+                                   (40000, 1000), (70001, 1983)])
+def test_select_random_rows_bit_exact(B, E, k_q):
+    rng = np.random.default_rng(E)
+    rows = rng.random((4, E), dtype=np.float32) ** 8       # skewed like softmax rows
+    idx = run_select(B, rows, k_q, H_kv=2)
+    assert np.array_equal(idx, O.select(rows, k_q, 3))
+
+
+def test_select_ties_lowest_position_wins(B):
+    E = 9000
+    rng = np.random.default_rng(5)
+    rows = np.empty((6, E), dtype=np.float32)
+    rows[0] = 0.25                                          # every score equal
+    rows[1] = rng.integers(0, 3, E)                         # three distinct values
+    rows[2] = rng.integers(0, 50, E) / 64.0
+    rows[3] = np.where(rng.random(E) < 0.01, 1.0, 0.5)      # few large, threshold inside a huge tie
+    rows[4] = rng.standard_normal(E)                        # negative values order correctly
+    rows[5] = -np.abs(rng.standard_normal(E)); rows[5, ::7] = -0.0; rows[5, 3::7] = 0.0
+    for k_q in (1, 17, 300, 4500, 9000):
+        idx = run_select(B, rows, k_q, H_kv=3)
+        assert np.array_equal(idx, O.select(rows, k_q, 3))
+
+
+def test_select_threshold_differs_only_in_low_bits(B):
+    E = 20000
+    base = np.float32(0.001)
+    ulps = np.random.default_rng(6).integers(0, 40, (2, E)).astype(np.uint32)
+    rows = (np.full((2, E), base, dtype=np.float32).view(np.uint32) + ulps).view(np.float32)
+    for k_q in (5, 999):
+        assert np.array_equal(run_select(B, rows, k_q), O.select(rows, k_q, 3))
+
+
+def test_select_is_deterministic(B):
+    rows = np.random.default_rng(8).random((4, 30000), dtype=np.float32)
+    a = run_select(B, rows, 479, H_kv=1)
+    b = run_select(B, rows, 479, H_kv=1)
+    assert np.array_equal(a, b)
+
+
+def test_argument_errors_are_reported_before_launch(B):
+    lib, C = B.lib, ctypes
+    sk = B.SageKV(8, 2, 128, 1, max_ctx=1000, max_len=200)
+    K = torch.zeros(1, 2, 1000, 128, dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros(1, 8, 128, dtype=torch.bfloat16, device="cuda")
+    sc = torch.zeros(8, 1000, dtype=torch.float32, device="cuda")
+    layer = sk.new_layer(4, 16, 32)
+    code = lambda f, *a: pytest.raises(B.SagekvError, f, *a).value.code
+    # score
+    assert code(B.sagekv_score, sk.ctx, None, K, 1000, 4, 16, sc, 1000) == B.ERR_INVALID
+    assert code(B.sagekv_score, sk.ctx, q, K, 1000, 600, 400, sc, 1000) == B.ERR_INVALID      # S+R+1 > N
+    assert code(B.sagekv_score, sk.ctx, q, K, 1000, -1, 16, sc, 1000) == B.ERR_INVALID
+    assert code(B.sagekv_score, sk.ctx, q, K, 1000, 4, 16, sc, 500) == B.ERR_INVALID          # row stride < E
+    assert code(B.sagekv_score, sk.ctx, q, K, 1000, 4, 16, sc, 998) == B.ERR_ALIGN            # stride % 4
+    assert code(B.sagekv_score, sk.ctx, q, K, 2000, 4, 16, sc, 2000) == B.ERR_UNSUPPORTED     # beyond max_ctx
+    assert code(B.sagekv_score, sk.ctx, q.view(-1)[4:].view(-1), K, 1000, 4, 16, sc, 1000) == B.ERR_ALIGN
+    # select_compact
+    sel = lambda **kw: B.sagekv_select_compact(sk.ctx, kw.get("sc", sc), kw.get("stride", 1000), K, K, 1000,
+                                               kw.get("S", 4), kw.get("R", 16), kw.get("k", 32), layer.idx,
+                                               layer.Kc, layer.Vc, layer.state)
+    assert pytest.raises(B.SagekvError, sel, k=30).value.code == B.ERR_INVALID                # k % G != 0
+    assert pytest.raises(B.SagekvError, sel, k=-4).value.code == B.ERR_INVALID
+    assert pytest.raises(B.SagekvError, sel, S=990).value.code == B.ERR_INVALID
+    assert pytest.raises(B.SagekvError, sel, k=400).value.code == B.ERR_UNSUPPORTED           # L > max_len
+    assert pytest.raises(B.SagekvError, sel, sc=None).value.code == B.ERR_INVALID
+    # decode
+    sel()
+    out = torch.empty_like(q)
+    kn = torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda")
+    assert code(B.sagekv_decode_attn, sk.ctx, q, kn, None, layer.Kc, layer.Vc, layer.state, out) == B.ERR_INVALID
+    assert code(B.sagekv_decode_attn, sk.ctx, None, None, None, layer.Kc, layer.Vc, layer.state, out) == B.ERR_INVALID
+    bad = B.CacheState(4, 8, 32, 16, 17, 99, layer.step.data_ptr())                           # len inconsistent
+    assert code(B.sagekv_decode_attn, sk.ctx, q, None, None, layer.Kc, layer.Vc, bad, out) == B.ERR_INVALID
+    B.sagekv_decode_attn(sk.ctx, q, None, None, layer.Kc, layer.Vc, layer.state, out)
+    torch.cuda.synchronize()                                                                   # context still healthy
+    # create
+    h = C.c_void_p()
+    shp = B.Shape(8, 2, 64, 1, 0.0)
+    assert lib.sagekv_create(C.byref(h), C.byref(shp), 1000, 100) == B.ERR_UNSUPPORTED and not h.value
+    shp = B.Shape(32, 2, 128, 1, 0.0)
+    assert lib.sagekv_create(C.byref(h), C.byref(shp), 1000, 100) == B.ERR_UNSUPPORTED        # G = 16
+    shp = B.Shape(8, 3, 128, 1, 0.0)
+    assert lib.sagekv_create(C.byref(h), C.byref(shp), 1000, 100) == B.ERR_INVALID
+    sk.close()
