@@ -120,7 +120,7 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
  *           (Step 3: C = Concat(S, E_topk, R, P_N)).  Rows are bit-exact copies.
  *   state   host struct, filled on return; state->d_step must already point to
  *           a device int32, which is set to 0 on the stream.
- * Comparisons are made on the fp32 bit patterns given; scores must not be NaN.
+ * Scores are compared as IEEE numbers (-0 equals +0); they must not be NaN.
  * Errors: INVALID (null, k < 0, k % G != 0, bad partition), ALIGN,
  * UNSUPPORTED (L above the context's max_len), CUDA. */
 int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_row_stride,

@@ -40,7 +40,7 @@ struct SelShared {
 static_assert(sizeof(SelShared) % 16 == 0, "staged scores must stay 16-byte aligned");
 
 __device__ __forceinline__ uint32_t score_key(float x) {
-  const uint32_t u = __float_as_uint(x);
+  const uint32_t u = __float_as_uint(x + 0.0f);         // -0 becomes +0: the two compare equal as numbers
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);   // larger float <=> larger unsigned key
 }
 
