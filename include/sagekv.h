@@ -41,7 +41,8 @@ enum {
   SAGEKV_ERR_ALIGN = -2,       /* pointer or stride breaks the alignment rules above     */
   SAGEKV_ERR_UNSUPPORTED = -3, /* head_dim != 128, G > 8, size beyond the context's max  */
   SAGEKV_ERR_CUDA = -4,        /* a CUDA runtime call failed (see sagekv_last_cuda_error) */
-  SAGEKV_ERR_NOMEM = -5        /* scratch allocation failed in sagekv_create             */
+  SAGEKV_ERR_NOMEM = -5,       /* scratch allocation failed in sagekv_create             */
+  SAGEKV_ERR_TOO_LARGE = -6    /* problem exceeds the fixed scratch of sagekv_score_static */
 };
 
 typedef struct sagekv_ctx sagekv_ctx; /* opaque; owns only its scratch memory */
@@ -148,6 +149,30 @@ int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_r
 int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const void *v_new,
                        void *Kc, void *Vc, sagekv_strides cs, const sagekv_cache_state *state,
                        void *out, float *lse, void *stream);
+
+/* The score step without any allocation (the paper has no counterpart: this is
+ * a deployment variant of sagekv_score, same arithmetic, same kernels, same
+ * output).  It exists for programs that cannot call cudaMalloc when they reach
+ * this step: inference servers hand nearly all device memory to their own
+ * cache manager at start-up, so the cudaMalloc inside sagekv_create may fail
+ * there, and it synchronises the whole device, which a serving loop with other
+ * streams in flight cannot afford.  This call needs no context: the softmax
+ * partials live in a fixed 256 KiB array inside the library image (present on
+ * every GPU that loads the library, until the process ends).
+ *   - Limit: batch * H_q * ceil(E / 256) <= 32768 partial entries; beyond it the
+ *     call returns SAGEKV_ERR_TOO_LARGE and launches nothing (E = 131072-class
+ *     contexts fit up to batch * H_q = 64).
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and caches it; make that first call outside any
+ *     stream capture.  Later calls only launch.
+ *   - All calls on a device share the array.  It needs no clearing (each entry
+ *     is written before it is read within a call), but two calls whose kernels
+ *     overlap on the GPU (different streams) race on it: keep them ordered.
+ * Arguments, layouts, alignment rules and the other error codes are those of
+ * sagekv_score, with `shape` taking the place of the context. */
+int sagekv_score_static(const sagekv_shape *shape, const void *q_last, const void *K, sagekv_strides ks,
+                        int64_t n_ctx, int32_t n_init, int32_t n_recent,
+                        float *scores, int64_t scores_row_stride, void *stream);
 
 /* Text for a return code; never NULL.  Static storage. */
 const char *sagekv_strerror(int code);

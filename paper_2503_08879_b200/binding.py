@@ -23,6 +23,7 @@ if not os.path.exists(_LIB_PATH):
 lib = C.CDLL(_LIB_PATH)
 
 OK, ERR_INVALID, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
+ERR_TOO_LARGE = -6
 
 
 class Shape(C.Structure):
@@ -47,6 +48,8 @@ lib.sagekv_score.argtypes = [_vp, _vp, _vp, Strides, _i64, _i32, _i32, _vp, _i64
 lib.sagekv_select_compact.argtypes = [_vp, _vp, _i64, _vp, _vp, Strides, _i64, _i32, _i32, _i32,
                                       _vp, _vp, _vp, Strides, C.POINTER(CacheState), _vp]
 lib.sagekv_decode_attn.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, Strides, C.POINTER(CacheState), _vp, _vp, _vp]
+lib.sagekv_score_static.argtypes = [C.POINTER(Shape), _vp, _vp, Strides, _i64, _i32, _i32, _vp, _i64, _vp]
+lib.sagekv_score_static.restype = C.c_int
 lib.sagekv_strerror.argtypes = [C.c_int]
 lib.sagekv_strerror.restype = C.c_char_p
 lib.sagekv_last_cuda_error.argtypes = [_vp]
@@ -105,6 +108,13 @@ def sagekv_destroy(ctx):
 def sagekv_score(ctx, q_last, K, n_ctx: int, n_init: int, n_recent: int, scores, scores_row_stride: int):
     _check(lib.sagekv_score(ctx, _ptr(q_last), _ptr(K), _kv_strides(K), n_ctx, n_init, n_recent, _ptr(scores),
                             scores_row_stride, _stream()), "sagekv_score", ctx)
+
+
+def sagekv_score_static(shape: Shape, q_last, K, n_ctx: int, n_init: int, n_recent: int, scores,
+                        scores_row_stride: int):
+    """sagekv_score without a context or any allocation: the partials live in the library's fixed array."""
+    _check(lib.sagekv_score_static(C.byref(shape), _ptr(q_last), _ptr(K), _kv_strides(K), n_ctx, n_init, n_recent,
+                                   _ptr(scores), scores_row_stride, _stream()), "sagekv_score_static")
 
 
 def sagekv_select_compact(ctx, scores, scores_row_stride: int, K, V, n_ctx: int, n_init: int, n_recent: int, k: int,

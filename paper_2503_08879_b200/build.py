@@ -11,7 +11,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsagekv.so")
-SOURCES = ["api.cu", "score.cu", "select_compact.cu", "decode_attn.cu"]
+SOURCES = ["api.cu", "score.cu", "score_static.cu", "select_compact.cu", "decode_attn.cu"]
 
 
 def nvcc_path() -> str:

@@ -243,6 +243,7 @@ const char *sagekv_strerror(int code) {
     case SAGEKV_ERR_UNSUPPORTED: return "unsupported shape or size";
     case SAGEKV_ERR_CUDA: return "CUDA runtime error";
     case SAGEKV_ERR_NOMEM: return "out of memory";
+    case SAGEKV_ERR_TOO_LARGE: return "problem larger than the fixed scratch array";
     default: return "unknown error code";
   }
 }
