@@ -15,7 +15,7 @@ struct sagekv_ctx {
   float scale;
   float2 *score_partials;   // [B*H_q, ceil(max_ctx / kScoreChunk)]
   int max_chunks;
-  float *decode_partials;   // [B*H_kv, max_splits, kPartialStride]
+  float *decode_partials;   // [B*H_kv, max_splits (clusters per head), kPartialStride]
   int max_splits;
   int32_t *tickets;         // [B*H_kv + 1], zero between launches
   int last_cuda_error;
@@ -61,7 +61,10 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   }
   ctx->n_sm = prop.multiProcessorCount;
   ctx->max_chunks = (int)((max_ctx + kScoreChunk - 1) / kScoreChunk);
-  ctx->max_splits = (max_len + kDecodeTile - 1) / kDecodeTile;
+  {
+    int cs, n_warps, smem;
+    decode_geometry(max_len, &ctx->max_splits, &cs, &n_warps, &smem);   // clusters per head at the largest L
+  }
   const size_t n_rows = (size_t)shape->batch * shape->n_q_heads;
   const size_t n_heads = (size_t)shape->batch * shape->n_kv_heads;
   cudaError_t e = cudaMalloc(&ctx->score_partials, n_rows * ctx->max_chunks * sizeof(float2));
@@ -70,6 +73,7 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   if (e == cudaSuccess) e = cudaMalloc(&ctx->tickets, (n_heads + 1) * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(ctx->tickets, 0, (n_heads + 1) * sizeof(int32_t));
   if (e == cudaSuccess) e = select_compact_setup();
+  if (e == cudaSuccess) e = decode_setup();
   if (e != cudaSuccess) {
     cudaFree(ctx->score_partials);
     cudaFree(ctx->decode_partials);
@@ -223,14 +227,6 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
   p.H_kv = ctx->shape.n_kv_heads;
   p.B = ctx->shape.batch;
   p.scale_log2 = ctx->scale * kLog2e;
-  // partitions of iters*64 rows: as many CTAs as keep about two per SM busy
-  const int heads = p.B * p.H_kv;
-  int iters = 1;
-  while (((p.L + iters * kDecodeTile - 1) / (iters * kDecodeTile)) * heads > 2 * ctx->n_sm &&
-         iters * kDecodeTile < p.L)
-    ++iters;
-  p.iters = iters;
-  p.n_splits = (p.L + iters * kDecodeTile - 1) / (iters * kDecodeTile);
   const cudaError_t e = launch_decode(p, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
 }

@@ -47,9 +47,9 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
 cudaError_t select_compact_setup();   // one-time function attributes
 
 // ---- decode attention ------------------------------------------------------
-constexpr int kDecodeWarps = 4;
-constexpr int kDecodeTile = kDecodeWarps * 16;                         // tokens per CTA iteration
-constexpr int kPartialStride = kMaxGroup * kHeadDim + 2 * kMaxGroup;   // floats per split partial: O[8][128], m[8], l[8]
+constexpr int kDecodeMaxWarps = 16;                                    // warps per CTA, one or two 16-row tiles each
+constexpr int kDecodeMaxTiles = 24;                                    // 16-row tiles (K and V) a CTA can stage: 192 KB
+constexpr int kPartialStride = kMaxGroup * kHeadDim + 2 * kMaxGroup;   // floats per cluster result: O[8][128], m[8], l[8]
 
 struct DecodeParams {
   const uint16_t *q;       // [B, H_q, 128]
@@ -59,14 +59,15 @@ struct DecodeParams {
   sagekv_strides cs;
   uint16_t *out;           // [B, H_q, 128]
   float *lse;              // [B, H_q] or null
-  float *partials;         // [B*H_kv, n_splits, kPartialStride]
+  float *partials;         // [B*H_kv, clusters per head, kPartialStride]; used only with several clusters per head
   int32_t *tickets;        // [B*H_kv] arrival counters + [1] finished-heads counter, all 0 between launches
   int32_t *d_step;
-  int n_splits, iters;     // every split covers iters * kDecodeTile rows
   int S, k_q, n_sel, ring_len, L, G, H_q, H_kv, B;
   float scale_log2;
 };
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream);
+cudaError_t decode_setup();           // one-time function attributes
+void decode_geometry(int L, int *n_clusters, int *cluster_size, int *n_warps, int *smem_bytes);
 
 // ---- device helpers --------------------------------------------------------
 #if defined(__CUDACC__)

@@ -1,25 +1,35 @@
 // Step 4: append the new token to the recent window, then attention of every query head over its view
 // of the reduced cache (sink + its own selected segment + window).
 //
-// Flash-decoding layout: the L rows of a KV head are cut into n_splits partitions; one CTA per
-// (partition, KV head, batch entry) streams its K and V rows once, straight from global memory into
-// tensor-core fragments, and keeps a running softmax.  Per 16-row tile of a warp
-//   S^T = Q K^T   heads (padded to 16) x 8 rows per mma; lane (g, c) loads 16-byte pieces of rows g and
-//                 g+8 and the query fragment uses the same column permutation, so no shuffle or shared
-//                 memory is needed to form the fragments;
-//   O^T += V^T P  head_dim x heads; the lane that owns logits of rows {2c, 2c+1, 2c+8, 2c+9} for head g
-//                 (the accumulator layout of the first product) is exactly the lane that must supply
-//                 those rows' weights for head g as the B fragment, and it loads the same four V rows
-//                 at 16 columns of its own, pairing two rows per register with a byte permute.
-// Every head masks the rows of the other heads' segments.  The partition results (max, sum, O) go to
-// scratch; the CTA that arrives last for a KV head (one atomic ticket, no waiting) merges them by
-// log-sum-exp and writes bf16 output.  The new token's row is taken from k_new / v_new by whichever
-// lane would have read the window slot it replaces, and the CTA owning that slot stores it.
+// Flash-decoding on thread-block clusters.  The L rows of one KV head are cut into 16-row tiles that are
+// dealt evenly to the CTAs of one cluster (more clusters per head only when L exceeds what a cluster's
+// shared memory holds).  Every warp owns one or two tiles.  It first issues 16-byte cp.async copies for
+// all its K and V rows, so the whole partition is in flight at once and costs no registers, then works
+// through its tiles as they land:
+//   S^T = Q K^T   heads (padded to 16) x 8 rows per mma.  Lane (g, c) reads 16-byte pieces of rows g and
+//                 g+8; the query fragment uses the same column permutation, so fragments come straight
+//                 from the staged rows with no transposition.
+//   O^T += V^T P  head_dim x heads.  The accumulator layout of the first product puts the weights of rows
+//                 {2c, 2c+1, 2c+8, 2c+9} for head g in lane (g, c), which is exactly the B fragment of the
+//                 second; the lane reads the same four V rows at 16 columns of its own and pairs two rows
+//                 per register with a byte permute.
+// The staged rows are XOR-swizzled so that both access patterns are free of bank conflicts.  Every head
+// masks the rows of the other heads' segments.  Warps are merged through shared memory, the CTAs of a
+// cluster through distributed shared memory (each CTA finishes a slice of the 128 columns), so with one
+// cluster per head nothing touches global scratch.  With several clusters per head the cluster results
+// go to scratch and the CTA that arrives last (one atomic ticket, no waiting) merges them.
+// The new token's row is read from k_new / v_new by whichever lane would have read the window slot it
+// replaces, and the CTA owning that slot stores it into the cache.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace sagekv {
 
-constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kTileBytes = 16 * 256;           // 16 rows of K (or V)
+constexpr int kResFloats = kMaxGroup * kHeadDim + 2 * kMaxGroup;
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
   uint32_t r;
@@ -31,9 +41,33 @@ __device__ __forceinline__ uint32_t reg_of(const uint4 &v, int i) {
   return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
 }
 
-__global__ void __launch_bounds__(kDecodeThreads) decode_attn_kernel(const DecodeParams p) {
-  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+// 16-byte piece `piece` of row `row` of a staged tile lives at piece ^ swz(row): rows g and g+1 land in
+// different halves of the 128-byte bank window (K fragment reads), rows 2c apart in different quarters
+// (V fragment reads).
+__device__ __forceinline__ int swz(int row) { return ((row & 1) << 2) ^ (((row >> 1) & 3) << 1); }
+
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+__global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const DecodeParams p) {
+  extern __shared__ __align__(128) unsigned char stage[];          // tiles: [K 4 KB | V 4 KB] each
+  __shared__ float res[kResFloats];                                 // this CTA's O[8][128], m[8], l[8]
+  __shared__ float sm_m[kDecodeMaxWarps][kMaxGroup], sm_l[kDecodeMaxWarps][kMaxGroup];
+  __shared__ int sm_last;
+
+  cg::cluster_group cluster = cg::this_cluster();
+  const int cs = cluster.num_blocks();
+  const int rank = cluster.block_rank();
+  const int ci = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;      // ci: CTA index within the head
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_warps = blockDim.x >> 5;
   const int g = lane >> 2, c = lane & 3;
   const bool append = p.k_new != nullptr;
 
@@ -42,11 +76,45 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_attn_kernel(const Decod
     step = *reinterpret_cast<const volatile int32_t *>(p.d_step);
     slot = p.S + p.n_sel + step % p.ring_len;
   }
-
   const uint16_t *Kh = p.Kc + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride;
   const uint16_t *Vh = p.Vc + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride;
   const uint16_t *kn = append ? p.k_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
   const uint16_t *vn = append ? p.v_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
+
+  // tiles of this CTA: an even deal of the head's n_tiles over the gridDim.x CTAs
+  const int n_tiles = (p.L + 15) >> 4;
+  const int base_n = n_tiles / (int)gridDim.x, rem = n_tiles % (int)gridDim.x;
+  const int first_tile = ci * base_n + min(ci, rem);
+  const int my_tiles = base_n + (ci < rem ? 1 : 0);
+  const int n_mine = warp < my_tiles ? (my_tiles - warp + n_warps - 1) / n_warps : 0;   // tiles of this warp: 0, 1 or 2
+
+  // ---- issue every copy of this warp's tiles ----
+  const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(stage);
+  for (int i = 0; i < n_mine; ++i) {
+    const int lt = warp + i * n_warps;
+    const int row0 = (first_tile + lt) << 4;
+    const uint32_t tk = stage_base + lt * 2 * kTileBytes, tv = tk + kTileBytes;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int flat = u * 32 + lane, row = flat >> 4, piece = flat & 15;
+      const int r = min(row0 + row, p.L - 1);
+      const uint32_t off = row * 256 + ((piece ^ swz(row)) << 4);
+      cp_async16(tk + off, (r == slot ? kn : Kh + (int64_t)r * p.cs.token_stride) + piece * 8);
+      cp_async16(tv + off, (r == slot ? vn : Vh + (int64_t)r * p.cs.token_stride) + piece * 8);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+
+  // the CTA that owns the replaced window slot stores the new token's row
+  if (append && warp == 0) {
+    const int st = slot >> 4;
+    if (st >= first_tile && st < first_tile + my_tiles) {
+      const uint16_t *src = (lane < 16 ? kn : vn) + (lane & 15) * 8;
+      uint16_t *dst = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
+                      (int64_t)slot * p.cs.token_stride + (lane & 15) * 8;
+      st_v4(dst, ld_v4(src));
+    }
+  }
 
   // A fragments of Q: head g in row g of the tile, rows 8..15 are padding
   uint4 qf[4];
@@ -62,41 +130,31 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_attn_kernel(const Decod
 
   float m_run = -INFINITY;   // running max of head g (log2 units), equal in the 4 lanes of a group
   float l_run = 0.f;         // this lane's share of the running sum of head g
-  float acc[8][4];           // O^T: [m-tile][(d_a,h 2c), (d_a,h 2c+1), (d_b,h 2c), (d_b,h 2c+1)]
+  float acc[8][4];           // O^T: [m-tile][(d_a,h 2c), (d_a,h 2c+1), (d_a+1,h 2c), (d_a+1,h 2c+1)]
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
 
-  const int split_lo = split * p.iters * kDecodeTile;
-  for (int it = 0; it < p.iters; ++it) {
-    const int base = split_lo + it * kDecodeTile + warp * 16;
-    if (base >= p.L) break;    // warp-uniform
-    // ---- loads: K rows g, g+8 (4 pieces each); V rows 2c, 2c+1, 2c+8, 2c+9 (2 pieces each) ----
-    uint4 ka[4], kb[4], vv[4][2];
-    {
-      const int r0 = min(base + g, p.L - 1), r1 = min(base + g + 8, p.L - 1);
-      const uint16_t *pa = (r0 == slot ? kn : Kh + (int64_t)r0 * p.cs.token_stride) + c * 8;
-      const uint16_t *pb = (r1 == slot ? kn : Kh + (int64_t)r1 * p.cs.token_stride) + c * 8;
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        ka[jj] = ld_v4(pa + jj * 32);
-        kb[jj] = ld_v4(pb + jj * 32);
-      }
-#pragma unroll
-      for (int s = 0; s < 4; ++s) {
-        const int r = min(base + 2 * c + (s & 1) + (s >> 1) * 8, p.L - 1);
-        const uint16_t *pv = (r == slot ? vn : Vh + (int64_t)r * p.cs.token_stride) + g * 8;
-        vv[s][0] = ld_v4(pv);
-        vv[s][1] = ld_v4(pv + 64);
-      }
-    }
+  for (int i = 0; i < n_mine; ++i) {
+    if (i + 1 < n_mine) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    const int lt = warp + i * n_warps;
+    const int base = (first_tile + lt) << 4;
+    const uint32_t tk = stage_base + lt * 2 * kTileBytes, tv = tk + kTileBytes;
     // ---- S^T = Q K^T for rows base..base+7 (s0,s1) and base+8..base+15 (s2,s3) ----
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+    {
+      const uint32_t ra = tk + g * 256, rb = tk + (g + 8) * 256;
+      const int sa = swz(g), sb = swz(g + 8);
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-      mma_bf16_16816(s0, s1, z0, z1, qf[jj].x, 0u, qf[jj].y, 0u, ka[jj].x, ka[jj].y);
-      mma_bf16_16816(s0, s1, z0, z1, qf[jj].z, 0u, qf[jj].w, 0u, ka[jj].z, ka[jj].w);
-      mma_bf16_16816(s2, s3, z2, z3, qf[jj].x, 0u, qf[jj].y, 0u, kb[jj].x, kb[jj].y);
-      mma_bf16_16816(s2, s3, z2, z3, qf[jj].z, 0u, qf[jj].w, 0u, kb[jj].z, kb[jj].w);
+      for (int jj = 0; jj < 4; ++jj) {
+        const uint4 ka = lds_v4(ra + (((c + 4 * jj) ^ sa) << 4));
+        const uint4 kb = lds_v4(rb + (((c + 4 * jj) ^ sb) << 4));
+        mma_bf16_16816(s0, s1, z0, z1, qf[jj].x, 0u, qf[jj].y, 0u, ka.x, ka.y);
+        mma_bf16_16816(s0, s1, z0, z1, qf[jj].z, 0u, qf[jj].w, 0u, ka.z, ka.w);
+        mma_bf16_16816(s2, s3, z2, z3, qf[jj].x, 0u, qf[jj].y, 0u, kb.x, kb.y);
+        mma_bf16_16816(s2, s3, z2, z3, qf[jj].z, 0u, qf[jj].w, 0u, kb.z, kb.w);
+      }
     }
     float sv[4] = {s0 * p.scale_log2, s1 * p.scale_log2, s2 * p.scale_log2, s3 * p.scale_log2};
     float tile_max = -INFINITY;
@@ -123,124 +181,134 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_attn_kernel(const Decod
     // rescale factors of heads 2c and 2c+1 live in the lanes of groups 2c and 2c+1
     const float al0 = __shfl_sync(0xffffffffu, alpha, (2 * c) * 4);
     const float al1 = __shfl_sync(0xffffffffu, alpha, (2 * c + 1) * 4);
-    // ---- O^T += V^T P ----
+    // ---- O^T += V^T P: rows 2c, 2c+1, 2c+8, 2c+9 at columns 8g..8g+7 and 64+8g..64+8g+7 ----
+    uint32_t vrow[4];
+    int vs[4];
 #pragma unroll
-    for (int mt = 0; mt < 8; ++mt) {
-      const int piece = mt >> 2, reg = mt & 3;           // columns 8g + 2*reg (+1) of piece 0, 64 + ... of piece 1
-      const uint32_t v0 = reg_of(vv[0][piece], reg), v1 = reg_of(vv[1][piece], reg);
-      const uint32_t v2 = reg_of(vv[2][piece], reg), v3 = reg_of(vv[3][piece], reg);
-      acc[mt][0] *= al0; acc[mt][1] *= al1; acc[mt][2] *= al0; acc[mt][3] *= al1;
-      mma_bf16_16816(acc[mt][0], acc[mt][1], acc[mt][2], acc[mt][3], prmt(v0, v1, 0x5410u), prmt(v0, v1, 0x7632u),
-                     prmt(v2, v3, 0x5410u), prmt(v2, v3, 0x7632u), pb0, pb1);
+    for (int s = 0; s < 4; ++s) {
+      const int row = 2 * c + (s & 1) + (s >> 1) * 8;
+      vrow[s] = tv + row * 256;
+      vs[s] = swz(row);
+    }
+#pragma unroll
+    for (int piece = 0; piece < 2; ++piece) {
+      uint4 vv[4];
+#pragma unroll
+      for (int s = 0; s < 4; ++s) vv[s] = lds_v4(vrow[s] + (((g + 8 * piece) ^ vs[s]) << 4));
+#pragma unroll
+      for (int reg = 0; reg < 4; ++reg) {
+        const int mt = piece * 4 + reg;                  // columns piece*64 + 8g + 2*reg (+1)
+        const uint32_t v0 = reg_of(vv[0], reg), v1 = reg_of(vv[1], reg);
+        const uint32_t v2 = reg_of(vv[2], reg), v3 = reg_of(vv[3], reg);
+        acc[mt][0] *= al0; acc[mt][1] *= al1; acc[mt][2] *= al0; acc[mt][3] *= al1;
+        mma_bf16_16816(acc[mt][0], acc[mt][1], acc[mt][2], acc[mt][3], prmt(v0, v1, 0x5410u), prmt(v0, v1, 0x7632u),
+                       prmt(v2, v3, 0x5410u), prmt(v2, v3, 0x7632u), pb0, pb1);
+      }
     }
   }
 
-  // ---- merge the warps of the CTA ----
-  __shared__ float sm_m[kDecodeWarps][kMaxGroup], sm_l[kDecodeWarps][kMaxGroup];
-  __shared__ float sm_o[kDecodeWarps][kMaxGroup][kHeadDim];
-  __shared__ float sm_w[kMaxGroup * 64];   // merge weights of the last-arriving CTA
-  __shared__ int sm_last;
+  // ---- merge the warps of the CTA (the staging area is reused for the exchange) ----
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
   if (c == 0) { sm_m[warp][g] = m_run; sm_l[warp][g] = l_run; }
-  __syncthreads();
-  {
+  __syncthreads();                                       // also: every warp is done reading its tiles
+  const int n_act = min(n_warps, my_tiles);              // warps that had a tile
+  float *xo = reinterpret_cast<float *>(stage);          // [n_act][8][128]
+  if (warp < n_act) {
     const int h0 = 2 * c, h1 = 2 * c + 1;
     float M0 = -INFINITY, M1 = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < kDecodeWarps; ++w) { M0 = fmaxf(M0, sm_m[w][h0]); M1 = fmaxf(M1, sm_m[w][h1]); }
+    for (int w = 0; w < n_act; ++w) { M0 = fmaxf(M0, sm_m[w][h0]); M1 = fmaxf(M1, sm_m[w][h1]); }
     const float f0 = M0 == -INFINITY ? 0.f : fast_exp2(sm_m[warp][h0] - M0);
     const float f1 = M1 == -INFINITY ? 0.f : fast_exp2(sm_m[warp][h1] - M1);
+    float *mine0 = xo + (warp * kMaxGroup + h0) * kHeadDim, *mine1 = xo + (warp * kMaxGroup + h1) * kHeadDim;
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
       const int d_a = (mt >> 2) * 64 + g * 8 + (mt & 3) * 2;
-      sm_o[warp][h0][d_a] = acc[mt][0] * f0;
-      sm_o[warp][h1][d_a] = acc[mt][1] * f1;
-      sm_o[warp][h0][d_a + 1] = acc[mt][2] * f0;
-      sm_o[warp][h1][d_a + 1] = acc[mt][3] * f1;
+      mine0[d_a] = acc[mt][0] * f0;
+      mine1[d_a] = acc[mt][1] * f1;
+      mine0[d_a + 1] = acc[mt][2] * f0;
+      mine1[d_a + 1] = acc[mt][3] * f1;
     }
   }
   __syncthreads();
-  // thread d owns column d of every head from here on
-  const int d = tid;
-  float o_cta[kMaxGroup], m_cta[kMaxGroup], l_cta[kMaxGroup];
-#pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) {
-    float M = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < kDecodeWarps; ++w) M = fmaxf(M, sm_m[w][h]);
-    float l = 0.f, o = 0.f;
-#pragma unroll
-    for (int w = 0; w < kDecodeWarps; ++w) {
-      l += M == -INFINITY ? 0.f : sm_l[w][h] * fast_exp2(sm_m[w][h] - M);
-      o += sm_o[w][h][d];
+  for (int item = tid; item < kMaxGroup * kHeadDim; item += blockDim.x) {
+    const int h = item >> 7;
+    float o = 0.f;
+    for (int w = 0; w < n_act; ++w) o += xo[w * kMaxGroup * kHeadDim + item];
+    res[item] = o;
+    if ((item & 127) == 0) {
+      float M = -INFINITY, l = 0.f;
+      for (int w = 0; w < n_act; ++w) M = fmaxf(M, sm_m[w][h]);
+      for (int w = 0; w < n_act; ++w) l += M == -INFINITY ? 0.f : sm_l[w][h] * fast_exp2(sm_m[w][h] - M);
+      res[kMaxGroup * kHeadDim + h] = M;
+      res[kMaxGroup * kHeadDim + kMaxGroup + h] = l;
     }
-    m_cta[h] = M; l_cta[h] = l; o_cta[h] = o;
   }
+  cluster.sync();
 
-  // the CTA that owns the replaced window slot stores the new token's row
-  if (append && slot >= split_lo && slot < split_lo + p.iters * kDecodeTile && tid < 32) {
-    const uint16_t *src = (lane < 16 ? kn : vn) + (lane & 15) * 8;
-    uint16_t *dst = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
-                    (int64_t)slot * p.cs.token_stride + (lane & 15) * 8;
-    st_v4(dst, ld_v4(src));
-  }
-
+  // ---- merge the CTAs of the cluster: this CTA finishes columns [rank*cols, (rank+1)*cols) of every head ----
+  const int cols = kHeadDim / cs;
   const int bk = b * p.H_kv + kvh;
-  if (p.n_splits > 1) {
-    float *part = p.partials + ((int64_t)bk * p.n_splits + split) * kPartialStride;
-#pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h)
-      if (h < p.G) part[h * kHeadDim + d] = o_cta[h];
-    if (d < p.G) {
-      part[kMaxGroup * kHeadDim + d] = m_cta[d];
-      part[kMaxGroup * kHeadDim + kMaxGroup + d] = l_cta[d];
+  const int n_clusters = (int)gridDim.x / cs, cl = ci / cs;
+  float *part = p.partials + ((int64_t)bk * n_clusters + cl) * kResFloats;
+  for (int item = tid; item < p.G * cols; item += blockDim.x) {
+    const int h = item / cols, col = rank * cols + item % cols;
+    float M = -INFINITY;
+    for (int r = 0; r < cs; ++r) M = fmaxf(M, cluster.map_shared_rank(res, r)[kMaxGroup * kHeadDim + h]);
+    float o = 0.f, l = 0.f;
+    for (int r = 0; r < cs; ++r) {
+      const float *rr = cluster.map_shared_rank(res, r);
+      const float wgt = M == -INFINITY ? 0.f : fast_exp2(rr[kMaxGroup * kHeadDim + h] - M);
+      o += rr[h * kHeadDim + col] * wgt;
+      l += rr[kMaxGroup * kHeadDim + kMaxGroup + h] * wgt;
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) sm_last = atomicAdd(&p.tickets[bk], 1) == p.n_splits - 1;
-    __syncthreads();
-    if (!sm_last) return;
-    __threadfence();
-    // ---- last arrival for this KV head: log-sum-exp merge of all partitions ----
-    const float *all = p.partials + (int64_t)bk * p.n_splits * kPartialStride;
-    for (int h = 0; h < p.G; ++h) {
-      float M = -INFINITY;
-      for (int i = 0; i < p.n_splits; ++i) M = fmaxf(M, __ldcg(all + (int64_t)i * kPartialStride + kMaxGroup * kHeadDim + h));
-      __syncthreads();                                   // sm_w of the previous head has been consumed
-      float lsum = 0.f;
-      for (int i0 = 0; i0 < p.n_splits; i0 += 64) {
-        const int n = min(64, p.n_splits - i0);
-        if (tid < n) {
-          const float mi = __ldcg(all + (int64_t)(i0 + tid) * kPartialStride + kMaxGroup * kHeadDim + h);
-          sm_w[tid] = (M == -INFINITY) ? 0.f : fast_exp2(mi - M);
-        }
-        __syncthreads();
-        float o = 0.f;
-        for (int i = 0; i < n; ++i) {
-          const float *pi = all + (int64_t)(i0 + i) * kPartialStride;
-          o += __ldcg(pi + h * kHeadDim + d) * sm_w[i];
-          lsum += __ldcg(pi + kMaxGroup * kHeadDim + kMaxGroup + h) * sm_w[i];
-        }
-        o_cta[0] = i0 == 0 ? o : o_cta[0] + o;
-        __syncthreads();
+    if (n_clusters == 1) {
+      const float outv = l > 0.f ? o / l : 0.f;
+      p.out[((int64_t)b * p.H_q + kvh * p.G + h) * kHeadDim + col] = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
+      if (p.lse != nullptr && col == 0)
+        p.lse[(int64_t)b * p.H_q + kvh * p.G + h] = l > 0.f ? (M + log2f(l)) * kLn2 : -INFINITY;
+    } else {
+      part[h * kHeadDim + col] = o;
+      if (col == 0) {
+        part[kMaxGroup * kHeadDim + h] = M;
+        part[kMaxGroup * kHeadDim + kMaxGroup + h] = l;
       }
-      const float outv = lsum > 0.f ? o_cta[0] / lsum : 0.f;
-      p.out[((int64_t)b * p.H_q + kvh * p.G + h) * kHeadDim + d] = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
-      if (p.lse != nullptr && d == 0)
-        p.lse[(int64_t)b * p.H_q + kvh * p.G + h] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
     }
-    if (tid == 0) p.tickets[bk] = 0;
-  } else {
-    for (int h = 0; h < p.G; ++h) {
-      const float outv = l_cta[h] > 0.f ? o_cta[h] / l_cta[h] : 0.f;
-      p.out[((int64_t)b * p.H_q + kvh * p.G + h) * kHeadDim + d] = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
-      if (p.lse != nullptr && d == 0)
-        p.lse[(int64_t)b * p.H_q + kvh * p.G + h] = l_cta[h] > 0.f ? (m_cta[h] + log2f(l_cta[h])) * kLn2 : -INFINITY;
+  }
+  cluster.sync();   // no CTA leaves while a peer may still read its shared memory
+
+  bool head_done = rank == 0;                            // one CTA per head reports completion
+  if (n_clusters > 1) {
+    // ---- several clusters per head: the last CTA to arrive merges the cluster results ----
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sm_last = atomicAdd(&p.tickets[bk], 1) == (int)gridDim.x - 1;
+    __syncthreads();
+    head_done = sm_last != 0;
+    if (head_done) {
+      __threadfence();
+      const float *all = p.partials + (int64_t)bk * n_clusters * kResFloats;
+      for (int item = tid; item < p.G * kHeadDim; item += blockDim.x) {
+        const int h = item >> 7, col = item & 127;
+        float M = -INFINITY;
+        for (int i = 0; i < n_clusters; ++i) M = fmaxf(M, __ldcg(all + i * kResFloats + kMaxGroup * kHeadDim + h));
+        float o = 0.f, l = 0.f;
+        for (int i = 0; i < n_clusters; ++i) {
+          const float *pi = all + i * kResFloats;
+          const float wgt = M == -INFINITY ? 0.f : fast_exp2(__ldcg(pi + kMaxGroup * kHeadDim + h) - M);
+          o += __ldcg(pi + h * kHeadDim + col) * wgt;
+          l += __ldcg(pi + kMaxGroup * kHeadDim + kMaxGroup + h) * wgt;
+        }
+        const float outv = l > 0.f ? o / l : 0.f;
+        p.out[((int64_t)b * p.H_q + kvh * p.G + h) * kHeadDim + col] = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
+        if (p.lse != nullptr && col == 0)
+          p.lse[(int64_t)b * p.H_q + kvh * p.G + h] = l > 0.f ? (M + log2f(l)) * kLn2 : -INFINITY;
+      }
+      if (tid == 0) p.tickets[bk] = 0;
     }
   }
   // ---- the last KV head to finish advances the step counter ----
-  if (tid == 0) {
+  if (head_done && tid == 0) {
     const int n_heads = p.B * p.H_kv;
     __threadfence();
     if (atomicAdd(&p.tickets[n_heads], 1) == n_heads - 1) {
@@ -250,10 +318,41 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_attn_kernel(const Decod
   }
 }
 
+cudaError_t decode_setup() {
+  return cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kDecodeMaxTiles * 2 * kTileBytes);
+}
+
+// Launch geometry for a reduced cache of L rows.
+void decode_geometry(int L, int *n_clusters, int *cs, int *n_warps, int *smem_bytes) {
+  const int n_tiles = (L + 15) / 16;
+  int c = 1;
+  while (c < 8 && c * 2 <= n_tiles) c <<= 1;                                      // cluster size 1, 2, 4 or 8
+  const int nc = (n_tiles + c * kDecodeMaxTiles - 1) / (c * kDecodeMaxTiles);    // clusters per head
+  const int per_cta = (n_tiles + c * nc - 1) / (c * nc);                         // most tiles a CTA gets
+  const int rounds = (per_cta + kDecodeMaxWarps - 1) / kDecodeMaxWarps;          // 1 or 2 tiles per warp
+  *n_clusters = nc;
+  *cs = c;
+  *n_warps = (per_cta + rounds - 1) / rounds;
+  *smem_bytes = per_cta * 2 * kTileBytes;
+}
+
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream) {
-  dim3 grid(p.n_splits, p.H_kv, p.B);
-  decode_attn_kernel<<<grid, kDecodeThreads, 0, stream>>>(p);
-  return cudaGetLastError();
+  int n_clusters, cs, n_warps, smem;
+  decode_geometry(p.L, &n_clusters, &cs, &n_warps, &smem);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(n_clusters * cs), (unsigned)p.H_kv, (unsigned)p.B);
+  cfg.blockDim = dim3((unsigned)(n_warps * 32), 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_attn_kernel, p);
 }
 
 }  // namespace sagekv
