@@ -58,7 +58,8 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
 
 __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char stage[];          // tiles: [K 4 KB | V 4 KB] each
-  __shared__ float res[kResFloats];                                 // this CTA's O[8][128], m[8], l[8]
+  __shared__ float inbox_o[kMaxGroup * kHeadDim];                   // [source CTA][head][my columns], pushed by the peers
+  __shared__ float inbox_m[kDecodeMaxCluster * kMaxGroup], inbox_l[kDecodeMaxCluster * kMaxGroup];
   __shared__ float sm_m[kDecodeMaxWarps][kMaxGroup], sm_l[kDecodeMaxWarps][kMaxGroup];
   __shared__ int sm_last;
 
@@ -70,6 +71,7 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   const int n_warps = blockDim.x >> 5;
   const int g = lane >> 2, c = lane & 3;
   const bool append = p.k_new != nullptr;
+  cluster.barrier_arrive();                              // waited for just before the first push into a peer
 
   int step = 0, slot = -1;
   if (append) {
@@ -208,59 +210,63 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   }
 
   // ---- merge the warps of the CTA (the staging area is reused for the exchange) ----
+  // Exchange order of the 8 x 128 values: idx = ((piece*8 + e)*8 + g)*8 + h for column piece*64 + g*8 + e,
+  // so that the float2 stores of a half-warp (g 0..3, heads 2c, 2c+1) fall into 32 different banks.
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
   if (c == 0) { sm_m[warp][g] = m_run; sm_l[warp][g] = l_run; }
   __syncthreads();                                       // also: every warp is done reading its tiles
   const int n_act = min(n_warps, my_tiles);              // warps that had a tile
-  float *xo = reinterpret_cast<float *>(stage);          // [n_act][8][128]
+  float *xo = reinterpret_cast<float *>(stage);          // [n_act][1024]
   if (warp < n_act) {
     const int h0 = 2 * c, h1 = 2 * c + 1;
     float M0 = -INFINITY, M1 = -INFINITY;
     for (int w = 0; w < n_act; ++w) { M0 = fmaxf(M0, sm_m[w][h0]); M1 = fmaxf(M1, sm_m[w][h1]); }
     const float f0 = M0 == -INFINITY ? 0.f : fast_exp2(sm_m[warp][h0] - M0);
     const float f1 = M1 == -INFINITY ? 0.f : fast_exp2(sm_m[warp][h1] - M1);
-    float *mine0 = xo + (warp * kMaxGroup + h0) * kHeadDim, *mine1 = xo + (warp * kMaxGroup + h1) * kHeadDim;
+    float *mine = xo + warp * (kMaxGroup * kHeadDim) + g * 8 + h0;
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
-      const int d_a = (mt >> 2) * 64 + g * 8 + (mt & 3) * 2;
-      mine0[d_a] = acc[mt][0] * f0;
-      mine1[d_a] = acc[mt][1] * f1;
-      mine0[d_a + 1] = acc[mt][2] * f0;
-      mine1[d_a + 1] = acc[mt][3] * f1;
+      const int pe = (mt >> 2) * 8 + (mt & 3) * 2;       // piece*8 + e of column d_a; d_a + 1 is the next e
+      *reinterpret_cast<float2 *>(mine + pe * 64) = make_float2(acc[mt][0] * f0, acc[mt][1] * f1);
+      *reinterpret_cast<float2 *>(mine + (pe + 1) * 64) = make_float2(acc[mt][2] * f0, acc[mt][3] * f1);
     }
   }
   __syncthreads();
-  for (int item = tid; item < kMaxGroup * kHeadDim; item += blockDim.x) {
-    const int h = item >> 7;
-    float o = 0.f;
-    for (int w = 0; w < n_act; ++w) o += xo[w * kMaxGroup * kHeadDim + item];
-    res[item] = o;
-    if ((item & 127) == 0) {
-      float M = -INFINITY, l = 0.f;
-      for (int w = 0; w < n_act; ++w) M = fmaxf(M, sm_m[w][h]);
-      for (int w = 0; w < n_act; ++w) l += M == -INFINITY ? 0.f : sm_l[w][h] * fast_exp2(sm_m[w][h] - M);
-      res[kMaxGroup * kHeadDim + h] = M;
-      res[kMaxGroup * kHeadDim + kMaxGroup + h] = l;
-    }
-  }
-  cluster.sync();
+  cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs
 
-  // ---- merge the CTAs of the cluster: this CTA finishes columns [rank*cols, (rank+1)*cols) of every head ----
-  const int cols = kHeadDim / cs;
+  // ---- push this CTA's result to the peers: the owner of a column slice receives it from every CTA ----
+  const int cols = kHeadDim / cs;                        // columns each CTA of the cluster finishes
+  for (int idx = tid; idx < kMaxGroup * kHeadDim; idx += blockDim.x) {
+    float o = 0.f;
+    for (int w = 0; w < n_act; ++w) o += xo[w * kMaxGroup * kHeadDim + idx];
+    const int h = idx & 7, col = (idx >> 9) * 64 + ((idx >> 3) & 7) * 8 + ((idx >> 6) & 7);
+    const int owner = col / cols;
+    cluster.map_shared_rank(inbox_o, owner)[(rank * kMaxGroup + h) * cols + (col - owner * cols)] = o;
+  }
+  for (int item = tid; item < kMaxGroup * cs; item += blockDim.x) {
+    const int h = item & 7, dst = item >> 3;
+    float M = -INFINITY, l = 0.f;
+    for (int w = 0; w < n_act; ++w) M = fmaxf(M, sm_m[w][h]);
+    for (int w = 0; w < n_act; ++w) l += M == -INFINITY ? 0.f : sm_l[w][h] * fast_exp2(sm_m[w][h] - M);
+    cluster.map_shared_rank(inbox_m, dst)[rank * kMaxGroup + h] = M;
+    cluster.map_shared_rank(inbox_l, dst)[rank * kMaxGroup + h] = l;
+  }
+  cluster.sync();   // all pushes have landed; no shared memory of a peer is touched after this point
+
+  // ---- finish columns [rank*cols, (rank+1)*cols) of every head from the inbox ----
   const int bk = b * p.H_kv + kvh;
   const int n_clusters = (int)gridDim.x / cs, cl = ci / cs;
   float *part = p.partials + ((int64_t)bk * n_clusters + cl) * kResFloats;
   for (int item = tid; item < p.G * cols; item += blockDim.x) {
-    const int h = item / cols, col = rank * cols + item % cols;
+    const int h = item / cols, lc = item - h * cols, col = rank * cols + lc;
     float M = -INFINITY;
-    for (int r = 0; r < cs; ++r) M = fmaxf(M, cluster.map_shared_rank(res, r)[kMaxGroup * kHeadDim + h]);
+    for (int r = 0; r < cs; ++r) M = fmaxf(M, inbox_m[r * kMaxGroup + h]);
     float o = 0.f, l = 0.f;
     for (int r = 0; r < cs; ++r) {
-      const float *rr = cluster.map_shared_rank(res, r);
-      const float wgt = M == -INFINITY ? 0.f : fast_exp2(rr[kMaxGroup * kHeadDim + h] - M);
-      o += rr[h * kHeadDim + col] * wgt;
-      l += rr[kMaxGroup * kHeadDim + kMaxGroup + h] * wgt;
+      const float wgt = M == -INFINITY ? 0.f : fast_exp2(inbox_m[r * kMaxGroup + h] - M);
+      o += inbox_o[(r * kMaxGroup + h) * cols + lc] * wgt;
+      l += inbox_l[r * kMaxGroup + h] * wgt;
     }
     if (n_clusters == 1) {
       const float outv = l > 0.f ? o / l : 0.f;
@@ -275,7 +281,6 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
       }
     }
   }
-  cluster.sync();   // no CTA leaves while a peer may still read its shared memory
 
   bool head_done = rank == 0;                            // one CTA per head reports completion
   if (n_clusters > 1) {
@@ -318,16 +323,38 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   }
 }
 
+static int g_max_cluster = 8;   // 16 where the device can co-schedule 16-CTA clusters of this kernel
+
 cudaError_t decode_setup() {
-  return cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              kDecodeMaxTiles * 2 * kTileBytes);
+  cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kDecodeMaxTiles * 2 * kTileBytes);
+  if (e != cudaSuccess) return e;
+  // clusters of 16 are beyond the portable size: allow them and ask whether enough of them fit
+  g_max_cluster = 8;
+  if (cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(16, 8, 1);
+    cfg.blockDim = dim3(kDecodeMaxWarps * 32, 1, 1);
+    cfg.dynamicSmemBytes = 12 * 2 * kTileBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 16;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, decode_attn_kernel, &cfg) == cudaSuccess && n >= 64) g_max_cluster = 16;
+  }
+  cudaGetLastError();
+  return cudaSuccess;
 }
 
 // Launch geometry for a reduced cache of L rows.
 void decode_geometry(int L, int *n_clusters, int *cs, int *n_warps, int *smem_bytes) {
   const int n_tiles = (L + 15) / 16;
   int c = 1;
-  while (c < 8 && c * 2 <= n_tiles) c <<= 1;                                      // cluster size 1, 2, 4 or 8
+  while (c < g_max_cluster && c * 2 <= n_tiles) c <<= 1;                         // cluster size 1, 2, 4, 8 or 16
   const int nc = (n_tiles + c * kDecodeMaxTiles - 1) / (c * kDecodeMaxTiles);    // clusters per head
   const int per_cta = (n_tiles + c * nc - 1) / (c * nc);                         // most tiles a CTA gets
   const int rounds = (per_cta + kDecodeMaxWarps - 1) / kDecodeMaxWarps;          // 1 or 2 tiles per warp
