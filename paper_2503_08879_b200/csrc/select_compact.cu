@@ -1,18 +1,25 @@
 // Step 2 (second half) and Step 3: per-query-head top-k over the score rows, then the gather that
 // builds the reduced cache  C = Concat(sink, selected, recent, last).
 //
-// One thread-block cluster owns one score row.  Each CTA of the cluster stages its contiguous slice of
-// the row in shared memory once (cp.async, 16 bytes per request) and every later pass works on that
-// copy, so the scores cross the memory system a single time.  The k-th largest key is found by a
-// three-digit radix select (11 + 11 + 10 bits of the order-preserving integer image of the fp32
-// score): per digit every CTA histograms its slice in shared memory, the histograms are added into
-// CTA 0's shared memory through distributed-shared-memory atomics, and after a cluster barrier every
-// CTA locates the digit in which the k-th key falls.  With the exact threshold known, a ballot/popcount
-// ranking in row order (warp -> CTA -> cluster prefix) gives every kept element its output slot
-// directly: strictly larger keys are kept, of the keys equal to the threshold the lowest positions are
-// kept, and the slots are ascending in position.  The CTA that owns an element also copies its K and V
-// rows into the head's segment of the reduced cache.  A few extra clusters copy the sink, recent and
-// last rows, which do not depend on the scores.
+// One thread-block cluster (up to 8 CTAs) owns one score row.  Each CTA stages its contiguous slice of
+// the row in shared memory once (cp.async, 16 bytes per request); every later step works on that copy, so
+// the scores cross the memory system a single time.
+//
+// Fast path (k_q small against the row, the normal case): a prefilter instead of a full radix select.
+//   1. every thread takes the maximum of its elements; the cluster's thread maxima are exchanged over
+//      distributed shared memory.  The k_q-th largest of these maxima is a lower bound T0 of the k_q-th
+//      largest score (k_q distinct elements are >= it), and it is tight: about k_q * (1 + few %) scores
+//      are >= T0.  T0 is taken as the lower edge of the histogram bin (2048 bins laid over the actual
+//      range of the maxima) in which that maximum falls.
+//   2. scores >= T0 become candidates (order-preserving key, position); the lists are exchanged.
+//   3. every CTA ranks its own candidates against all candidates (8 threads per candidate); rank < k_q
+//      means kept.  Keys are compared with the position as tie-break, so the lowest positions win ties.
+//   4. kept counts are exchanged; slot = kept in lower CTAs + kept before it in this CTA: ascending order.
+// General path (k_q large, tiny rows, or more candidates than the buffers hold, e.g. a row of equal
+// scores): three-digit radix select (11 + 11 + 10 bits) with histograms merged in CTA 0's shared memory by
+// distributed-shared-memory atomics, then a ballot/popcount ranking in row order.
+// Either way the CTA that owns a kept element copies its K and V rows into the head's segment of the
+// reduced cache, and a few extra clusters copy the sink, recent and last rows.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -26,16 +33,22 @@ constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kMaxCluster = 8;
 constexpr int kMaxBins = 2048;
 constexpr int kSelSmemLimit = 200 * 1024;
+constexpr int kGeneralScratch = 3 * kMaxBins * 4;   // merged histograms of the general path
 
 struct SelShared {
   uint32_t hist_local[kMaxBins];
-  uint32_t hist_merged[3][kMaxBins];   // merge target: only cluster rank 0's copy is written
-  int totals[kMaxCluster][2];          // (kept-larger, equal-to-threshold) per CTA; rank 0's copy
+  uint32_t gmax[kSelThreads];          // thread maxima of this CTA, read by the peers
+  uint32_t red[3][kSelWarps];
+  int totals[kMaxCluster][2];          // general path: (kept-larger, equal-to-threshold) per CTA; rank 0's copy
+  int cand_cnt[kMaxCluster];           // fast path: candidates per CTA, pushed by each CTA to every peer
+  int sel_cnt[kMaxCluster];            // fast path: kept per CTA
   int warp_cnt[kSelWarps][2];
   int scan_tmp[kSelWarps];
   int found[2];
   int list_count;
-  int pad_[1];
+  int n_cand_local;
+  int n_sel_local;
+  int pad_[3];
 };
 static_assert(sizeof(SelShared) % 16 == 0, "staged scores must stay 16-byte aligned");
 
@@ -59,6 +72,35 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *tmp) {
   int base = 0;
   for (int w = 0; w < warp; ++w) base += tmp[w];
   return base + inc - v;
+}
+
+// In a histogram of nb bins (nb = 1024 or 2048), find the bin in which the k-th largest key falls, counting
+// from the top bin down.  found[0] = bin, found[1] = rank of the key inside that bin.  Ends with a barrier.
+__device__ __forceinline__ void find_bin_from_top(const uint32_t *hist, int nb, int k, SelShared &sh) {
+  const int tid = threadIdx.x;
+  const int per = nb / kSelThreads;    // thread t looks at bins nb-1-t*per ... downwards
+  uint32_t cnt[4];
+  int mine = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    cnt[e] = 0;
+    if (e < per) {
+      cnt[e] = hist[nb - 1 - (tid * per + e)];
+      mine += (int)cnt[e];
+    }
+  }
+  int above = block_exclusive_scan(mine, sh.scan_tmp);   // keys in higher bins
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    if (e < per) {
+      if (above < k && above + (int)cnt[e] >= k) {
+        sh.found[0] = nb - 1 - (tid * per + e);
+        sh.found[1] = k - above;
+      }
+      above += (int)cnt[e];
+    }
+  }
+  __syncthreads();
 }
 
 // one warp copies one K row (lanes 0-15) and one V row (lanes 16-31), 16 bytes per lane
@@ -88,51 +130,176 @@ __device__ void copy_static_rows(const SelectParams &p, int cta, int n_ctas) {
   if (cta == 0 && threadIdx.x == 0) *p.d_step = 0;
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const SelectParams p, int n_rows, int chunk,
-                                                                      int resident, int list_cap) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  cg::cluster_group cluster = cg::this_cluster();
-  const int cs = cluster.num_blocks();
-  const int rank = cluster.block_rank();
-  const int cid = blockIdx.x / cs;
-  if (cid >= n_rows) {   // whole cluster takes this branch together; it touches no peer's memory
-    copy_static_rows(p, (cid - n_rows) * cs + rank, (gridDim.x / cs - n_rows) * cs);
-    return;
-  }
+// Geometry shared by the two paths
+struct SelCtx {
+  int cs, rank, row, lo, n_local, chunk;
+  const float *data;       // this CTA's slice (shared memory when staged, else global)
+  int2 *list;              // (slot, position) of the rows this CTA has to gather
+  int list_cap;
+  unsigned char *scratch;  // union: general-path histograms / fast-path candidate buffers
+  int cand_cap;            // candidates per CTA and in total that the fast path can hold
+};
 
-  SelShared &sh = *reinterpret_cast<SelShared *>(smem_raw);
-  float *staged = reinterpret_cast<float *>(smem_raw + sizeof(SelShared));
-  int2 *list = reinterpret_cast<int2 *>(smem_raw + sizeof(SelShared) + (resident ? (size_t)chunk * sizeof(float) : 0));
-
+// ---- fast path ----------------------------------------------------------------------------------
+// Returns false (for every CTA of the cluster alike) when the prefilter cannot be used for this row;
+// nothing has been written to global memory in that case.
+__device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int row = cid;
-  const int b = row / p.H_q, h = row - b * p.H_q;
-  const int kvh = h / p.G, j = h - kvh * p.G;
-  const int lo = rank * chunk;
-  const int n_local = max(0, min(p.E - lo, chunk));
-  const float *grow = p.scores + (int64_t)row * p.row_stride + lo;   // 16-byte aligned: chunk % 4 == 0
+  unsigned long long *cand_local = reinterpret_cast<unsigned long long *>(c.scratch);
+  unsigned long long *cand_all = cand_local + c.cand_cap;
+  int *sel_pos = reinterpret_cast<int *>(cand_all + c.cand_cap);
+  const int n_vec = c.n_local >> 2;
+  const float4 *data4 = reinterpret_cast<const float4 *>(c.data);
 
+  // 1. thread maxima
+  uint32_t tmax = 0;   // 0 is below the key of every number: "no element"
+  for (int v = tid; v < n_vec; v += kSelThreads) {
+    const float4 x = data4[v];
+    tmax = max(max(tmax, score_key(x.x)), max(score_key(x.y), max(score_key(x.z), score_key(x.w))));
+  }
+  for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) tmax = max(tmax, score_key(c.data[i]));
+  sh.gmax[tid] = tmax;
+  if (tid == 0) { sh.n_cand_local = 0; sh.n_sel_local = 0; }
+  cluster.sync();
+
+  // 2. all maxima of the cluster -> T0
+  uint32_t gm[kMaxCluster];
+#pragma unroll
+  for (int r = 0; r < kMaxCluster; ++r) gm[r] = r < c.cs ? cluster.map_shared_rank(sh.gmax, r)[tid] : 0u;
+  uint32_t kmin = 0xffffffffu, kmax = 0u, n_ne = 0u;
+#pragma unroll
+  for (int r = 0; r < kMaxCluster; ++r) {
+    if (gm[r] != 0u) { kmin = min(kmin, gm[r]); kmax = max(kmax, gm[r]); ++n_ne; }
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  n_ne = __reduce_add_sync(0xffffffffu, n_ne);
+  if (lane == 0) { sh.red[0][warp] = kmin; sh.red[1][warp] = kmax; sh.red[2][warp] = n_ne; }
+  __syncthreads();
+  kmin = 0xffffffffu; kmax = 0u; n_ne = 0u;
+#pragma unroll
+  for (int w = 0; w < kSelWarps; ++w) {
+    kmin = min(kmin, sh.red[0][w]); kmax = max(kmax, sh.red[1][w]); n_ne += sh.red[2][w];
+  }
+  if ((int)n_ne < 2 * p.k_q) return false;              // too few groups for a tight bound (same answer in every CTA)
+  const uint32_t diff = kmax ^ kmin;
+  const int hi = diff ? 31 - __clz(diff) : -1;           // highest bit in which the maxima differ
+  const int shift = hi > 10 ? hi - 10 : 0;               // 2048 bins cover [kmin, kmax]
+  const uint32_t base = kmin >> shift;
+#pragma unroll
+  for (int r = 0; r < kMaxCluster; ++r)
+    if (gm[r] != 0u) atomicAdd(&sh.hist_local[(gm[r] >> shift) - base], 1u);
+  __syncthreads();
+  find_bin_from_top(sh.hist_local, kMaxBins, p.k_q, sh);
+  const uint32_t T0 = (base + (uint32_t)sh.found[0]) << shift;
+  __syncthreads();
+  for (int i = tid; i < kMaxBins; i += kSelThreads) sh.hist_local[i] = 0;   // leave it clean for the general path
+
+  // 3. candidates: (key, position) packed so that a larger value precedes in (score desc, position asc)
+  for (int v = tid; v < n_vec; v += kSelThreads) {
+    const float4 x = data4[v];
+    const uint32_t k4[4] = {score_key(x.x), score_key(x.y), score_key(x.z), score_key(x.w)};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (k4[e] >= T0) {
+        const int n = atomicAdd(&sh.n_cand_local, 1);
+        if (n < c.cand_cap)
+          cand_local[n] = ((unsigned long long)k4[e] << 32) | (0xffffffffu - (uint32_t)(c.lo + 4 * v + e));
+      }
+    }
+  }
+  for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) {
+    const uint32_t k = score_key(c.data[i]);
+    if (k >= T0) {
+      const int n = atomicAdd(&sh.n_cand_local, 1);
+      if (n < c.cand_cap) cand_local[n] = ((unsigned long long)k << 32) | (0xffffffffu - (uint32_t)(c.lo + i));
+    }
+  }
+  __syncthreads();
+  const int n_loc = sh.n_cand_local;
+  if (tid < c.cs) cluster.map_shared_rank(sh.cand_cnt, tid)[c.rank] = n_loc;
+  cluster.sync();
+  int start[kMaxCluster + 1];
+  bool overflow = false;
+  start[0] = 0;
+#pragma unroll
+  for (int r = 0; r < kMaxCluster; ++r) {
+    const int n = r < c.cs ? sh.cand_cnt[r] : 0;
+    overflow |= n > c.cand_cap;
+    start[r + 1] = start[r] + n;
+  }
+  const int M = start[kMaxCluster];
+  if (overflow || M > c.cand_cap) return false;         // same counts in every CTA: the whole cluster falls back
+  for (int i = tid; i < M; i += kSelThreads) {
+    int r = 0;
+#pragma unroll
+    for (int q = 1; q < kMaxCluster; ++q) r += i >= start[q] ? 1 : 0;
+    cand_all[i] = cluster.map_shared_rank(cand_local, r)[i - start[r]];
+  }
+  __syncthreads();
+
+  // 4. rank of every own candidate among all candidates: 8 threads share one candidate
+  const int sub = tid & 7;
+  for (int c0 = 0; c0 < n_loc; c0 += kSelThreads / 8) {
+    const int ci = c0 + (tid >> 3);
+    const bool valid = ci < n_loc;
+    const unsigned long long mine = valid ? cand_local[ci] : 0ull;
+    int before = 0;
+    if (valid)
+      for (int i = sub; i < M; i += 8) before += cand_all[i] > mine ? 1 : 0;
+    before += __shfl_xor_sync(0xffffffffu, before, 1);
+    before += __shfl_xor_sync(0xffffffffu, before, 2);
+    before += __shfl_xor_sync(0xffffffffu, before, 4);
+    if (valid && sub == 0 && before < p.k_q) {
+      const int n = atomicAdd(&sh.n_sel_local, 1);
+      sel_pos[n] = (int)(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+    }
+  }
+  __syncthreads();
+  const int n_sel = sh.n_sel_local;
+  if (tid < c.cs) cluster.map_shared_rank(sh.sel_cnt, tid)[c.rank] = n_sel;
+  cluster.sync();   // last access to a peer's shared memory
+  int offset = 0;
+  for (int r = 0; r < c.rank; ++r) offset += sh.sel_cnt[r];
+
+  // 5. output slots in ascending position
+  int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
+  for (int c0 = 0; c0 < n_sel; c0 += kSelThreads / 8) {
+    const int ci = c0 + (tid >> 3);
+    const bool valid = ci < n_sel;
+    const int mine = valid ? sel_pos[ci] : 0;
+    int before = 0;
+    if (valid)
+      for (int i = sub; i < n_sel; i += 8) before += sel_pos[i] < mine ? 1 : 0;
+    before += __shfl_xor_sync(0xffffffffu, before, 1);
+    before += __shfl_xor_sync(0xffffffffu, before, 2);
+    before += __shfl_xor_sync(0xffffffffu, before, 4);
+    if (valid && sub == 0) {
+      const int slot = offset + before;
+      idx_row[slot] = p.S + mine;
+      if (ci < c.list_cap) c.list[ci] = make_int2(slot, p.S + mine);
+    }
+  }
+  if (tid == 0) sh.list_count = n_sel;
+  __syncthreads();
+  return true;
+}
+
+// ---- general path -------------------------------------------------------------------------------
+__device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t(*hist_merged)[kMaxBins] = reinterpret_cast<uint32_t(*)[kMaxBins]>(c.scratch);   // only rank 0's copy is used
+  const float *data = c.data;
+  const int n_local = c.n_local;
   for (int i = tid; i < kMaxBins; i += kSelThreads) {
     sh.hist_local[i] = 0;
-    sh.hist_merged[0][i] = 0; sh.hist_merged[1][i] = 0; sh.hist_merged[2][i] = 0;
+    hist_merged[0][i] = 0; hist_merged[1][i] = 0; hist_merged[2][i] = 0;
   }
   if (tid == 0) sh.list_count = 0;
-
-  const float *data = grow;
-  if (resident) {
-    const int n_vec = n_local >> 2;
-    for (int v = tid; v < n_vec; v += kSelThreads) {
-      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(staged + 4 * v);
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(grow + 4 * v) : "memory");
-    }
-    for (int i = (n_vec << 2) + tid; i < n_local; i += kSelThreads) staged[i] = grow[i];
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    data = staged;
-  }
   __syncthreads();
   cluster.sync();   // every CTA's merge histograms are zero before any peer adds into them
 
-  // ---- radix select: threshold key and how many keys equal to it are kept ----
+  // radix select: threshold key and how many keys equal to it are kept
   uint32_t prefix = 0;        // digits found so far, right-aligned
   int k_rem = p.k_q;          // rank of the wanted key among keys matching `prefix`
 #pragma unroll
@@ -157,7 +324,7 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
       }
     }
     __syncthreads();
-    uint32_t *merged0 = cluster.map_shared_rank(&sh.hist_merged[pass][0], 0);
+    uint32_t *merged0 = cluster.map_shared_rank(&hist_merged[pass][0], 0);
     for (int bin = tid; bin < nb; bin += kSelThreads) {
       const uint32_t v = sh.hist_local[bin];
       if (v) {
@@ -166,30 +333,7 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
       }
     }
     cluster.sync();
-    // thread t looks at bins nb-1-t*per ... downwards; `above` = keys in higher bins
-    const int per = nb / kSelThreads;
-    uint32_t cnt[4];
-    int mine = 0;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      cnt[e] = 0;
-      if (e < per) {
-        cnt[e] = merged0[nb - 1 - (tid * per + e)];
-        mine += (int)cnt[e];
-      }
-    }
-    int above = block_exclusive_scan(mine, sh.scan_tmp);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      if (e < per) {
-        if (above < k_rem && above + (int)cnt[e] >= k_rem) {
-          sh.found[0] = nb - 1 - (tid * per + e);
-          sh.found[1] = k_rem - above;
-        }
-        above += (int)cnt[e];
-      }
-    }
-    __syncthreads();
+    find_bin_from_top(merged0, nb, k_rem, sh);
     prefix = (prefix << bits) | (uint32_t)sh.found[0];
     k_rem = sh.found[1];
     __syncthreads();                                    // found[] is rewritten by the next pass
@@ -197,8 +341,8 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
   const uint32_t tau = prefix;                          // exact key of the k-th largest score
   const int ties_kept = k_rem;                          // >= 1 keys equal to tau are kept, lowest positions first
 
-  // ---- ranks in row order: warp w owns the contiguous range [w*wlen, (w+1)*wlen) of the slice ----
-  const int wlen = (((chunk + kSelWarps - 1) / kSelWarps) + 31) & ~31;
+  // ranks in row order: warp w owns the contiguous range [w*wlen, (w+1)*wlen) of the slice
+  const int wlen = (((c.chunk + kSelWarps - 1) / kSelWarps) + 31) & ~31;
   const int wlo = warp * wlen, whi = min(n_local, wlo + wlen);
   int n_gt = 0, n_eq = 0;
   for (int base = wlo; base < whi; base += 32) {
@@ -217,16 +361,16 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
   }
   if (tid == 0) {
     int *t0 = cluster.map_shared_rank(&sh.totals[0][0], 0);
-    t0[2 * rank] = cta_gt;
-    t0[2 * rank + 1] = cta_eq;
+    t0[2 * c.rank] = cta_gt;
+    t0[2 * c.rank + 1] = cta_eq;
   }
   cluster.sync();
   {
     const int *t0 = cluster.map_shared_rank(&sh.totals[0][0], 0);
-    for (int r = 0; r < rank; ++r) { gt_before += t0[2 * r]; eq_before += t0[2 * r + 1]; }
+    for (int r = 0; r < c.rank; ++r) { gt_before += t0[2 * r]; eq_before += t0[2 * r + 1]; }
   }
 
-  int32_t *idx_row = p.idx + (int64_t)row * p.k_q;
+  int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
   for (int base = wlo; base < whi; base += 32) {
     const int i = base + lane;
     const uint32_t key = i < whi ? score_key(data[i]) : 0u;
@@ -238,27 +382,78 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
     if (gt) slot = g_here + min(e_here, ties_kept);
     else if (eq && e_here < ties_kept) slot = g_here + e_here;
     if (slot >= 0) {
-      const int pos = p.S + lo + i;
+      const int pos = p.S + c.lo + i;
       idx_row[slot] = pos;
       const int n = atomicAdd(&sh.list_count, 1);
-      if (n < list_cap) list[n] = make_int2(slot, pos);
+      if (n < c.list_cap) c.list[n] = make_int2(slot, pos);
     }
     gt_before += __popc(bg);
     eq_before += __popc(be);
   }
   __syncthreads();
-
-  // ---- gather this CTA's kept rows into head j's segment of the reduced cache ----
-  const int n_list = min(sh.list_count, list_cap);
-  for (int e = warp; e < n_list; e += kSelWarps) {
-    const int2 sp = list[e];
-    copy_kv_row(p, b, kvh, sp.y, (int64_t)p.S + (int64_t)j * p.k_q + sp.x, lane);
-  }
-  cluster.sync();   // no CTA leaves while a peer may still read its shared memory
+  cluster.sync();   // no CTA moves on (and may exit) while a peer still reads its shared memory
 }
 
-static size_t select_smem_bytes(int chunk, int list_cap, bool resident) {
-  return sizeof(SelShared) + (size_t)list_cap * sizeof(int2) + (resident ? (size_t)chunk * sizeof(float) : 0);
+__global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const SelectParams p, int n_rows, int chunk,
+                                                                      int resident, int list_cap, int cand_cap,
+                                                                      int try_fast) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int cs = cluster.num_blocks();
+  const int rank = cluster.block_rank();
+  const int cid = blockIdx.x / cs;
+  if (cid >= n_rows) {   // whole cluster takes this branch together; it touches no peer's memory
+    copy_static_rows(p, (cid - n_rows) * cs + rank, (gridDim.x / cs - n_rows) * cs);
+    return;
+  }
+
+  SelShared &sh = *reinterpret_cast<SelShared *>(smem_raw);
+  float *staged = reinterpret_cast<float *>(smem_raw + sizeof(SelShared));
+  unsigned char *after = smem_raw + sizeof(SelShared) + (resident ? (size_t)chunk * sizeof(float) : 0);
+  SelCtx c;
+  c.cs = cs; c.rank = rank; c.row = cid; c.chunk = chunk;
+  c.lo = rank * chunk;
+  c.n_local = max(0, min(p.E - c.lo, chunk));
+  c.list = reinterpret_cast<int2 *>(after);
+  c.list_cap = list_cap;
+  c.scratch = after + (size_t)list_cap * sizeof(int2);   // 8-byte aligned
+  c.cand_cap = cand_cap;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = c.row / p.H_q, h = c.row - b * p.H_q;
+  const int kvh = h / p.G, j = h - kvh * p.G;
+  const float *grow = p.scores + (int64_t)c.row * p.row_stride + c.lo;   // 16-byte aligned: chunk % 4 == 0
+
+  for (int i = tid; i < kMaxBins; i += kSelThreads) sh.hist_local[i] = 0;
+  c.data = grow;
+  if (resident) {
+    const int n_vec = c.n_local >> 2;
+    for (int v = tid; v < n_vec; v += kSelThreads) {
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(staged + 4 * v);
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(grow + 4 * v) : "memory");
+    }
+    for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) staged[i] = grow[i];
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    c.data = staged;
+  }
+  __syncthreads();
+
+  bool done = false;
+  if (try_fast) done = fast_select(cluster, sh, p, c);
+  if (!done) general_select(cluster, sh, p, c);
+
+  // gather this CTA's kept rows into head j's segment of the reduced cache
+  const int n_list = min(sh.list_count, list_cap);
+  for (int e = warp; e < n_list; e += kSelWarps) {
+    const int2 sp = c.list[e];
+    copy_kv_row(p, b, kvh, sp.y, (int64_t)p.S + (int64_t)j * p.k_q + sp.x, lane);
+  }
+}
+
+static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, bool resident) {
+  size_t scratch = (size_t)cand_cap * (8 + 8 + 4);
+  if (scratch < (size_t)kGeneralScratch) scratch = kGeneralScratch;
+  return sizeof(SelShared) + (size_t)list_cap * sizeof(int2) + scratch + (resident ? (size_t)chunk * sizeof(float) : 0);
 }
 
 cudaError_t select_compact_setup() {
@@ -275,8 +470,11 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   chunk = (chunk + 3) & ~3;
   if (chunk < 4) chunk = 4;
   const int list_cap = chunk < p.k_q ? chunk : (p.k_q > 0 ? p.k_q : 1);
-  const bool resident = select_smem_bytes(chunk, list_cap, true) <= (size_t)kSelSmemLimit;
-  const size_t smem = select_smem_bytes(chunk, list_cap, resident);
+  // the prefilter needs at least 2*k_q thread maxima; its buffers hold 2*k_q + 256 candidates
+  const int try_fast = select && 2 * (int64_t)p.k_q <= (int64_t)cs * kSelThreads;
+  const int cand_cap = try_fast ? 2 * p.k_q + 256 : 0;
+  const bool resident = select_smem_bytes(chunk, list_cap, cand_cap, true) <= (size_t)kSelSmemLimit;
+  const size_t smem = select_smem_bytes(chunk, list_cap, cand_cap, resident);
 
   const int static_items = p.B * p.H_kv * (p.S + p.R + 1);
   int copy_clusters = (static_items + cs * kSelWarps * 2 - 1) / (cs * kSelWarps * 2);
@@ -296,7 +494,8 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, select_compact_kernel, p, n_rows, chunk, (int)resident, list_cap);
+  return cudaLaunchKernelEx(&cfg, select_compact_kernel, p, n_rows, chunk, (int)resident, list_cap, cand_cap,
+                            try_fast);
 }
 
 }  // namespace sagekv
