@@ -39,6 +39,7 @@ struct SelShared {
   uint32_t hist_local[kMaxBins];
   uint32_t gmax[kSelThreads];          // thread maxima of this CTA, read by the peers
   uint32_t red[3][kSelWarps];
+  uint32_t gstat[kMaxCluster][4];      // (min, max, count) of every CTA's non-empty thread maxima, pushed by the peers
   int totals[kMaxCluster][2];          // general path: (kept-larger, equal-to-threshold) per CTA; rank 0's copy
   int cand_cnt[kMaxCluster];           // fast path: candidates per CTA, pushed by each CTA to every peer
   int sel_cnt[kMaxCluster];            // fast path: kept per CTA
@@ -55,6 +56,10 @@ static_assert(sizeof(SelShared) % 16 == 0, "staged scores must stay 16-byte alig
 __device__ __forceinline__ uint32_t score_key(float x) {
   const uint32_t u = __float_as_uint(x + 0.0f);         // -0 becomes +0: the two compare equal as numbers
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);   // larger float <=> larger unsigned key
+}
+
+__device__ __forceinline__ float key_to_score(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
 // exclusive prefix of v over the CTA in thread order
@@ -140,79 +145,126 @@ struct SelCtx {
   int cand_cap;            // candidates per CTA and in total that the fast path can hold
 };
 
+// Eight float4 of this thread's elements (vector indices v0 + tid + u*512), all loads issued before any use.
+// Missing ones (index >= n_vec) read as -inf, which is below every threshold and never a maximum.
+template <bool kStaged>
+__device__ __forceinline__ void load8(const float *data, int v0, int n_vec, float4 (&x)[8]) {
+  const float ninf = -INFINITY;
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int v = v0 + (int)threadIdx.x + u * kSelThreads;
+    x[u] = make_float4(ninf, ninf, ninf, ninf);
+    if (v < n_vec) {
+      if (kStaged) {
+        const uint32_t a = (uint32_t)__cvta_generic_to_shared(data + 4 * v);
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x[u].x), "=f"(x[u].y), "=f"(x[u].z), "=f"(x[u].w) : "r"(a));
+      } else {
+        asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(x[u].x), "=f"(x[u].y), "=f"(x[u].z), "=f"(x[u].w) : "l"(data + 4 * v));
+      }
+    }
+  }
+}
+
 // ---- fast path ----------------------------------------------------------------------------------
 // Returns false (for every CTA of the cluster alike) when the prefilter cannot be used for this row;
 // nothing has been written to global memory in that case.
+template <bool kStaged>
 __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned long long *cand_local = reinterpret_cast<unsigned long long *>(c.scratch);
-  unsigned long long *cand_all = cand_local + c.cand_cap;
-  int *sel_pos = reinterpret_cast<int *>(cand_all + c.cand_cap);
+  unsigned long long *cand_all = cand_local + c.cand_cap;            // 16-byte aligned: cand_cap is even
+  int *sel_pos = reinterpret_cast<int *>(cand_all + c.cand_cap + 2);
   const int n_vec = c.n_local >> 2;
-  const float4 *data4 = reinterpret_cast<const float4 *>(c.data);
 
-  // 1. thread maxima
+  // 1. thread maxima (float order equals key order, so one fmaxf per element and one key per thread)
   uint32_t tmax = 0;   // 0 is below the key of every number: "no element"
-  for (int v = tid; v < n_vec; v += kSelThreads) {
-    const float4 x = data4[v];
-    tmax = max(max(tmax, score_key(x.x)), max(score_key(x.y), max(score_key(x.z), score_key(x.w))));
+  {
+    float fm = -INFINITY;
+    for (int v0 = 0; v0 < n_vec; v0 += 8 * kSelThreads) {
+      float4 x[8];
+      load8<kStaged>(c.data, v0, n_vec, x);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) fm = fmaxf(fmaxf(fm, x[u].x), fmaxf(x[u].y, fmaxf(x[u].z, x[u].w)));
+    }
+    bool any = tid < n_vec;
+    for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) { fm = fmaxf(fm, c.data[i]); any = true; }
+    if (any) tmax = score_key(fm);
   }
-  for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) tmax = max(tmax, score_key(c.data[i]));
   sh.gmax[tid] = tmax;
+  {
+    const uint32_t wmin = __reduce_min_sync(0xffffffffu, tmax ? tmax : 0xffffffffu);
+    const uint32_t wmax = __reduce_max_sync(0xffffffffu, tmax);
+    const uint32_t wcnt = __popc(__ballot_sync(0xffffffffu, tmax != 0u));
+    if (lane == 0) { sh.red[0][warp] = wmin; sh.red[1][warp] = wmax; sh.red[2][warp] = wcnt; }
+  }
   if (tid == 0) { sh.n_cand_local = 0; sh.n_sel_local = 0; }
+  __syncthreads();
+  if (warp == 0) {   // (min, max, count) of this CTA's maxima, pushed into every peer's gstat table
+    uint32_t mn = lane < kSelWarps ? sh.red[0][lane] : 0xffffffffu;
+    uint32_t mx = lane < kSelWarps ? sh.red[1][lane] : 0u;
+    uint32_t cnt = lane < kSelWarps ? sh.red[2][lane] : 0u;
+    mn = __reduce_min_sync(0xffffffffu, mn);
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (lane < c.cs) {
+      uint32_t *gs = cluster.map_shared_rank(&sh.gstat[0][0], lane) + 4 * c.rank;
+      gs[0] = mn; gs[1] = mx; gs[2] = cnt;
+    }
+  }
   cluster.sync();
 
-  // 2. all maxima of the cluster -> T0
+  // 2. all maxima of the cluster -> T0 (512 bins laid over [kmin, kmax])
   uint32_t gm[kMaxCluster];
-#pragma unroll
-  for (int r = 0; r < kMaxCluster; ++r) gm[r] = r < c.cs ? cluster.map_shared_rank(sh.gmax, r)[tid] : 0u;
   uint32_t kmin = 0xffffffffu, kmax = 0u, n_ne = 0u;
 #pragma unroll
   for (int r = 0; r < kMaxCluster; ++r) {
-    if (gm[r] != 0u) { kmin = min(kmin, gm[r]); kmax = max(kmax, gm[r]); ++n_ne; }
-  }
-  kmin = __reduce_min_sync(0xffffffffu, kmin);
-  kmax = __reduce_max_sync(0xffffffffu, kmax);
-  n_ne = __reduce_add_sync(0xffffffffu, n_ne);
-  if (lane == 0) { sh.red[0][warp] = kmin; sh.red[1][warp] = kmax; sh.red[2][warp] = n_ne; }
-  __syncthreads();
-  kmin = 0xffffffffu; kmax = 0u; n_ne = 0u;
-#pragma unroll
-  for (int w = 0; w < kSelWarps; ++w) {
-    kmin = min(kmin, sh.red[0][w]); kmax = max(kmax, sh.red[1][w]); n_ne += sh.red[2][w];
+    gm[r] = 0u;
+    if (r < c.cs) {
+      gm[r] = cluster.map_shared_rank(sh.gmax, r)[tid];
+      kmin = min(kmin, sh.gstat[r][0]); kmax = max(kmax, sh.gstat[r][1]); n_ne += sh.gstat[r][2];
+    }
   }
   if ((int)n_ne < 2 * p.k_q) return false;              // too few groups for a tight bound (same answer in every CTA)
   const uint32_t diff = kmax ^ kmin;
   const int hi = diff ? 31 - __clz(diff) : -1;           // highest bit in which the maxima differ
-  const int shift = hi > 10 ? hi - 10 : 0;               // 2048 bins cover [kmin, kmax]
+  const int shift = hi > 8 ? hi - 8 : 0;                 // (kmax >> shift) - (kmin >> shift) < 512
   const uint32_t base = kmin >> shift;
 #pragma unroll
   for (int r = 0; r < kMaxCluster; ++r)
     if (gm[r] != 0u) atomicAdd(&sh.hist_local[(gm[r] >> shift) - base], 1u);
   __syncthreads();
-  find_bin_from_top(sh.hist_local, kMaxBins, p.k_q, sh);
+  find_bin_from_top(sh.hist_local, kSelThreads, p.k_q, sh);
   const uint32_t T0 = (base + (uint32_t)sh.found[0]) << shift;
-  __syncthreads();
-  for (int i = tid; i < kMaxBins; i += kSelThreads) sh.hist_local[i] = 0;   // leave it clean for the general path
+  const float T0f = key_to_score(T0);
+  sh.hist_local[tid] = 0;                                // leave it clean (only the first 512 bins were used)
 
   // 3. candidates: (key, position) packed so that a larger value precedes in (score desc, position asc)
-  for (int v = tid; v < n_vec; v += kSelThreads) {
-    const float4 x = data4[v];
-    const uint32_t k4[4] = {score_key(x.x), score_key(x.y), score_key(x.z), score_key(x.w)};
+  for (int v0 = 0; v0 < n_vec; v0 += 8 * kSelThreads) {
+    float4 x[8];
+    load8<kStaged>(c.data, v0, n_vec, x);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      if (k4[e] >= T0) {
-        const int n = atomicAdd(&sh.n_cand_local, 1);
-        if (n < c.cand_cap)
-          cand_local[n] = ((unsigned long long)k4[e] << 32) | (0xffffffffu - (uint32_t)(c.lo + 4 * v + e));
+    for (int u = 0; u < 8; ++u) {
+      if (x[u].x >= T0f || x[u].y >= T0f || x[u].z >= T0f || x[u].w >= T0f) {
+        const float xs[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+        const int v = v0 + tid + u * kSelThreads;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (xs[e] >= T0f) {
+            const int n = atomicAdd(&sh.n_cand_local, 1);
+            if (n < c.cand_cap)
+              cand_local[n] = ((unsigned long long)score_key(xs[e]) << 32) | (0xffffffffu - (uint32_t)(c.lo + 4 * v + e));
+          }
+        }
       }
     }
   }
   for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) {
-    const uint32_t k = score_key(c.data[i]);
-    if (k >= T0) {
+    const float x = c.data[i];
+    if (x >= T0f) {
       const int n = atomicAdd(&sh.n_cand_local, 1);
-      if (n < c.cand_cap) cand_local[n] = ((unsigned long long)k << 32) | (0xffffffffu - (uint32_t)(c.lo + i));
+      if (n < c.cand_cap)
+        cand_local[n] = ((unsigned long long)score_key(x) << 32) | (0xffffffffu - (uint32_t)(c.lo + i));
     }
   }
   __syncthreads();
@@ -238,21 +290,42 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   }
   __syncthreads();
 
-  // 4. rank of every own candidate among all candidates: 8 threads share one candidate
-  const int sub = tid & 7;
-  for (int c0 = 0; c0 < n_loc; c0 += kSelThreads / 8) {
-    const int ci = c0 + (tid >> 3);
-    const bool valid = ci < n_loc;
-    const unsigned long long mine = valid ? cand_local[ci] : 0ull;
-    int before = 0;
-    if (valid)
-      for (int i = sub; i < M; i += 8) before += cand_all[i] > mine ? 1 : 0;
-    before += __shfl_xor_sync(0xffffffffu, before, 1);
-    before += __shfl_xor_sync(0xffffffffu, before, 2);
-    before += __shfl_xor_sync(0xffffffffu, before, 4);
-    if (valid && sub == 0 && before < p.k_q) {
-      const int n = atomicAdd(&sh.n_sel_local, 1);
-      sel_pos[n] = (int)(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
+  // 4. rank of every own candidate among all candidates.  A group of tpc threads takes four own candidates
+  //    (four independent compare chains per loaded pair of candidates) and strides over the full list.
+  const int n_quads = (n_loc + 3) >> 2;
+  int tpc = 32;
+  while (tpc > 1 && n_quads * tpc > kSelThreads) tpc >>= 1;
+  const int sub = tid & (tpc - 1);
+  const int M2 = (M + 1) >> 1;
+  if ((M & 1) && tid == 0) cand_all[M] = 0ull;           // pad to an even count with a value that precedes nothing
+  __syncthreads();
+  const uint32_t all_addr = (uint32_t)__cvta_generic_to_shared(cand_all);
+  for (int q0 = 0; q0 < n_quads; q0 += kSelThreads / tpc) {
+    const int qi = q0 + tid / tpc;
+    unsigned long long mine[4];
+    int before[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int u = 0; u < 4; ++u) mine[u] = (qi < n_quads && 4 * qi + u < n_loc) ? cand_local[4 * qi + u] : ~0ull;
+    if (qi < n_quads) {
+#pragma unroll 2
+      for (int i = sub; i < M2; i += tpc) {
+        unsigned long long ox, oy;
+        asm volatile("ld.shared.v2.u64 {%0,%1}, [%2];" : "=l"(ox), "=l"(oy) : "r"(all_addr + 16u * (uint32_t)i));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) before[u] += (ox > mine[u] ? 1 : 0) + (oy > mine[u] ? 1 : 0);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      for (int off = 1; off < tpc; off <<= 1) before[u] += __shfl_xor_sync(0xffffffffu, before[u], off);
+    if (qi < n_quads && sub == 0) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (4 * qi + u < n_loc && before[u] < p.k_q) {
+          const int n = atomicAdd(&sh.n_sel_local, 1);
+          sel_pos[n] = (int)(0xffffffffu - (uint32_t)(mine[u] & 0xffffffffull));
+        }
+      }
     }
   }
   __syncthreads();
@@ -264,17 +337,18 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
 
   // 5. output slots in ascending position
   int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
-  for (int c0 = 0; c0 < n_sel; c0 += kSelThreads / 8) {
-    const int ci = c0 + (tid >> 3);
+  int tps = 32;
+  while (tps > 1 && n_sel * tps > kSelThreads) tps >>= 1;
+  const int sub2 = tid & (tps - 1);
+  for (int c0 = 0; c0 < n_sel; c0 += kSelThreads / tps) {
+    const int ci = c0 + tid / tps;
     const bool valid = ci < n_sel;
     const int mine = valid ? sel_pos[ci] : 0;
     int before = 0;
     if (valid)
-      for (int i = sub; i < n_sel; i += 8) before += sel_pos[i] < mine ? 1 : 0;
-    before += __shfl_xor_sync(0xffffffffu, before, 1);
-    before += __shfl_xor_sync(0xffffffffu, before, 2);
-    before += __shfl_xor_sync(0xffffffffu, before, 4);
-    if (valid && sub == 0) {
+      for (int i = sub2; i < n_sel; i += tps) before += sel_pos[i] < mine ? 1 : 0;
+    for (int off = 1; off < tps; off <<= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
+    if (valid && sub2 == 0) {
       const int slot = offset + before;
       idx_row[slot] = p.S + mine;
       if (ci < c.list_cap) c.list[ci] = make_int2(slot, p.S + mine);
@@ -407,6 +481,7 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
     return;
   }
 
+  cluster.barrier_arrive();   // completed below: every CTA of the cluster runs before anyone writes into a peer
   SelShared &sh = *reinterpret_cast<SelShared *>(smem_raw);
   float *staged = reinterpret_cast<float *>(smem_raw + sizeof(SelShared));
   unsigned char *after = smem_raw + sizeof(SelShared) + (resident ? (size_t)chunk * sizeof(float) : 0);
@@ -416,7 +491,7 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
   c.n_local = max(0, min(p.E - c.lo, chunk));
   c.list = reinterpret_cast<int2 *>(after);
   c.list_cap = list_cap;
-  c.scratch = after + (size_t)list_cap * sizeof(int2);   // 8-byte aligned
+  c.scratch = after + (((size_t)list_cap * sizeof(int2) + 15) & ~(size_t)15);   // 16-byte aligned
   c.cand_cap = cand_cap;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -437,23 +512,39 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
     c.data = staged;
   }
   __syncthreads();
+  cluster.barrier_wait();
 
   bool done = false;
-  if (try_fast) done = fast_select(cluster, sh, p, c);
+  if (try_fast) done = resident ? fast_select<true>(cluster, sh, p, c) : fast_select<false>(cluster, sh, p, c);
   if (!done) general_select(cluster, sh, p, c);
 
-  // gather this CTA's kept rows into head j's segment of the reduced cache
+  // gather this CTA's kept rows into head j's segment of the reduced cache: a warp moves four rows at a
+  // time (K in lanes 0-15, V in lanes 16-31), all loads issued before the stores
   const int n_list = min(sh.list_count, list_cap);
-  for (int e = warp; e < n_list; e += kSelWarps) {
-    const int2 sp = c.list[e];
-    copy_kv_row(p, b, kvh, sp.y, (int64_t)p.S + (int64_t)j * p.k_q + sp.x, lane);
+  const uint16_t *src_base = (lane < 16 ? p.K : p.V) + (int64_t)b * p.ks.batch_stride + (int64_t)kvh * p.ks.head_stride +
+                             (lane & 15) * 8;
+  uint16_t *dst_base = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
+                       ((int64_t)p.S + (int64_t)j * p.k_q) * p.cs.token_stride + (lane & 15) * 8;
+  for (int e0 = warp * 4; e0 < n_list; e0 += kSelWarps * 4) {
+    uint4 v[4];
+    int slot[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int2 sp = c.list[min(e0 + u, n_list - 1)];
+      slot[u] = sp.x;
+      v[u] = ld_stream_v4(src_base + (int64_t)sp.y * p.ks.token_stride);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (e0 + u < n_list) st_v4(dst_base + (int64_t)slot[u] * p.cs.token_stride, v[u]);
   }
 }
 
 static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, bool resident) {
-  size_t scratch = (size_t)cand_cap * (8 + 8 + 4);
+  size_t scratch = (size_t)cand_cap * (8 + 8 + 4) + 16;
   if (scratch < (size_t)kGeneralScratch) scratch = kGeneralScratch;
-  return sizeof(SelShared) + (size_t)list_cap * sizeof(int2) + scratch + (resident ? (size_t)chunk * sizeof(float) : 0);
+  return sizeof(SelShared) + (((size_t)list_cap * sizeof(int2) + 15) & ~(size_t)15) + scratch +
+         (resident ? (size_t)chunk * sizeof(float) : 0);
 }
 
 cudaError_t select_compact_setup() {
