@@ -235,6 +235,10 @@ def run_cuda(args, w):
                 d = lay["dec"][t]
                 sk.decode_attn(d["q"], d["k_new"], d["v_new"], lay["cache"], lay["out"])
 
+    # decode launches overlap with their predecessor; with several layers the kernel before a decode call
+    # belongs to another layer, so the reduced cache may be prefetched before the dependency wait
+    overlap = args.overlap if args.overlap is not None else (2 if n_layers > 1 else 1)
+    sk.set_overlap(overlap)
     phase_a(); phase_b(); phase_c()          # eager once: loads modules, sets function attributes
     torch.cuda.synchronize()
     graphs = []
@@ -310,7 +314,7 @@ def run_cuda(args, w):
                            w.n_q_heads, w.n_kv_heads, w.head_dim),
                        "layers": n_layers, "batch": w.batch, "n_ctx": w.n_ctx, "budget": w.budget, "n_init": w.n_init,
                        "n_recent": w.n_recent, "k_per_kv_head": w.n_sel, "k_q": w.k_q,
-                       "decode_steps_per_step": decode_steps, "parallelism": "replicas x%d" % args.gpus,
+                       "decode_steps_per_step": decode_steps, "decode_overlap_mode": overlap, "parallelism": "replicas x%d" % args.gpus,
                        "l2": "inputs larger than L2: layers visited round-robin, %.0f MB of K per layer, %.0f MB of "
                              "reduced caches per decode step" % (ab["score"] / 1e6, ab["decode_attn"] * n_layers / 1e6)},
             "score_us_per_layer": a_us, "select_compact_us_per_layer": b_us, "decode_attn_us_per_layer_step": c_us,
@@ -393,6 +397,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (0 = the workload's)")
     ap.add_argument("--decode-steps", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--overlap", type=int, default=None, help="sagekv_set_overlap mode for the decode phase")
     args = ap.parse_args()
     from paper_2503_08879_b200 import synth
     w = synth.workload(args.workload)

@@ -150,6 +150,22 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
                        void *Kc, void *Vc, sagekv_strides cs, const sagekv_cache_state *state,
                        void *out, float *lse, void *stream);
 
+/* How sagekv_decode_attn launches overlap with the kernel before them on the
+ * stream (Step 4 runs once per layer and per generated token, so at batch 1
+ * the launch-to-launch gap is a large share of its cost).
+ *   0  (default) plain launch: starts when the previous kernel has finished.
+ *   1  programmatic dependent launch: the kernel may be scheduled while its
+ *      predecessor drains, and waits on the device for the predecessor to
+ *      finish before it reads or writes anything.  Always safe.
+ *   2  as 1, but the rows of the reduced cache are requested BEFORE that wait.
+ *      Only for callers who guarantee that the kernel directly before a
+ *      sagekv_decode_attn call on the stream does not write the Kc / Vc passed
+ *      to that call (for example a decode call for another layer, or work that
+ *      only produces q, k_new, v_new).  q, k_new, v_new and the step counter
+ *      are still read after the wait.
+ * Errors: INVALID for a null context or a mode outside 0..2. */
+int sagekv_set_overlap(sagekv_ctx *ctx, int mode);
+
 /* The score step without any allocation (the paper has no counterpart: this is
  * a deployment variant of sagekv_score, same arithmetic, same kernels, same
  * output).  It exists for programs that cannot call cudaMalloc when they reach

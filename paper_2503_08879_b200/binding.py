@@ -50,6 +50,8 @@ lib.sagekv_select_compact.argtypes = [_vp, _vp, _i64, _vp, _vp, Strides, _i64, _
 lib.sagekv_decode_attn.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, Strides, C.POINTER(CacheState), _vp, _vp, _vp]
 lib.sagekv_score_static.argtypes = [C.POINTER(Shape), _vp, _vp, Strides, _i64, _i32, _i32, _vp, _i64, _vp]
 lib.sagekv_score_static.restype = C.c_int
+lib.sagekv_set_overlap.argtypes = [_vp, C.c_int]
+lib.sagekv_set_overlap.restype = C.c_int
 lib.sagekv_strerror.argtypes = [C.c_int]
 lib.sagekv_strerror.restype = C.c_char_p
 lib.sagekv_last_cuda_error.argtypes = [_vp]
@@ -110,6 +112,10 @@ def sagekv_score(ctx, q_last, K, n_ctx: int, n_init: int, n_recent: int, scores,
                             scores_row_stride, _stream()), "sagekv_score", ctx)
 
 
+def sagekv_set_overlap(ctx, mode: int):
+    _check(lib.sagekv_set_overlap(ctx, mode), "sagekv_set_overlap", ctx)
+
+
 def sagekv_score_static(shape: Shape, q_last, K, n_ctx: int, n_init: int, n_recent: int, scores,
                         scores_row_stride: int):
     """sagekv_score without a context or any allocation: the partials live in the library's fixed array."""
@@ -160,6 +166,9 @@ class SageKV:
         self.G = n_q_heads // n_kv_heads
         with torch.cuda.device(self.device):
             self.ctx = sagekv_create(n_q_heads, n_kv_heads, head_dim, batch, max_ctx, max_len, softmax_scale)
+
+    def set_overlap(self, mode: int):
+        sagekv_set_overlap(self.ctx, mode)
 
     def close(self):
         if self.ctx is not None:

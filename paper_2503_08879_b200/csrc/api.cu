@@ -19,6 +19,7 @@ struct sagekv_ctx {
   int max_splits;
   int32_t *tickets;         // [B*H_kv + 1], zero between launches
   int last_cuda_error;
+  int overlap;              // 0, 1 or 2: see sagekv_set_overlap
 };
 
 namespace {
@@ -53,6 +54,7 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   ctx->max_len = max_len;
   ctx->scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.0f / sqrtf((float)shape->head_dim);
   ctx->last_cuda_error = 0;
+  ctx->overlap = 0;
   int dev = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
@@ -227,8 +229,15 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
   p.H_kv = ctx->shape.n_kv_heads;
   p.B = ctx->shape.batch;
   p.scale_log2 = ctx->scale * kLog2e;
+  p.pdl_mode = ctx->overlap;
   const cudaError_t e = launch_decode(p, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
+}
+
+int sagekv_set_overlap(sagekv_ctx *ctx, int mode) {
+  if (ctx == nullptr || mode < 0 || mode > 2) return SAGEKV_ERR_INVALID;
+  ctx->overlap = mode;
+  return SAGEKV_OK;
 }
 
 const char *sagekv_strerror(int code) {

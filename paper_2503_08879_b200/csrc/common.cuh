@@ -65,6 +65,7 @@ struct DecodeParams {
   int32_t *d_step;
   int S, k_q, n_sel, ring_len, L, G, H_q, H_kv, B;
   float scale_log2;
+  int pdl_mode;            // 0 plain launch, 1 programmatic dependent launch, 2 also prefetch the cache before the wait
 };
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream);
 cudaError_t decode_setup();           // one-time function attributes

@@ -18,8 +18,8 @@
 // cluster through distributed shared memory (each CTA finishes a slice of the 128 columns), so with one
 // cluster per head nothing touches global scratch.  With several clusters per head the cluster results
 // go to scratch and the CTA that arrives last (one atomic ticket, no waiting) merges them.
-// The new token's row is read from k_new / v_new by whichever lane would have read the window slot it
-// replaces, and the CTA owning that slot stores it into the cache.
+// The staged copy of the window row that the new token replaces is overwritten in shared memory from
+// k_new / v_new once it has landed, and the CTA owning that row stores the new token into the cache.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -73,15 +73,17 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   const bool append = p.k_new != nullptr;
   cluster.barrier_arrive();                              // waited for just before the first push into a peer
 
-  int step = 0, slot = -1;
-  if (append) {
-    step = *reinterpret_cast<const volatile int32_t *>(p.d_step);
-    slot = p.S + p.n_sel + step % p.ring_len;
+  // Programmatic dependent launch: until the wait returns, nothing that an earlier kernel on the stream may
+  // still be writing is read (q, k_new, v_new, the step counter) and nothing at all is written.  In
+  // prefetch mode the rows of the reduced cache are requested first: the caller has promised that the
+  // kernel directly before this one does not write this layer's cache.  The successor is released only
+  // after the wait, so at most one kernel runs ahead of its dependency.
+  if (p.pdl_mode < 2) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
   const uint16_t *Kh = p.Kc + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride;
   const uint16_t *Vh = p.Vc + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride;
-  const uint16_t *kn = append ? p.k_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
-  const uint16_t *vn = append ? p.v_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
 
   // tiles of this CTA: an even deal of the head's n_tiles over the gridDim.x CTAs
   const int n_tiles = (p.L + 15) >> 4;
@@ -101,11 +103,23 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
       const int flat = u * 32 + lane, row = flat >> 4, piece = flat & 15;
       const int r = min(row0 + row, p.L - 1);
       const uint32_t off = row * 256 + ((piece ^ swz(row)) << 4);
-      cp_async16(tk + off, (r == slot ? kn : Kh + (int64_t)r * p.cs.token_stride) + piece * 8);
-      cp_async16(tv + off, (r == slot ? vn : Vh + (int64_t)r * p.cs.token_stride) + piece * 8);
+      cp_async16(tk + off, Kh + (int64_t)r * p.cs.token_stride + piece * 8);
+      cp_async16(tv + off, Vh + (int64_t)r * p.cs.token_stride + piece * 8);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   }
+
+  if (p.pdl_mode >= 2) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
+  int step = 0, slot = -1;
+  if (append) {
+    step = *reinterpret_cast<const volatile int32_t *>(p.d_step);
+    slot = p.S + p.n_sel + step % p.ring_len;
+  }
+  const uint16_t *kn = append ? p.k_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
+  const uint16_t *vn = append ? p.v_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
 
   // the CTA that owns the replaced window slot stores the new token's row
   if (append && warp == 0) {
@@ -143,6 +157,13 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
     const int lt = warp + i * n_warps;
     const int base = (first_tile + lt) << 4;
     const uint32_t tk = stage_base + lt * 2 * kTileBytes, tv = tk + kTileBytes;
+    if (slot >= base && slot < base + 16) {              // the staged copy of the replaced row is stale: patch it
+      const int row = slot - base, piece = lane & 15;
+      const uint4 nv = ld_v4((lane < 16 ? kn : vn) + piece * 8);
+      const uint32_t dst = (lane < 16 ? tk : tv) + row * 256 + ((piece ^ swz(row)) << 4);
+      asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(nv.x), "r"(nv.y), "r"(nv.z), "r"(nv.w) : "memory");
+      __syncwarp();
+    }
     // ---- S^T = Q K^T for rows base..base+7 (s0,s1) and base+8..base+15 (s2,s3) ----
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
     {
@@ -372,13 +393,15 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream) {
   cfg.blockDim = dim3((unsigned)(n_warps * 32), 1, 1);
   cfg.dynamicSmemBytes = (size_t)smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = cs;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = p.pdl_mode > 0 ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, decode_attn_kernel, p);
 }
 

@@ -72,7 +72,7 @@ def check_out(out, ref):
     assert np.all(err <= OUT_ATOL + OUT_RTOL * np.abs(ref)), float(err.max())
 
 
-def run_pipeline(B, w, n_decode, device="cuda", strided=False):
+def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0):
     """All four steps on one layer of workload `w`, every result checked against the oracle."""
     lay = synth.make_layer(w, 0, device)
     K, V = lay["K"], lay["V"]
@@ -83,6 +83,7 @@ def run_pipeline(B, w, n_decode, device="cuda", strided=False):
         Vp[:, :, : w.n_ctx, :128] = V
         K, V = Kp[:, :, : w.n_ctx, :128], Vp[:, :, : w.n_ctx, :128]
     sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    sk.set_overlap(overlap)
     scores = sk.score(lay["q_last"], K, w.n_init, w.n_recent)
     layer = sk.select_compact(scores, K, V, w.n_init, w.n_recent, w.n_sel)
     torch.cuda.synchronize()
@@ -201,4 +202,70 @@ def test_full_size_qwen_128k_batch4_sampled(B):
         check_out(out[b], ref)
         Kc, Vc = layer.cache()
         assert np.array_equal(bits(Kc[b]), Kc_ref) and np.array_equal(bits(Vc[b]), Vc_ref)
+    sk.close()
+
+
+def test_dependent_launch_same_layer_back_to_back(B):
+    """Overlap mode 1 (wait before touching anything) must be right for any predecessor, here the previous
+    step of the same layer, issued without host synchronisation in between."""
+    w = synth.workload("C1").with_(n_ctx=3001, budget=128, n_recent_min=8)
+    run_pipeline(B, w, 12, overlap=1)
+    dev = "cuda"
+    lay = synth.make_layer(w, 0, dev)
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    sk.set_overlap(1)
+    scores = sk.score(lay["q_last"], lay["K"], w.n_init, w.n_recent)
+    layer = sk.select_compact(scores, lay["K"], lay["V"], w.n_init, w.n_recent, w.n_sel)
+    torch.cuda.synchronize()
+    idx = layer.indices()[0].cpu().numpy()
+    Kc_ref, Vc_ref = O.compact(bits(lay["K"][0]), bits(lay["V"][0]), idx, w.n_init, w.n_recent)
+    n = 25
+    ins = [synth.make_decode_inputs(w, 0, t, dev) for t in range(n)]
+    outs = [torch.empty_like(ins[0]["q"]) for _ in range(n)]
+    for t in range(n):                                   # no synchronisation between the launches
+        sk.decode_attn(ins[t]["q"], ins[t]["k_new"], ins[t]["v_new"], layer, outs[t])
+    torch.cuda.synchronize()
+    step = 0
+    for t in range(n):
+        ref, _, step = O.decode_step(bits(ins[t]["q"][0]), bits(ins[t]["k_new"][0]), bits(ins[t]["v_new"][0]),
+                                     Kc_ref, Vc_ref, step, w.n_init, w.k_q, w.n_recent)
+        check_out(outs[t][0], ref)
+    assert int(layer.step.item()) == n
+    sk.close()
+
+
+def test_prefetch_overlap_across_layers(B):
+    """Overlap mode 2: decode calls of different layers alternate on one stream, so the kernel before each
+    call never writes that call's cache, which is what the mode asks the caller to guarantee."""
+    w = synth.workload("C2").with_(n_ctx=6000, n_layers=3)
+    dev = "cuda"
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    layers, refs = [], []
+    for l in range(3):
+        lay = synth.make_layer(w, l, dev)
+        scores = sk.score(lay["q_last"], lay["K"], w.n_init, w.n_recent)
+        layer = sk.select_compact(scores, lay["K"], lay["V"], w.n_init, w.n_recent, w.n_sel)
+        torch.cuda.synchronize()
+        idx = layer.indices()[0].cpu().numpy()
+        refs.append(list(O.compact(bits(lay["K"][0]), bits(lay["V"][0]), idx, w.n_init, w.n_recent)))
+        layers.append(layer)
+    sk.set_overlap(2)
+    n = 6
+    ins = [[synth.make_decode_inputs(w, l, t, dev) for l in range(3)] for t in range(n)]
+    outs = [[torch.empty_like(ins[0][0]["q"]) for _ in range(3)] for _ in range(n)]
+    for t in range(n):
+        for l in range(3):
+            d = ins[t][l]
+            sk.decode_attn(d["q"], d["k_new"], d["v_new"], layers[l], outs[t][l])
+    torch.cuda.synchronize()
+    steps = [0, 0, 0]
+    for t in range(n):
+        for l in range(3):
+            d = ins[t][l]
+            ref, _, steps[l] = O.decode_step(bits(d["q"][0]), bits(d["k_new"][0]), bits(d["v_new"][0]),
+                                             refs[l][0], refs[l][1], steps[l], w.n_init, w.k_q, w.n_recent)
+            check_out(outs[t][l][0], ref)
+    for l in range(3):
+        Kc, Vc = layers[l].cache()
+        assert np.array_equal(bits(Kc[0]), refs[l][0]) and np.array_equal(bits(Vc[0]), refs[l][1])
     sk.close()
