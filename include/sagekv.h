@@ -151,8 +151,10 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
                        void *out, float *lse, void *stream);
 
 /* How sagekv_decode_attn launches overlap with the kernel before them on the
- * stream (Step 4 runs once per layer and per generated token, so at batch 1
- * the launch-to-launch gap is a large share of its cost).
+ * stream.  Step 4 runs once per layer and per generated token, so at batch 1 the
+ * launch-to-launch gap is a large share of its cost.  (The score and
+ * select+compact launches are always plain: measured, early scheduling of their
+ * successors cost them more than the hidden launch latency gained.)
  *   0  (default) plain launch: starts when the previous kernel has finished.
  *   1  programmatic dependent launch: the kernel may be scheduled while its
  *      predecessor drains, and waits on the device for the predecessor to

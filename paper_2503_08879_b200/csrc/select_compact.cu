@@ -33,10 +33,10 @@ constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kMaxCluster = 8;
 constexpr int kMaxBins = 2048;
 constexpr int kSelSmemLimit = 200 * 1024;
-constexpr int kGeneralScratch = 3 * kMaxBins * 4;   // merged histograms of the general path
+constexpr int kGeneralScratch = 4 * kMaxBins * 4;   // general path: three merged histograms and the local one
 
 struct SelShared {
-  uint32_t hist_local[kMaxBins];
+  uint32_t hist_fast[kSelThreads];     // fast path: histogram of the thread maxima
   uint32_t gmax[kSelThreads];          // thread maxima of this CTA, read by the peers
   uint32_t red[3][kSelWarps];
   uint32_t gstat[kMaxCluster][4];      // (min, max, count) of every CTA's non-empty thread maxima, pushed by the peers
@@ -232,12 +232,11 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   const uint32_t base = kmin >> shift;
 #pragma unroll
   for (int r = 0; r < kMaxCluster; ++r)
-    if (gm[r] != 0u) atomicAdd(&sh.hist_local[(gm[r] >> shift) - base], 1u);
+    if (gm[r] != 0u) atomicAdd(&sh.hist_fast[(gm[r] >> shift) - base], 1u);
   __syncthreads();
-  find_bin_from_top(sh.hist_local, kSelThreads, p.k_q, sh);
+  find_bin_from_top(sh.hist_fast, kSelThreads, p.k_q, sh);
   const uint32_t T0 = (base + (uint32_t)sh.found[0]) << shift;
   const float T0f = key_to_score(T0);
-  sh.hist_local[tid] = 0;                                // leave it clean (only the first 512 bins were used)
 
   // 3. candidates: (key, position) packed so that a larger value precedes in (score desc, position asc)
   for (int v0 = 0; v0 < n_vec; v0 += 8 * kSelThreads) {
@@ -363,10 +362,11 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
 __device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t(*hist_merged)[kMaxBins] = reinterpret_cast<uint32_t(*)[kMaxBins]>(c.scratch);   // only rank 0's copy is used
+  uint32_t *hist_local = reinterpret_cast<uint32_t *>(c.scratch) + 3 * kMaxBins;
   const float *data = c.data;
   const int n_local = c.n_local;
   for (int i = tid; i < kMaxBins; i += kSelThreads) {
-    sh.hist_local[i] = 0;
+    hist_local[i] = 0;
     hist_merged[0][i] = 0; hist_merged[1][i] = 0; hist_merged[2][i] = 0;
   }
   if (tid == 0) sh.list_count = 0;
@@ -392,18 +392,18 @@ __device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const 
       const uint32_t mn = __reduce_min_sync(0xffffffffu, bin);
       const uint32_t mx = __reduce_max_sync(0xffffffffu, bin);
       if (mn == mx) {                                   // whole warp in one bin (or nothing to count)
-        if (lane == 0 && bin != 0xffffffffu) atomicAdd(&sh.hist_local[bin], 32u);
+        if (lane == 0 && bin != 0xffffffffu) atomicAdd(&hist_local[bin], 32u);
       } else if (bin != 0xffffffffu) {
-        atomicAdd(&sh.hist_local[bin], 1u);
+        atomicAdd(&hist_local[bin], 1u);
       }
     }
     __syncthreads();
     uint32_t *merged0 = cluster.map_shared_rank(&hist_merged[pass][0], 0);
     for (int bin = tid; bin < nb; bin += kSelThreads) {
-      const uint32_t v = sh.hist_local[bin];
+      const uint32_t v = hist_local[bin];
       if (v) {
         atomicAdd(merged0 + bin, v);
-        sh.hist_local[bin] = 0;
+        hist_local[bin] = 0;
       }
     }
     cluster.sync();
@@ -499,7 +499,7 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
   const int kvh = h / p.G, j = h - kvh * p.G;
   const float *grow = p.scores + (int64_t)c.row * p.row_stride + c.lo;   // 16-byte aligned: chunk % 4 == 0
 
-  for (int i = tid; i < kMaxBins; i += kSelThreads) sh.hist_local[i] = 0;
+  sh.hist_fast[tid] = 0;
   c.data = grow;
   if (resident) {
     const int n_vec = c.n_local >> 2;
@@ -541,7 +541,7 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
 }
 
 static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, bool resident) {
-  size_t scratch = (size_t)cand_cap * (8 + 8 + 4) + 16;
+  size_t scratch = (size_t)cand_cap * (8 + 8) + 16 + (size_t)list_cap * 4;   // candidates (own, all) and kept positions
   if (scratch < (size_t)kGeneralScratch) scratch = kGeneralScratch;
   return sizeof(SelShared) + (((size_t)list_cap * sizeof(int2) + 15) & ~(size_t)15) + scratch +
          (resident ? (size_t)chunk * sizeof(float) : 0);
@@ -561,9 +561,9 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   chunk = (chunk + 3) & ~3;
   if (chunk < 4) chunk = 4;
   const int list_cap = chunk < p.k_q ? chunk : (p.k_q > 0 ? p.k_q : 1);
-  // the prefilter needs at least 2*k_q thread maxima; its buffers hold 2*k_q + 256 candidates
+  // the prefilter needs at least 2*k_q thread maxima; its buffers hold 1.5*k_q + 256 candidates
   const int try_fast = select && 2 * (int64_t)p.k_q <= (int64_t)cs * kSelThreads;
-  const int cand_cap = try_fast ? 2 * p.k_q + 256 : 0;
+  const int cand_cap = try_fast ? (p.k_q + p.k_q / 2 + 256) & ~1 : 0;
   const bool resident = select_smem_bytes(chunk, list_cap, cand_cap, true) <= (size_t)kSelSmemLimit;
   const size_t smem = select_smem_bytes(chunk, list_cap, cand_cap, resident);
 
