@@ -58,8 +58,8 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
 
 __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char stage[];          // tiles: [K 4 KB | V 4 KB] each
-  __shared__ float inbox_o[kMaxGroup * kHeadDim];                   // [source CTA][head][my columns], pushed by the peers
-  __shared__ float inbox_m[kDecodeMaxCluster * kMaxGroup], inbox_l[kDecodeMaxCluster * kMaxGroup];
+  __shared__ __align__(16) float inbox_o[kMaxGroup * kHeadDim];     // [source CTA][head][my columns], pushed by the peers
+  __shared__ float2 inbox_ml[kDecodeMaxCluster * kMaxGroup];        // [source CTA][head] (max, sum)
   __shared__ float sm_m[kDecodeMaxWarps][kMaxGroup], sm_l[kDecodeMaxWarps][kMaxGroup];
   __shared__ int sm_last;
 
@@ -256,22 +256,30 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   __syncthreads();
   cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs
 
-  // ---- push this CTA's result to the peers: the owner of a column slice receives it from every CTA ----
-  const int cols = kHeadDim / cs;                        // columns each CTA of the cluster finishes
-  for (int idx = tid; idx < kMaxGroup * kHeadDim; idx += blockDim.x) {
-    float o = 0.f;
-    for (int w = 0; w < n_act; ++w) o += xo[w * kMaxGroup * kHeadDim + idx];
-    const int h = idx & 7, col = (idx >> 9) * 64 + ((idx >> 3) & 7) * 8 + ((idx >> 6) & 7);
-    const int owner = col / cols;
-    cluster.map_shared_rank(inbox_o, owner)[(rank * kMaxGroup + h) * cols + (col - owner * cols)] = o;
+  // ---- push this CTA's result to the peers: the owner of a column slice receives it from every CTA.
+  // One thread sums four neighbouring columns of one head over the warps and sends them as one 16-byte store.
+  const int cols = kHeadDim / cs;                        // columns each CTA of the cluster finishes (a multiple of 4)
+  for (int item = tid; item < p.G * (kHeadDim / 4); item += blockDim.x) {
+    const int h = item >> 5, col0 = (item & 31) * 4;
+    const float *src = xo + (((col0 >> 6) * 8 + (col0 & 7)) * 8 + ((col0 >> 3) & 7)) * 8 + h;   // column col0 + e: + 64*e
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int w = 0; w < n_act; ++w) {
+      const float *sw = src + w * kMaxGroup * kHeadDim;
+      o.x += sw[0]; o.y += sw[64]; o.z += sw[128]; o.w += sw[192];
+    }
+    const int owner = col0 / cols;
+    *reinterpret_cast<float4 *>(cluster.map_shared_rank(inbox_o, owner) + (rank * kMaxGroup + h) * cols +
+                                (col0 - owner * cols)) = o;
   }
-  for (int item = tid; item < kMaxGroup * cs; item += blockDim.x) {
-    const int h = item & 7, dst = item >> 3;
-    float M = -INFINITY, l = 0.f;
-    for (int w = 0; w < n_act; ++w) M = fmaxf(M, sm_m[w][h]);
-    for (int w = 0; w < n_act; ++w) l += M == -INFINITY ? 0.f : sm_l[w][h] * fast_exp2(sm_m[w][h] - M);
-    cluster.map_shared_rank(inbox_m, dst)[rank * kMaxGroup + h] = M;
-    cluster.map_shared_rank(inbox_l, dst)[rank * kMaxGroup + h] = l;
+  for (int h = warp; h < p.G; h += n_warps) {            // one warp per head, one lane per contributing warp
+    const float mw = lane < n_act ? sm_m[lane][h] : -INFINITY;
+    float M = mw;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+    float l = (lane < n_act && M != -INFINITY) ? sm_l[lane][h] * fast_exp2(mw - M) : 0.f;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+    if (lane < cs) cluster.map_shared_rank(inbox_ml, lane)[rank * kMaxGroup + h] = make_float2(M, l);
   }
   cluster.sync();   // all pushes have landed; no shared memory of a peer is touched after this point
 
@@ -282,12 +290,13 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   for (int item = tid; item < p.G * cols; item += blockDim.x) {
     const int h = item / cols, lc = item - h * cols, col = rank * cols + lc;
     float M = -INFINITY;
-    for (int r = 0; r < cs; ++r) M = fmaxf(M, inbox_m[r * kMaxGroup + h]);
+    for (int r = 0; r < cs; ++r) M = fmaxf(M, inbox_ml[r * kMaxGroup + h].x);
     float o = 0.f, l = 0.f;
     for (int r = 0; r < cs; ++r) {
-      const float wgt = M == -INFINITY ? 0.f : fast_exp2(inbox_m[r * kMaxGroup + h] - M);
+      const float2 ml = inbox_ml[r * kMaxGroup + h];
+      const float wgt = M == -INFINITY ? 0.f : fast_exp2(ml.x - M);
       o += inbox_o[(r * kMaxGroup + h) * cols + lc] * wgt;
-      l += inbox_l[r * kMaxGroup + h] * wgt;
+      l += ml.y * wgt;
     }
     if (n_clusters == 1) {
       const float outv = l > 0.f ? o / l : 0.f;
