@@ -150,82 +150,100 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
 
-  for (int i = 0; i < n_mine; ++i) {
-    if (i + 1 < n_mine) asm volatile("cp.async.wait_group 1;" ::: "memory");
-    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+  // A warp with two tiles works on both at once: twice as many independent mma chains, one softmax update.
+  if (n_mine > 0) {
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncwarp();
-    const int lt = warp + i * n_warps;
-    const int base = (first_tile + lt) << 4;
-    const uint32_t tk = stage_base + lt * 2 * kTileBytes, tv = tk + kTileBytes;
-    if (slot >= base && slot < base + 16) {              // the staged copy of the replaced row is stale: patch it
-      const int row = slot - base, piece = lane & 15;
-      const uint4 nv = ld_v4((lane < 16 ? kn : vn) + piece * 8);
-      const uint32_t dst = (lane < 16 ? tk : tv) + row * 256 + ((piece ^ swz(row)) << 4);
-      asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(nv.x), "r"(nv.y), "r"(nv.z), "r"(nv.w) : "memory");
-      __syncwarp();
+    uint32_t tk[2], tv[2];
+    int base[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int lt = warp + (t < n_mine ? t : 0) * n_warps;
+      base[t] = (first_tile + lt) << 4;
+      tk[t] = stage_base + lt * 2 * kTileBytes;
+      tv[t] = tk[t] + kTileBytes;
+      if (t < n_mine && slot >= base[t] && slot < base[t] + 16) {   // the staged copy of the replaced row is stale: patch it
+        const int row = slot - base[t], piece = lane & 15;
+        const uint4 nv = ld_v4((lane < 16 ? kn : vn) + piece * 8);
+        const uint32_t dst = (lane < 16 ? tk[t] : tv[t]) + row * 256 + ((piece ^ swz(row)) << 4);
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(nv.x), "r"(nv.y), "r"(nv.z), "r"(nv.w) : "memory");
+      }
     }
-    // ---- S^T = Q K^T for rows base..base+7 (s0,s1) and base+8..base+15 (s2,s3) ----
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+    __syncwarp();
+    // ---- S^T = Q K^T: per tile, rows base..base+7 -> sv[t][0..1], rows base+8..base+15 -> sv[t][2..3] ----
+    float sv[2][4];
     {
-      const uint32_t ra = tk + g * 256, rb = tk + (g + 8) * 256;
+      float z[2][4];
+#pragma unroll
+      for (int t = 0; t < 2; ++t)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { sv[t][e] = 0.f; z[t][e] = 0.f; }
       const int sa = swz(g), sb = swz(g + 8);
 #pragma unroll
       for (int jj = 0; jj < 4; ++jj) {
-        const uint4 ka = lds_v4(ra + (((c + 4 * jj) ^ sa) << 4));
-        const uint4 kb = lds_v4(rb + (((c + 4 * jj) ^ sb) << 4));
-        mma_bf16_16816(s0, s1, z0, z1, qf[jj].x, 0u, qf[jj].y, 0u, ka.x, ka.y);
-        mma_bf16_16816(s0, s1, z0, z1, qf[jj].z, 0u, qf[jj].w, 0u, ka.z, ka.w);
-        mma_bf16_16816(s2, s3, z2, z3, qf[jj].x, 0u, qf[jj].y, 0u, kb.x, kb.y);
-        mma_bf16_16816(s2, s3, z2, z3, qf[jj].z, 0u, qf[jj].w, 0u, kb.z, kb.w);
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          if (t < n_mine) {
+            const uint4 ka = lds_v4(tk[t] + g * 256 + (((c + 4 * jj) ^ sa) << 4));
+            const uint4 kb = lds_v4(tk[t] + (g + 8) * 256 + (((c + 4 * jj) ^ sb) << 4));
+            mma_bf16_16816(sv[t][0], sv[t][1], z[t][0], z[t][1], qf[jj].x, 0u, qf[jj].y, 0u, ka.x, ka.y);
+            mma_bf16_16816(sv[t][2], sv[t][3], z[t][2], z[t][3], qf[jj].x, 0u, qf[jj].y, 0u, kb.x, kb.y);
+            mma_bf16_16816(sv[t][0], sv[t][1], z[t][0], z[t][1], qf[jj].z, 0u, qf[jj].w, 0u, ka.z, ka.w);
+            mma_bf16_16816(sv[t][2], sv[t][3], z[t][2], z[t][3], qf[jj].z, 0u, qf[jj].w, 0u, kb.z, kb.w);
+          }
+        }
       }
     }
-    float sv[4] = {s0 * p.scale_log2, s1 * p.scale_log2, s2 * p.scale_log2, s3 * p.scale_log2};
     float tile_max = -INFINITY;
 #pragma unroll
-    for (int s = 0; s < 4; ++s) {
-      const int r = base + 2 * c + (s & 1) + (s >> 1) * 8;
-      const bool vis = g < p.G && r < p.L && (r < p.S || r >= win_lo || (r >= seg_lo && r < seg_hi));
-      sv[s] = vis ? sv[s] : -INFINITY;
-      tile_max = fmaxf(tile_max, sv[s]);
+    for (int t = 0; t < 2; ++t) {
+#pragma unroll
+      for (int s = 0; s < 4; ++s) {
+        const int r = base[t] + 2 * c + (s & 1) + (s >> 1) * 8;
+        const bool vis = t < n_mine && g < p.G && r < p.L && (r < p.S || r >= win_lo || (r >= seg_lo && r < seg_hi));
+        sv[t][s] = vis ? sv[t][s] * p.scale_log2 : -INFINITY;
+        tile_max = fmaxf(tile_max, sv[t][s]);
+      }
     }
     tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 1));
     tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 2));
-    const float m_new = fmaxf(m_run, tile_max);
-    const float m_safe = m_new == -INFINITY ? 0.f : m_new;
-    const float alpha = fast_exp2(m_run - m_safe);      // 0 while nothing has been seen
-    float pw[4];
-#pragma unroll
-    for (int s = 0; s < 4; ++s) pw[s] = fast_exp2(sv[s] - m_safe);
+    m_run = tile_max;                                     // the warp's only pass: nothing to rescale
+    const float m_safe = m_run == -INFINITY ? 0.f : m_run;
     // the weights enter the second product as bf16; sum the rounded values so numerator and denominator agree
-    const uint32_t pb0 = pack_bf16x2(pw[0], pw[1]), pb1 = pack_bf16x2(pw[2], pw[3]);
-    l_run = l_run * alpha + (__uint_as_float(pb0 << 16) + __uint_as_float(pb0 & 0xffff0000u)) +
-            (__uint_as_float(pb1 << 16) + __uint_as_float(pb1 & 0xffff0000u));
-    m_run = m_new;
-    // rescale factors of heads 2c and 2c+1 live in the lanes of groups 2c and 2c+1
-    const float al0 = __shfl_sync(0xffffffffu, alpha, (2 * c) * 4);
-    const float al1 = __shfl_sync(0xffffffffu, alpha, (2 * c + 1) * 4);
+    uint32_t pb[2][2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      pb[t][0] = pack_bf16x2(fast_exp2(sv[t][0] - m_safe), fast_exp2(sv[t][1] - m_safe));
+      pb[t][1] = pack_bf16x2(fast_exp2(sv[t][2] - m_safe), fast_exp2(sv[t][3] - m_safe));
+      l_run += (__uint_as_float(pb[t][0] << 16) + __uint_as_float(pb[t][0] & 0xffff0000u)) +
+               (__uint_as_float(pb[t][1] << 16) + __uint_as_float(pb[t][1] & 0xffff0000u));
+    }
     // ---- O^T += V^T P: rows 2c, 2c+1, 2c+8, 2c+9 at columns 8g..8g+7 and 64+8g..64+8g+7 ----
-    uint32_t vrow[4];
     int vs[4];
+    uint32_t voff[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
       const int row = 2 * c + (s & 1) + (s >> 1) * 8;
-      vrow[s] = tv + row * 256;
+      voff[s] = row * 256;
       vs[s] = swz(row);
     }
 #pragma unroll
     for (int piece = 0; piece < 2; ++piece) {
-      uint4 vv[4];
 #pragma unroll
-      for (int s = 0; s < 4; ++s) vv[s] = lds_v4(vrow[s] + (((g + 8 * piece) ^ vs[s]) << 4));
+      for (int t = 0; t < 2; ++t) {
+        if (t < n_mine) {
+          uint4 vv[4];
 #pragma unroll
-      for (int reg = 0; reg < 4; ++reg) {
-        const int mt = piece * 4 + reg;                  // columns piece*64 + 8g + 2*reg (+1)
-        const uint32_t v0 = reg_of(vv[0], reg), v1 = reg_of(vv[1], reg);
-        const uint32_t v2 = reg_of(vv[2], reg), v3 = reg_of(vv[3], reg);
-        acc[mt][0] *= al0; acc[mt][1] *= al1; acc[mt][2] *= al0; acc[mt][3] *= al1;
-        mma_bf16_16816(acc[mt][0], acc[mt][1], acc[mt][2], acc[mt][3], prmt(v0, v1, 0x5410u), prmt(v0, v1, 0x7632u),
-                       prmt(v2, v3, 0x5410u), prmt(v2, v3, 0x7632u), pb0, pb1);
+          for (int s = 0; s < 4; ++s) vv[s] = lds_v4(tv[t] + voff[s] + (((g + 8 * piece) ^ vs[s]) << 4));
+#pragma unroll
+          for (int reg = 0; reg < 4; ++reg) {
+            const int mt = piece * 4 + reg;              // columns piece*64 + 8g + 2*reg (+1)
+            const uint32_t v0 = reg_of(vv[0], reg), v1 = reg_of(vv[1], reg);
+            const uint32_t v2 = reg_of(vv[2], reg), v3 = reg_of(vv[3], reg);
+            mma_bf16_16816(acc[mt][0], acc[mt][1], acc[mt][2], acc[mt][3], prmt(v0, v1, 0x5410u),
+                           prmt(v0, v1, 0x7632u), prmt(v2, v3, 0x5410u), prmt(v2, v3, 0x7632u), pb[t][0], pb[t][1]);
+          }
+        }
       }
     }
   }
