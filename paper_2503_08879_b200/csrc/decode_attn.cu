@@ -277,17 +277,22 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   // ---- push this CTA's result to the peers: the owner of a column slice receives it from every CTA.
   // One thread sums four neighbouring columns of one head over the warps and sends them as one 16-byte store.
   const int cols = kHeadDim / cs;                        // columns each CTA of the cluster finishes (a multiple of 4)
-  for (int item = tid; item < p.G * (kHeadDim / 4); item += blockDim.x) {
-    const int h = item >> 5, col0 = (item & 31) * 4;
-    const float *src = xo + (((col0 >> 6) * 8 + (col0 & 7)) * 8 + ((col0 >> 3) & 7)) * 8 + h;   // column col0 + e: + 64*e
-    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int w = 0; w < n_act; ++w) {
-      const float *sw = src + w * kMaxGroup * kHeadDim;
-      o.x += sw[0]; o.y += sw[64]; o.z += sw[128]; o.w += sw[192];
+  // A warp's 32 items are 8 column groups (g) x 4 heads at one (piece, e): their exchange addresses g*8 + h
+  // fall into 32 different banks.
+  for (int item = tid; item < 8 * 32; item += blockDim.x) {
+    const int g8 = item & 7, h = ((item >> 3) & 3) + ((item >> 5) & 1) * 4, pg = item >> 6;   // pg = piece*2 + e0/4
+    if (h < p.G) {
+      const int col0 = (pg >> 1) * 64 + g8 * 8 + (pg & 1) * 4;
+      const float *src = xo + (((pg >> 1) * 8 + (pg & 1) * 4) * 8 + g8) * 8 + h;             // column col0 + e: + 64*e
+      float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int w = 0; w < n_act; ++w) {
+        const float *sw = src + w * kMaxGroup * kHeadDim;
+        o.x += sw[0]; o.y += sw[64]; o.z += sw[128]; o.w += sw[192];
+      }
+      const int owner = col0 / cols;
+      *reinterpret_cast<float4 *>(cluster.map_shared_rank(inbox_o, owner) + (rank * kMaxGroup + h) * cols +
+                                  (col0 - owner * cols)) = o;
     }
-    const int owner = col0 / cols;
-    *reinterpret_cast<float4 *>(cluster.map_shared_rank(inbox_o, owner) + (rank * kMaxGroup + h) * cols +
-                                (col0 - owner * cols)) = o;
   }
   for (int h = warp; h < p.G; h += n_warps) {            // one warp per head, one lane per contributing warp
     const float mw = lane < n_act ? sm_m[lane][h] : -INFINITY;
@@ -361,12 +366,12 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
     }
   }
   // ---- the last KV head to finish advances the step counter ----
-  if (head_done && tid == 0) {
+  // (every CTA read the counter before it got here, so the update cannot reach a reader of this launch)
+  if (append && head_done && tid == 0) {
     const int n_heads = p.B * p.H_kv;
-    __threadfence();
     if (atomicAdd(&p.tickets[n_heads], 1) == n_heads - 1) {
       p.tickets[n_heads] = 0;
-      if (append) *p.d_step = step + 1;
+      *p.d_step = step + 1;
     }
   }
 }
