@@ -12,8 +12,8 @@
 //      are >= T0.  T0 is taken as the lower edge of the histogram bin (2048 bins laid over the actual
 //      range of the maxima) in which that maximum falls.
 //   2. scores >= T0 become candidates (order-preserving key, position); the lists are exchanged.
-//   3. every CTA ranks its own candidates against all candidates (8 threads per candidate); rank < k_q
-//      means kept.  Keys are compared with the position as tie-break, so the lowest positions win ties.
+//   3. a histogram of all candidate keys finds the bin of the k_q-th largest; own candidates above it are
+//      kept, the few inside it are ranked exactly, with the position as tie-break (lowest positions win).
 //   4. kept counts are exchanged; slot = kept in lower CTAs + kept before it in this CTA: ascending order.
 // General path (k_q large, tiny rows, or more candidates than the buffers hold, e.g. a row of equal
 // scores): three-digit radix select (11 + 11 + 10 bits) with histograms merged in CTA 0's shared memory by
@@ -237,6 +237,7 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   find_bin_from_top(sh.hist_fast, kSelThreads, p.k_q, sh);
   const uint32_t T0 = (base + (uint32_t)sh.found[0]) << shift;
   const float T0f = key_to_score(T0);
+  sh.hist_fast[tid] = 0;                                 // reused in step 4 (barriers in between)
 
   // 3. candidates: (key, position) packed so that a larger value precedes in (score desc, position asc)
   for (int v0 = 0; v0 < n_vec; v0 += 8 * kSelThreads) {
@@ -289,40 +290,40 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   }
   __syncthreads();
 
-  // 4. rank of every own candidate among all candidates.  A group of tpc threads takes four own candidates
-  //    (four independent compare chains per loaded pair of candidates) and strides over the full list.
-  const int n_quads = (n_loc + 3) >> 2;
-  int tpc = 32;
-  while (tpc > 1 && n_quads * tpc > kSelThreads) tpc >>= 1;
-  const int sub = tid & (tpc - 1);
-  const int M2 = (M + 1) >> 1;
-  if ((M & 1) && tid == 0) cand_all[M] = 0ull;           // pad to an even count with a value that precedes nothing
-  __syncthreads();
-  const uint32_t all_addr = (uint32_t)__cvta_generic_to_shared(cand_all);
-  for (int q0 = 0; q0 < n_quads; q0 += kSelThreads / tpc) {
-    const int qi = q0 + tid / tpc;
-    unsigned long long mine[4];
-    int before[4] = {0, 0, 0, 0};
-#pragma unroll
-    for (int u = 0; u < 4; ++u) mine[u] = (qi < n_quads && 4 * qi + u < n_loc) ? cand_local[4 * qi + u] : ~0ull;
-    if (qi < n_quads) {
-#pragma unroll 2
-      for (int i = sub; i < M2; i += tpc) {
-        unsigned long long ox, oy;
-        asm volatile("ld.shared.v2.u64 {%0,%1}, [%2];" : "=l"(ox), "=l"(oy) : "r"(all_addr + 16u * (uint32_t)i));
-#pragma unroll
-        for (int u = 0; u < 4; ++u) before[u] += (ox > mine[u] ? 1 : 0) + (oy > mine[u] ? 1 : 0);
+  // 4. which own candidates are kept.  A 512-bin histogram of ALL candidate keys over [T0, row maximum]
+  //    locates the bin b1 holding the k_q-th largest candidate: higher bins are kept, lower bins dropped,
+  //    and only the few candidates inside b1 are ranked exactly (key, then position) against their bin.
+  {
+    const uint32_t d2 = kmax ^ T0;
+    const int hb = d2 ? 31 - __clz(d2) : -1;
+    const int shift2 = hb > 8 ? hb - 8 : 0;
+    const uint32_t base2 = T0 >> shift2;
+    for (int i = tid; i < M; i += kSelThreads)
+      atomicAdd(&sh.hist_fast[(uint32_t)(cand_all[i] >> (32 + shift2)) - base2], 1u);
+    __syncthreads();
+    find_bin_from_top(sh.hist_fast, kSelThreads, p.k_q, sh);
+    const uint32_t b1 = (uint32_t)sh.found[0];
+    const int r1 = sh.found[1];                          // the k_q-th largest is the r1-th largest inside b1
+    for (int ci = tid; ci < n_loc; ci += kSelThreads) {  // the clear cases, one thread each
+      const unsigned long long mine = cand_local[ci];
+      if ((uint32_t)(mine >> (32 + shift2)) - base2 > b1) {
+        const int n = atomicAdd(&sh.n_sel_local, 1);
+        sel_pos[n] = (int)(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
       }
     }
+    for (int ci = warp; ci < n_loc; ci += kSelWarps) {   // the border cases, one warp each
+      const unsigned long long mine = cand_local[ci];
+      if ((uint32_t)(mine >> (32 + shift2)) - base2 == b1) {
+        int before = 0;
+        for (int i = lane; i < M; i += 32) {
+          const unsigned long long o = cand_all[i];
+          before += ((uint32_t)(o >> (32 + shift2)) - base2 == b1 && o > mine) ? 1 : 0;
+        }
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
-      for (int off = 1; off < tpc; off <<= 1) before[u] += __shfl_xor_sync(0xffffffffu, before[u], off);
-    if (qi < n_quads && sub == 0) {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (4 * qi + u < n_loc && before[u] < p.k_q) {
+        for (int off = 1; off < 32; off <<= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
+        if (lane == 0 && before < r1) {
           const int n = atomicAdd(&sh.n_sel_local, 1);
-          sel_pos[n] = (int)(0xffffffffu - (uint32_t)(mine[u] & 0xffffffffull));
+          sel_pos[n] = (int)(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
         }
       }
     }
