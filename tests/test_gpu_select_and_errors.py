@@ -78,6 +78,27 @@ def test_select_ties_lowest_position_wins(B):
         assert np.array_equal(idx, O.select(rows, k_q, 3))
 
 
+def test_select_tie_group_straddles_the_cut_in_the_prefilter_path(B):
+    """Few enough equal scores that the prefilter path is taken, placed so that the k-th score lies inside
+    the group: exactly the lowest positions of the group must be kept."""
+    E, k_q = 60000, 300
+    rng = np.random.default_rng(11)
+    rows = (rng.random((4, E), dtype=np.float32) * 0.5).astype(np.float32)
+    for h in range(4):
+        top = rng.choice(E, 280, replace=False)               # 280 clear winners
+        rows[h, top] = 0.9 + 0.05 * rng.random(280, dtype=np.float32)
+        rest = np.setdiff1d(np.arange(E), top)
+        tie = rng.choice(rest, 40, replace=False)             # 40 equal scores: 20 of them make the cut
+        rows[h, tie] = 0.75
+    idx = run_select(B, rows, k_q, H_kv=2)
+    want = O.select(rows, k_q, 3)
+    assert np.array_equal(idx, want)
+    for h in range(4):
+        tie_pos = np.sort(np.nonzero(rows[h] == np.float32(0.75))[0]) + 3
+        kept = np.intersect1d(idx[h], tie_pos)
+        assert np.array_equal(kept, tie_pos[:20])
+
+
 def test_select_threshold_differs_only_in_low_bits(B):
     E = 20000
     base = np.float32(0.001)
