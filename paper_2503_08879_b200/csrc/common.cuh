@@ -47,8 +47,9 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
 cudaError_t select_compact_setup();   // one-time function attributes
 
 // ---- decode attention ------------------------------------------------------
-constexpr int kDecodeMaxWarps = 16;                                    // warps per CTA, one or two 16-row tiles each
-constexpr int kDecodeMaxCluster = 16;                                  // CTAs per cluster (8 where 16 is not available)
+constexpr int kDecodeMaxWarps = 12;                                    // warps per CTA, one or two 16-row tiles each
+constexpr int kDecodeMaxCluster = 8;                                   // CTAs per cluster (the portable limit)
+constexpr int kDecodeMaxPasses = 4;                                    // passes over the staging area before a head gets more clusters
 constexpr int kDecodeMaxTiles = 24;                                    // 16-row tiles (K and V) a CTA can stage: 192 KB
 constexpr int kPartialStride = kMaxGroup * kHeadDim + 2 * kMaxGroup;   // floats per cluster result: O[8][128], m[8], l[8]
 

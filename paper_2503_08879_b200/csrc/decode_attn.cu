@@ -2,10 +2,11 @@
 // of the reduced cache (sink + its own selected segment + window).
 //
 // Flash-decoding on thread-block clusters.  The L rows of one KV head are cut into 16-row tiles that are
-// dealt evenly to the CTAs of one cluster (more clusters per head only when L exceeds what a cluster's
-// shared memory holds).  Every warp owns one or two tiles.  It first issues 16-byte cp.async copies for
-// all its K and V rows, so the whole partition is in flight at once and costs no registers, then works
-// through its tiles as they land:
+// dealt evenly to the CTAs of one cluster.  Every warp owns two staging slots: it issues 16-byte cp.async
+// copies for the K and V rows of its first two tiles at once (in flight together, no registers held),
+// works on both tiles, and, when the partition is longer than the staging area, refills its own two
+// slots for the next pass (no block-wide synchronisation: the slots belong to the warp).  Only beyond
+// four passes does a head get more than one cluster.  Per pair of tiles:
 //   S^T = Q K^T   heads (padded to 16) x 8 rows per mma.  Lane (g, c) reads 16-byte pieces of rows g and
 //                 g+8; the query fragment uses the same column permutation, so fragments come straight
 //                 from the staged rows with no transposition.
@@ -56,6 +57,8 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 
+// kPasses: the CTA's partition is longer than its staging area (false keeps the common case free of the pass loop)
+template <bool kPasses>
 __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char stage[];          // tiles: [K 4 KB | V 4 KB] each
   __shared__ __align__(16) float inbox_o[kMaxGroup * kHeadDim];     // [source CTA][head][my columns], pushed by the peers
@@ -90,14 +93,13 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   const int base_n = n_tiles / (int)gridDim.x, rem = n_tiles % (int)gridDim.x;
   const int first_tile = ci * base_n + min(ci, rem);
   const int my_tiles = base_n + (ci < rem ? 1 : 0);
-  const int n_mine = warp < my_tiles ? (my_tiles - warp + n_warps - 1) / n_warps : 0;   // tiles of this warp: 0, 1 or 2
+  const int n_mine = warp < my_tiles ? (my_tiles - warp + n_warps - 1) / n_warps : 0;   // tiles of this warp
 
-  // ---- issue every copy of this warp's tiles ----
+  // ---- issue the copies of this warp's first two tiles (its later tiles reuse the same two slots) ----
   const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(stage);
-  for (int i = 0; i < n_mine; ++i) {
-    const int lt = warp + i * n_warps;
-    const int row0 = (first_tile + lt) << 4;
-    const uint32_t tk = stage_base + lt * 2 * kTileBytes, tv = tk + kTileBytes;
+  auto issue_tile = [&](int i) {   // i-th tile of this warp -> slot i & 1
+    const int row0 = (first_tile + warp + i * n_warps) << 4;
+    const uint32_t tk = stage_base + (warp + (i & 1) * n_warps) * 2 * kTileBytes, tv = tk + kTileBytes;
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const int flat = u * 32 + lane, row = flat >> 4, piece = flat & 15;
@@ -106,8 +108,9 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
       cp_async16(tk + off, Kh + (int64_t)r * p.cs.token_stride + piece * 8);
       cp_async16(tv + off, Vh + (int64_t)r * p.cs.token_stride + piece * 8);
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-  }
+  };
+  for (int i = 0; i < min(n_mine, 2); ++i) issue_tile(i);
+  asm volatile("cp.async.commit_group;" ::: "memory");
 
   if (p.pdl_mode >= 2) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -150,19 +153,25 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
 
-  // A warp with two tiles works on both at once: twice as many independent mma chains, one softmax update.
-  if (n_mine > 0) {
+  // A warp works on two tiles at once (twice as many independent mma chains, one softmax update) and,
+  // when the partition is longer than the staging area, goes through its tiles in passes of two.
+  for (int i0 = 0; i0 < (kPasses ? n_mine : min(n_mine, 2)); i0 += 2) {
+    const int nt = min(2, n_mine - i0);                    // tiles of this pass
+    if (kPasses && i0 > 0) {                                          // the slots are free: this warp alone used them
+      __syncwarp();
+      for (int i = i0; i < i0 + nt; ++i) issue_tile(i);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncwarp();
     uint32_t tk[2], tv[2];
     int base[2];
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
-      const int lt = warp + (t < n_mine ? t : 0) * n_warps;
-      base[t] = (first_tile + lt) << 4;
-      tk[t] = stage_base + lt * 2 * kTileBytes;
+      base[t] = (first_tile + warp + (i0 + (t < nt ? t : 0)) * n_warps) << 4;
+      tk[t] = stage_base + (warp + (t < nt ? t : 0) * n_warps) * 2 * kTileBytes;
       tv[t] = tk[t] + kTileBytes;
-      if (t < n_mine && slot >= base[t] && slot < base[t] + 16) {   // the staged copy of the replaced row is stale: patch it
+      if (t < nt && slot >= base[t] && slot < base[t] + 16) {   // the staged copy of the replaced row is stale: patch it
         const int row = slot - base[t], piece = lane & 15;
         const uint4 nv = ld_v4((lane < 16 ? kn : vn) + piece * 8);
         const uint32_t dst = (lane < 16 ? tk[t] : tv[t]) + row * 256 + ((piece ^ swz(row)) << 4);
@@ -183,7 +192,7 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
       for (int jj = 0; jj < 4; ++jj) {
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-          if (t < n_mine) {
+          if (t < nt) {
             const uint4 ka = lds_v4(tk[t] + g * 256 + (((c + 4 * jj) ^ sa) << 4));
             const uint4 kb = lds_v4(tk[t] + (g + 8) * 256 + (((c + 4 * jj) ^ sb) << 4));
             mma_bf16_16816(sv[t][0], sv[t][1], z[t][0], z[t][1], qf[jj].x, 0u, qf[jj].y, 0u, ka.x, ka.y);
@@ -200,15 +209,24 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
 #pragma unroll
       for (int s = 0; s < 4; ++s) {
         const int r = base[t] + 2 * c + (s & 1) + (s >> 1) * 8;
-        const bool vis = t < n_mine && g < p.G && r < p.L && (r < p.S || r >= win_lo || (r >= seg_lo && r < seg_hi));
+        const bool vis = t < nt && g < p.G && r < p.L && (r < p.S || r >= win_lo || (r >= seg_lo && r < seg_hi));
         sv[t][s] = vis ? sv[t][s] * p.scale_log2 : -INFINITY;
         tile_max = fmaxf(tile_max, sv[t][s]);
       }
     }
     tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 1));
     tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 2));
-    m_run = tile_max;                                     // the warp's only pass: nothing to rescale
-    const float m_safe = m_run == -INFINITY ? 0.f : m_run;
+    const float m_new = fmaxf(m_run, tile_max);
+    const float m_safe = m_new == -INFINITY ? 0.f : m_new;
+    if (kPasses && i0 > 0) {                              // a later pass: bring sum and accumulators to the new maximum
+      const float alpha = fast_exp2(m_run - m_safe);
+      l_run *= alpha;
+      // the factors of heads 2c and 2c+1 live in the lanes of groups 2c and 2c+1
+      const float al0 = __shfl_sync(0xffffffffu, alpha, (2 * c) * 4), al1 = __shfl_sync(0xffffffffu, alpha, (2 * c + 1) * 4);
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) { acc[mt][0] *= al0; acc[mt][1] *= al1; acc[mt][2] *= al0; acc[mt][3] *= al1; }
+    }
+    m_run = m_new;
     // the weights enter the second product as bf16; sum the rounded values so numerator and denominator agree
     uint32_t pb[2][2];
 #pragma unroll
@@ -231,7 +249,7 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
     for (int piece = 0; piece < 2; ++piece) {
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
-        if (t < n_mine) {
+        if (t < nt) {
           uint4 vv[4];
 #pragma unroll
           for (int s = 0; s < 4; ++s) vv[s] = lds_v4(tv[t] + voff[s] + (((g + 8 * piece) ^ vs[s]) << 4));
@@ -376,45 +394,33 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   }
 }
 
-static int g_max_cluster = 8;   // 16 where the device can co-schedule 16-CTA clusters of this kernel
-
+// Clusters of 8 CTAs, the portable limit.  (16-CTA clusters were tried: too few of them are co-resident on
+// this part, so the grid ran in two waves.)
 cudaError_t decode_setup() {
-  cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kDecodeMaxTiles * 2 * kTileBytes);
   if (e != cudaSuccess) return e;
-  // clusters of 16 are beyond the portable size: allow them and ask whether enough of them fit
-  g_max_cluster = 8;
-  if (cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(16, 8, 1);
-    cfg.blockDim = dim3(kDecodeMaxWarps * 32, 1, 1);
-    cfg.dynamicSmemBytes = 12 * 2 * kTileBytes;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 16;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, decode_attn_kernel, &cfg) == cudaSuccess && n >= 64) g_max_cluster = 16;
-  }
-  cudaGetLastError();
-  return cudaSuccess;
+  return cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kDecodeMaxTiles * 2 * kTileBytes);
 }
 
-// Launch geometry for a reduced cache of L rows.
+// Launch geometry for a reduced cache of L rows: one cluster per KV head whose CTAs go through their
+// tiles in passes of (two tiles per warp); more clusters per head only beyond kDecodeMaxPasses passes.
 void decode_geometry(int L, int *n_clusters, int *cs, int *n_warps, int *smem_bytes) {
   const int n_tiles = (L + 15) / 16;
   int c = 1;
-  while (c < g_max_cluster && c * 2 <= n_tiles) c <<= 1;                         // cluster size 1, 2, 4, 8 or 16
-  const int nc = (n_tiles + c * kDecodeMaxTiles - 1) / (c * kDecodeMaxTiles);    // clusters per head
+  while (c < kDecodeMaxCluster && c * 2 <= n_tiles) c <<= 1;                     // cluster size 1, 2, 4 or 8
+  const int per_pass = kDecodeMaxTiles;                                          // tiles a CTA can stage at once
+  const int nc = (n_tiles + c * per_pass * kDecodeMaxPasses - 1) / (c * per_pass * kDecodeMaxPasses);
   const int per_cta = (n_tiles + c * nc - 1) / (c * nc);                         // most tiles a CTA gets
-  const int rounds = (per_cta + kDecodeMaxWarps - 1) / kDecodeMaxWarps;          // 1 or 2 tiles per warp
+  int w = (per_cta + 1) / 2;                                                     // two tiles per warp and pass
+  if (per_cta > 2 * 9) w = kDecodeMaxTiles / 2;                                  // several passes: use every slot
+  else if (w > 9) w = 9;
+  if (w < 1) w = 1;
   *n_clusters = nc;
   *cs = c;
-  *n_warps = (per_cta + rounds - 1) / rounds;
-  *smem_bytes = per_cta * 2 * kTileBytes;
+  *n_warps = w;
+  *smem_bytes = (per_cta < 2 * w ? per_cta : 2 * w) * 2 * kTileBytes;
 }
 
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream) {
@@ -434,7 +440,10 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = p.pdl_mode > 0 ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, decode_attn_kernel, p);
+  const int n_tiles = (p.L + 15) / 16;
+  const int per_cta = (n_tiles + n_clusters * cs - 1) / (n_clusters * cs);
+  return per_cta > 2 * n_warps ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true>, p)
+                               : cudaLaunchKernelEx(&cfg, decode_attn_kernel<false>, p);
 }
 
 }  // namespace sagekv
