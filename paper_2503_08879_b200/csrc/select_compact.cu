@@ -335,23 +335,52 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   int offset = 0;
   for (int r = 0; r < c.rank; ++r) offset += sh.sel_cnt[r];
 
-  // 5. output slots in ascending position
+  // 5. output slots in ascending position: offset + number of kept positions of this CTA below one's own.
   int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
-  int tps = 32;
-  while (tps > 1 && n_sel * tps > kSelThreads) tps >>= 1;
-  const int sub2 = tid & (tps - 1);
-  for (int c0 = 0; c0 < n_sel; c0 += kSelThreads / tps) {
-    const int ci = c0 + tid / tps;
-    const bool valid = ci < n_sel;
-    const int mine = valid ? sel_pos[ci] : 0;
-    int before = 0;
-    if (valid)
-      for (int i = sub2; i < n_sel; i += tps) before += sel_pos[i] < mine ? 1 : 0;
-    for (int off = 1; off < tps; off <<= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
-    if (valid && sub2 == 0) {
+  const int n_words = (c.n_local + 31) >> 5;
+  if (n_sel > 128 && (size_t)n_words * 4 <= (size_t)c.cand_cap * 8) {
+    // many kept rows in this CTA (clustered scores): a bitmap of the slice and a popcount prefix, O(n) instead
+    // of the pairwise count.  The candidate list is no longer needed (every CTA is past its ranking).
+    uint32_t *bm = reinterpret_cast<uint32_t *>(cand_all);
+    uint32_t *thread_base = sh.gmax;                     // free since step 2
+    for (int w = tid; w < n_words; w += kSelThreads) bm[w] = 0u;
+    __syncthreads();
+    for (int ci = tid; ci < n_sel; ci += kSelThreads) {
+      const int lp = sel_pos[ci] - c.lo;
+      atomicOr(&bm[lp >> 5], 1u << (lp & 31));
+    }
+    __syncthreads();
+    const int wpt = (n_words + kSelThreads - 1) / kSelThreads;   // words per thread
+    int mine_cnt = 0;
+    for (int w = tid * wpt; w < min(n_words, (tid + 1) * wpt); ++w) mine_cnt += __popc(bm[w]);
+    thread_base[tid] = (uint32_t)block_exclusive_scan(mine_cnt, sh.scan_tmp);
+    __syncthreads();
+    for (int ci = tid; ci < n_sel; ci += kSelThreads) {
+      const int pos = sel_pos[ci], lp = pos - c.lo, w0 = lp >> 5, t = w0 / wpt;
+      int before = (int)thread_base[t];
+      for (int w = t * wpt; w < w0; ++w) before += __popc(bm[w]);
+      before += __popc(bm[w0] & ((1u << (lp & 31)) - 1u));
       const int slot = offset + before;
-      idx_row[slot] = p.S + mine;
-      if (ci < c.list_cap) c.list[ci] = make_int2(slot, p.S + mine);
+      idx_row[slot] = p.S + pos;
+      if (ci < c.list_cap) c.list[ci] = make_int2(slot, p.S + pos);
+    }
+  } else {
+    int tps = 32;
+    while (tps > 1 && n_sel * tps > kSelThreads) tps >>= 1;
+    const int sub2 = tid & (tps - 1);
+    for (int c0 = 0; c0 < n_sel; c0 += kSelThreads / tps) {
+      const int ci = c0 + tid / tps;
+      const bool valid = ci < n_sel;
+      const int mine = valid ? sel_pos[ci] : 0;
+      int before = 0;
+      if (valid)
+        for (int i = sub2; i < n_sel; i += tps) before += sel_pos[i] < mine ? 1 : 0;
+      for (int off = 1; off < tps; off <<= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
+      if (valid && sub2 == 0) {
+        const int slot = offset + before;
+        idx_row[slot] = p.S + mine;
+        if (ci < c.list_cap) c.list[ci] = make_int2(slot, p.S + mine);
+      }
     }
   }
   if (tid == 0) sh.list_count = n_sel;

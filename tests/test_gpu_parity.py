@@ -141,6 +141,11 @@ def test_c1_full_config(B):
     ("C5-4096", dict(n_ctx=30000, budget=1024, n_recent_min=64), 3),
     # reduced cache longer than one partition pass: several tiles per CTA in decode
     ("C3-4096", dict(n_ctx=40000), 3),
+    # k_q too large for the prefilter (radix path at scale) and a reduced cache long enough for several
+    # clusters per KV head in decode (partition results merged through scratch)
+    ("C3-4096", dict(n_ctx=30000, budget=12600), 2),
+    # clustered heavy tokens with a large budget: hundreds of kept rows in one CTA of the select cluster
+    ("C5-8192", dict(n_ctx=60000, budget=4096, n_recent_min=64), 2),
 ])
 def test_scaled_configs(B, name, kw, n_decode):
     w = synth.workload(name).with_(n_layers=1, **kw)
