@@ -383,8 +383,14 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
       }
     }
   }
-  if (tid == 0) sh.list_count = n_sel;
+  // When the kept rows sit in few CTAs (clustered scores) the gather is re-dealt evenly: the positions are
+  // in idx by now, so after one more cluster barrier every CTA copies an equal range of slots.
+  int most = 0;
+  for (int r = 0; r < c.cs; ++r) most = max(most, sh.sel_cnt[r]);
+  const bool redeal = c.cs > 1 && most > 2 * (p.k_q / c.cs) + 64;   // same answer in every CTA
+  if (tid == 0) sh.list_count = redeal ? -1 : n_sel;
   __syncthreads();
+  if (redeal) cluster.sync();                            // every CTA's idx entries are written (and visible in the cluster)
   return true;
 }
 
@@ -550,7 +556,11 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
 
   // gather this CTA's kept rows into head j's segment of the reduced cache: a warp moves four rows at a
   // time (K in lanes 0-15, V in lanes 16-31), all loads issued before the stores
-  const int n_list = min(sh.list_count, list_cap);
+  const bool redeal = sh.list_count < 0;                 // take slots [rank, rank+1) * k_q / cs, positions from idx
+  const int per_cta = (p.k_q + cs - 1) / cs;
+  const int slot_lo = redeal ? min(p.k_q, rank * per_cta) : 0;
+  const int n_list = redeal ? min(p.k_q, slot_lo + per_cta) - slot_lo : min(sh.list_count, list_cap);
+  const int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
   const uint16_t *src_base = (lane < 16 ? p.K : p.V) + (int64_t)b * p.ks.batch_stride + (int64_t)kvh * p.ks.head_stride +
                              (lane & 15) * 8;
   uint16_t *dst_base = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
@@ -560,7 +570,8 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
     int slot[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int2 sp = c.list[min(e0 + u, n_list - 1)];
+      const int e = min(e0 + u, n_list - 1);
+      const int2 sp = redeal ? make_int2(slot_lo + e, __ldcg(idx_row + slot_lo + e)) : c.list[e];
       slot[u] = sp.x;
       v[u] = ld_stream_v4(src_base + (int64_t)sp.y * p.ks.token_stride);
     }
