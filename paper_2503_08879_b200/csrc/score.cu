@@ -130,14 +130,25 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_finalize_kernel(const 
   float *rowp = p.scores + (int64_t)row * p.row_stride;
   const int lo = blockIdx.x * per_slice;            // per_slice is a multiple of 4
   const int hi = min(p.E, lo + per_slice);
-  for (int i = lo + threadIdx.x * 4; i < hi; i += kFinalizeThreads * 4) {
-    if (i + 3 < hi) {
-      float4 v = *reinterpret_cast<float4 *>(rowp + i);
-      v.x = fast_exp2(v.x - m) * inv; v.y = fast_exp2(v.y - m) * inv;
-      v.z = fast_exp2(v.z - m) * inv; v.w = fast_exp2(v.w - m) * inv;
-      *reinterpret_cast<float4 *>(rowp + i) = v;
-    } else {
-      for (int e = i; e < hi; ++e) rowp[e] = fast_exp2(rowp[e] - m) * inv;
+  // eight 16-byte loads in flight per thread before the first store (the row is read and written in place,
+  // so the compiler would otherwise keep every load behind the previous store)
+  for (int i0 = lo + threadIdx.x * 4; i0 < hi; i0 += kFinalizeThreads * 4 * 8) {
+    float4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kFinalizeThreads * 4;
+      if (i + 3 < hi) v[u] = *reinterpret_cast<const float4 *>(rowp + i);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kFinalizeThreads * 4;
+      if (i + 3 < hi) {
+        v[u].x = fast_exp2(v[u].x - m) * inv; v[u].y = fast_exp2(v[u].y - m) * inv;
+        v[u].z = fast_exp2(v[u].z - m) * inv; v[u].w = fast_exp2(v[u].w - m) * inv;
+        *reinterpret_cast<float4 *>(rowp + i) = v[u];
+      } else if (i < hi) {
+        for (int e = i; e < hi; ++e) rowp[e] = fast_exp2(rowp[e] - m) * inv;
+      }
     }
   }
 }
