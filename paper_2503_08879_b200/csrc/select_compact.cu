@@ -9,17 +9,20 @@
 //   1. every thread takes the maximum of its elements; the cluster's thread maxima are exchanged over
 //      distributed shared memory.  The k_q-th largest of these maxima is a lower bound T0 of the k_q-th
 //      largest score (k_q distinct elements are >= it), and it is tight: about k_q * (1 + few %) scores
-//      are >= T0.  T0 is taken as the lower edge of the histogram bin (2048 bins laid over the actual
+//      are >= T0.  T0 is taken as the lower edge of the histogram bin (512 bins laid over the actual
 //      range of the maxima) in which that maximum falls.
-//   2. scores >= T0 become candidates (order-preserving key, position); the lists are exchanged.
-//   3. a histogram of all candidate keys finds the bin of the k_q-th largest; own candidates above it are
-//      kept, the few inside it are ranked exactly, with the position as tie-break (lowest positions win).
-//   4. kept counts are exchanged; slot = kept in lower CTAs + kept before it in this CTA: ascending order.
+//   2. scores >= T0 become candidates (order-preserving key, position), written in position order; every
+//      CTA takes a copy of all lists, CTA by CTA, so each holds the same position-sorted candidate list.
+//   3. every CTA decides for all candidates: a histogram of the candidate keys finds the bin of the k_q-th
+//      largest; candidates above it are kept, the few inside it are ranked exactly, with the position as
+//      tie-break (lowest positions win).
+//   4. a kept candidate's output slot is the number of kept candidates before it in the list (one prefix sum):
+//      ascending positions.  Each CTA writes and gathers an even share of the slots.
 // General path (k_q large, tiny rows, or more candidates than the buffers hold, e.g. a row of equal
 // scores): three-digit radix select (11 + 11 + 10 bits) with histograms merged in CTA 0's shared memory by
 // distributed-shared-memory atomics, then a ballot/popcount ranking in row order.
-// Either way the CTA that owns a kept element copies its K and V rows into the head's segment of the
-// reduced cache, and a few extra clusters copy the sink, recent and last rows.
+// The rows on a CTA's list are then copied into the head's segment of the reduced cache (general path: the
+// CTA that owns a kept element copies it), and a few extra clusters copy the sink, recent and last rows.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -32,7 +35,7 @@ constexpr int kSelThreads = 512;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kMaxCluster = 8;
 constexpr int kMaxBins = 2048;
-constexpr int kSelSmemLimit = 200 * 1024;
+constexpr int kSelSmemLimit = 227 * 1024;             // the most a CTA can have on this part
 constexpr int kGeneralScratch = 4 * kMaxBins * 4;   // general path: three merged histograms and the local one
 
 struct SelShared {
@@ -42,13 +45,12 @@ struct SelShared {
   uint32_t gstat[kMaxCluster][4];      // (min, max, count) of every CTA's non-empty thread maxima, pushed by the peers
   int totals[kMaxCluster][2];          // general path: (kept-larger, equal-to-threshold) per CTA; rank 0's copy
   int cand_cnt[kMaxCluster];           // fast path: candidates per CTA, pushed by each CTA to every peer
-  int sel_cnt[kMaxCluster];            // fast path: kept per CTA
+  int wsum[kSelWarps + 1];             // fast path: candidates per warp, then those among the slice's tail elements
   int warp_cnt[kSelWarps][2];
   int scan_tmp[kSelWarps];
   int found[2];
   int list_count;
-  int n_cand_local;
-  int n_sel_local;
+  int n_border;
   int pad_[3];
 };
 static_assert(sizeof(SelShared) % 16 == 0, "staged scores must stay 16-byte aligned");
@@ -145,14 +147,19 @@ struct SelCtx {
   int cand_cap;            // candidates per CTA and in total that the fast path can hold
 };
 
-// Eight float4 of this thread's elements (vector indices v0 + tid + u*512), all loads issued before any use.
-// Missing ones (index >= n_vec) read as -inf, which is below every threshold and never a maximum.
+// Which 16-byte vectors of the CTA's slice a thread works on: vector (it*8 + u)*512 + tid for iteration it and
+// u = 0..7, so that a run of neighbouring scores is spread over as many threads as it has vectors (the bound of
+// step 1 is only tight when large scores do not share a thread).  (it, u, tid, element) order is position order.
+__device__ __forceinline__ int n_iterations(int n_vec) { return (n_vec + 8 * kSelThreads - 1) / (8 * kSelThreads); }
+
+// The eight vectors of iteration `it` of this thread, all loads issued before any use.  Missing ones read as
+// -inf, which is below every threshold and never a maximum.
 template <bool kStaged>
-__device__ __forceinline__ void load8(const float *data, int v0, int n_vec, float4 (&x)[8]) {
+__device__ __forceinline__ void load8(const float *data, int n_vec, int it, float4 (&x)[8]) {
   const float ninf = -INFINITY;
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
-    const int v = v0 + (int)threadIdx.x + u * kSelThreads;
+    const int v = (it * 8 + u) * kSelThreads + (int)threadIdx.x;
     x[u] = make_float4(ninf, ninf, ninf, ninf);
     if (v < n_vec) {
       if (kStaged) {
@@ -166,30 +173,57 @@ __device__ __forceinline__ void load8(const float *data, int v0, int n_vec, floa
   }
 }
 
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory");
+}
+
 // ---- fast path ----------------------------------------------------------------------------------
 // Returns false (for every CTA of the cluster alike) when the prefilter cannot be used for this row;
 // nothing has been written to global memory in that case.
+// With kStaged the slice arrives through the four cp.async groups the kernel body has issued; every thread
+// reads only the vectors it copied itself, so it waits for its own groups and needs no barrier.
 template <bool kStaged>
 __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned long long *cand_local = reinterpret_cast<unsigned long long *>(c.scratch);
   unsigned long long *cand_all = cand_local + c.cand_cap;            // 16-byte aligned: cand_cap is even
-  int *sel_pos = reinterpret_cast<int *>(cand_all + c.cand_cap + 2);
+  unsigned char *flag = reinterpret_cast<unsigned char *>(cand_all + c.cand_cap + 2);
   const int n_vec = c.n_local >> 2;
+  const int n_it = n_iterations(n_vec);
+  const int tail_i = (n_vec << 2) + tid;                 // the slice's last (n_local % 4) elements: threads 0..2
+  const bool has_tail = tail_i < c.n_local;
 
   // 1. thread maxima (float order equals key order, so one fmaxf per element and one key per thread)
   uint32_t tmax = 0;   // 0 is below the key of every number: "no element"
   {
     float fm = -INFINITY;
-    for (int v0 = 0; v0 < n_vec; v0 += 8 * kSelThreads) {
-      float4 x[8];
-      load8<kStaged>(c.data, v0, n_vec, x);
+    if (kStaged) {
+      const int q = n_it * 2;                            // items (it, u) per copy group
 #pragma unroll
-      for (int u = 0; u < 8; ++u) fm = fmaxf(fmaxf(fm, x[u].x), fmaxf(x[u].y, fmaxf(x[u].z, x[u].w)));
+      for (int g = 0; g < 4; ++g) {
+        if (g == 0) cp_async_wait<3>();
+        if (g == 1) cp_async_wait<2>();
+        if (g == 2) cp_async_wait<1>();
+        if (g == 3) cp_async_wait<0>();
+        for (int k = g * q; k < (g + 1) * q; ++k) {
+          const int v = k * kSelThreads + tid;
+          if (v < n_vec) {
+            const float4 x = *reinterpret_cast<const float4 *>(c.data + 4 * v);
+            fm = fmaxf(fmaxf(fm, x.x), fmaxf(x.y, fmaxf(x.z, x.w)));
+          }
+        }
+      }
+    } else {
+      for (int it = 0; it < n_it; ++it) {
+        float4 x[8];
+        load8<false>(c.data, n_vec, it, x);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) fm = fmaxf(fmaxf(fm, x[u].x), fmaxf(x[u].y, fmaxf(x[u].z, x[u].w)));
+      }
     }
-    bool any = tid < n_vec;
-    for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) { fm = fmaxf(fm, c.data[i]); any = true; }
-    if (any) tmax = score_key(fm);
+    if (has_tail) fm = fmaxf(fm, c.data[tail_i]);
+    if (tid < n_vec || has_tail) tmax = score_key(fm);
   }
   sh.gmax[tid] = tmax;
   {
@@ -198,8 +232,9 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
     const uint32_t wcnt = __popc(__ballot_sync(0xffffffffu, tmax != 0u));
     if (lane == 0) { sh.red[0][warp] = wmin; sh.red[1][warp] = wmax; sh.red[2][warp] = wcnt; }
   }
-  if (tid == 0) { sh.n_cand_local = 0; sh.n_sel_local = 0; }
+  if (tid == 0) sh.n_border = 0;
   __syncthreads();
+  cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs
   if (warp == 0) {   // (min, max, count) of this CTA's maxima, pushed into every peer's gstat table
     uint32_t mn = lane < kSelWarps ? sh.red[0][lane] : 0xffffffffu;
     uint32_t mx = lane < kSelWarps ? sh.red[1][lane] : 0u;
@@ -239,37 +274,102 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   const float T0f = key_to_score(T0);
   sh.hist_fast[tid] = 0;                                 // reused in step 4 (barriers in between)
 
-  // 3. candidates: (key, position) packed so that a larger value precedes in (score desc, position asc)
-  for (int v0 = 0; v0 < n_vec; v0 += 8 * kSelThreads) {
+  // 3. candidates: scores >= T0 as (key, position), packed so that a larger value precedes in
+  //    (score desc, position asc), written in position order.  A thread's hits of one iteration are a 32-bit
+  //    mask (bit 4u + e: element e of its vector u); a row is the 512 vectors of one (it, u).  Pass A leaves the
+  //    hits of every (row, warp) in a byte table, pass B turns the table into offsets and writes.
+  auto hit_mask = [&](int it) {
     float4 x[8];
-    load8<kStaged>(c.data, v0, n_vec, x);
+    load8<kStaged>(c.data, n_vec, it, x);
+    uint32_t m = 0;
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      if (x[u].x >= T0f || x[u].y >= T0f || x[u].z >= T0f || x[u].w >= T0f) {
-        const float xs[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
-        const int v = v0 + tid + u * kSelThreads;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (xs[e] >= T0f) {
-            const int n = atomicAdd(&sh.n_cand_local, 1);
-            if (n < c.cand_cap)
-              cand_local[n] = ((unsigned long long)score_key(xs[e]) << 32) | (0xffffffffu - (uint32_t)(c.lo + 4 * v + e));
-          }
-        }
-      }
-    }
+    for (int u = 0; u < 8; ++u)
+      m |= ((x[u].x >= T0f ? 1u : 0u) | (x[u].y >= T0f ? 2u : 0u) | (x[u].z >= T0f ? 4u : 0u) | (x[u].w >= T0f ? 8u : 0u)) << (4 * u);
+    return m;
+  };
+  // hits per vector u (0..4) as bytes: u = 0..3 in lo, 4..7 in hi
+  auto nibble_counts = [](uint32_t m, uint32_t &lo, uint32_t &hi) {
+    uint32_t v = m - ((m >> 1) & 0x55555555u);
+    v = (v & 0x33333333u) + ((v >> 2) & 0x33333333u);                  // every nibble holds its bit count
+    lo = v & 0xffffu; hi = v >> 16;
+    lo = (lo | (lo << 8)) & 0x00ff00ffu; lo = (lo | (lo << 4)) & 0x0f0f0f0fu;
+    hi = (hi | (hi << 8)) & 0x00ff00ffu; hi = (hi | (hi << 4)) & 0x0f0f0f0fu;
+  };
+  unsigned char *table = reinterpret_cast<unsigned char *>(cand_all);   // [it][u][warp], free until the lists are exchanged
+  uint32_t mask = 0;                                     // of the last iteration (the only one when the slice is short)
+  for (int it = 0; it < n_it; ++it) {
+    mask = hit_mask(it);
+    uint32_t c_lo, c_hi;
+    nibble_counts(mask, c_lo, c_hi);
+    const uint32_t t_lo = __reduce_add_sync(0xffffffffu, c_lo), t_hi = __reduce_add_sync(0xffffffffu, c_hi);   // <= 128 per byte
+    if (lane < 8) table[(it * 8 + lane) * kSelWarps + warp] = (unsigned char)(((lane < 4 ? t_lo : t_hi) >> (8 * (lane & 3))) & 0xffu);
   }
-  for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) {
-    const float x = c.data[i];
-    if (x >= T0f) {
-      const int n = atomicAdd(&sh.n_cand_local, 1);
-      if (n < c.cand_cap)
-        cand_local[n] = ((unsigned long long)score_key(x) << 32) | (0xffffffffu - (uint32_t)(c.lo + i));
-    }
+  if (warp == 0) {                                       // the tail elements come last in position order
+    const uint32_t hits = __ballot_sync(0xffffffffu, has_tail && c.data[tail_i] >= T0f);
+    if (lane == 0) sh.wsum[0] = __popc(hits);
   }
   __syncthreads();
-  const int n_loc = sh.n_cand_local;
+  auto byte_sum = [](uint32_t w) { return (w & 0xffu) + ((w >> 8) & 0xffu) + ((w >> 16) & 0xffu) + (w >> 24); };
+  int n_loc = sh.wsum[0];
+  for (int it = 0; it < n_it; ++it)                      // lane l holds row l/4, warps 4*(l%4) .. +3 of the iteration's table
+    n_loc += (int)__reduce_add_sync(0xffffffffu, byte_sum(reinterpret_cast<const uint32_t *>(table)[it * 32 + lane]));
   if (tid < c.cs) cluster.map_shared_rank(sh.cand_cnt, tid)[c.rank] = n_loc;
+  if (n_loc <= c.cand_cap) {
+    int run_base = 0;                                    // hits of the iterations before this one
+    for (int it = 0; it < n_it; ++it) {
+      if (n_it > 1) mask = hit_mask(it);
+      const uint32_t word = reinterpret_cast<const uint32_t *>(table)[it * 32 + lane];
+      const uint32_t mine = byte_sum(word);
+      uint32_t inc = mine;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += n;
+      }
+      const int it_total = (int)__shfl_sync(0xffffffffu, inc, 31);
+      if (__any_sync(0xffffffffu, mask != 0u)) {
+        // hits before this warp's part of row u: in the rows before, and in the lower warps of the row
+        const uint32_t slot = inc - mine + byte_sum(word & ((1u << (8 * (warp & 3))) - 1u));
+        uint32_t rb[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) rb[u] = (uint32_t)run_base + __shfl_sync(0xffffffffu, slot, u * 4 + (warp >> 2));
+        // hits in the lower lanes of the warp, all eight rows at once (a row has at most 128 per warp: bytes suffice)
+        uint32_t c_lo, c_hi;
+        nibble_counts(mask, c_lo, c_hi);
+        uint32_t s_lo = c_lo, s_hi = c_hi;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const uint32_t t_lo = __shfl_up_sync(0xffffffffu, s_lo, off), t_hi = __shfl_up_sync(0xffffffffu, s_hi, off);
+          if (lane >= off) { s_lo += t_lo; s_hi += t_hi; }
+        }
+        const uint32_t x_lo = s_lo - c_lo, x_hi = s_hi - c_hi;          // per byte: no borrow, s >= c
+        // as 16-bit pairs (offsets stay below cand_cap < 65536 here)
+        const uint32_t b01 = (rb[0] | (rb[1] << 16)) + __byte_perm(x_lo, 0, 0x4140), b23 = (rb[2] | (rb[3] << 16)) + __byte_perm(x_lo, 0, 0x4342);
+        const uint32_t b45 = (rb[4] | (rb[5] << 16)) + __byte_perm(x_hi, 0, 0x4140), b67 = (rb[6] | (rb[7] << 16)) + __byte_perm(x_hi, 0, 0x4342);
+        const int elem0 = 4 * (it * 8 * kSelThreads + tid);             // slice index of element 0 of vector u = 0
+        uint32_t m = mask;
+        while (m) {
+          const int bit = __ffs(m) - 1;
+          m &= m - 1;
+          const int u = bit >> 2;
+          const uint32_t w = (u & 4) ? ((u & 2) ? b67 : b45) : ((u & 2) ? b23 : b01);
+          const int before = (int)((w >> ((u & 1) * 16)) & 0xffffu);
+          const int within = __popc(mask & ((1u << bit) - 1u) & (0xfu << (4 * u)));
+          const int i = elem0 + u * (4 * kSelThreads) + (bit & 3);
+          cand_local[before + within] =
+              ((unsigned long long)score_key(c.data[i]) << 32) | (0xffffffffu - (uint32_t)(c.lo + i));
+        }
+      }
+      run_base += it_total;
+    }
+    if (warp == 0) {
+      const bool hit = has_tail && c.data[tail_i] >= T0f;
+      const uint32_t hits = __ballot_sync(0xffffffffu, hit);
+      if (hit)
+        cand_local[n_loc - __popc(hits) + __popc(hits & ((1u << lane) - 1u))] =
+            ((unsigned long long)score_key(c.data[tail_i]) << 32) | (0xffffffffu - (uint32_t)(c.lo + tail_i));
+    }
+  }
   cluster.sync();
   int start[kMaxCluster + 1];
   bool overflow = false;
@@ -282,6 +382,7 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   }
   const int M = start[kMaxCluster];
   if (overflow || M > c.cand_cap) return false;         // same counts in every CTA: the whole cluster falls back
+  // every CTA takes a copy of all candidates, in CTA order: the list is sorted by position
   for (int i = tid; i < M; i += kSelThreads) {
     int r = 0;
 #pragma unroll
@@ -289,108 +390,70 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
     cand_all[i] = cluster.map_shared_rank(cand_local, r)[i - start[r]];
   }
   __syncthreads();
+  cluster.barrier_arrive();   // this CTA is done with its peers' shared memory; waited for before the kernel ends
 
-  // 4. which own candidates are kept.  A 512-bin histogram of ALL candidate keys over [T0, row maximum]
-  //    locates the bin b1 holding the k_q-th largest candidate: higher bins are kept, lower bins dropped,
-  //    and only the few candidates inside b1 are ranked exactly (key, then position) against their bin.
+  // 4. which candidates are kept (every CTA decides for all of them).  A 512-bin histogram of the candidate
+  //    keys over [T0, row maximum] locates the bin b1 holding the k_q-th largest: higher bins are kept, lower
+  //    bins dropped, and the few candidates inside b1 are ranked exactly (key, then position).
+  const uint32_t d2 = kmax ^ T0;
+  const int hb = d2 ? 31 - __clz(d2) : -1;
+  const int shift2 = hb > 8 ? hb - 8 : 0;
+  const uint32_t base2 = T0 >> shift2;
+  for (int i = tid; i < M; i += kSelThreads)
+    atomicAdd(&sh.hist_fast[(uint32_t)(cand_all[i] >> (32 + shift2)) - base2], 1u);
+  __syncthreads();
+  find_bin_from_top(sh.hist_fast, kSelThreads, p.k_q, sh);
+  const uint32_t b1 = (uint32_t)sh.found[0];
+  const int r1 = sh.found[1];                            // the k_q-th largest is the r1-th largest inside b1
+  uint32_t *border = sh.gmax;                            // free: every peer is past step 2
+  for (int i = tid; i < M; i += kSelThreads) {
+    const uint32_t bin = (uint32_t)(cand_all[i] >> (32 + shift2)) - base2;
+    flag[i] = bin > b1 ? 1 : 0;
+    if (bin == b1) {
+      const int n = atomicAdd(&sh.n_border, 1);
+      if (n < kSelThreads) border[n] = (uint32_t)i;
+    }
+  }
+  __syncthreads();
+  const int nb = sh.n_border;
+  if (nb > kSelThreads) {                                // a large group of near-equal scores at the cut
+    cluster.barrier_wait();
+    return false;
+  }
+  for (int j = warp; j < nb; j += kSelWarps) {           // one warp per candidate of the border bin
+    const uint32_t i = border[j];
+    const unsigned long long mine = cand_all[i];
+    int before = 0;
+    for (int jj = lane; jj < nb; jj += 32) before += cand_all[border[jj]] > mine ? 1 : 0;
+    before = __reduce_add_sync(0xffffffffu, before);
+    if (lane == 0) flag[i] = before < r1 ? 1 : 0;
+  }
+  __syncthreads();
+
+  // 5. output slots: the list is in position order, so a kept candidate's slot is the number of kept ones
+  //    before it.  The CTA writes and gathers an even share of the slots, wherever the rows come from.
   {
-    const uint32_t d2 = kmax ^ T0;
-    const int hb = d2 ? 31 - __clz(d2) : -1;
-    const int shift2 = hb > 8 ? hb - 8 : 0;
-    const uint32_t base2 = T0 >> shift2;
-    for (int i = tid; i < M; i += kSelThreads)
-      atomicAdd(&sh.hist_fast[(uint32_t)(cand_all[i] >> (32 + shift2)) - base2], 1u);
-    __syncthreads();
-    find_bin_from_top(sh.hist_fast, kSelThreads, p.k_q, sh);
-    const uint32_t b1 = (uint32_t)sh.found[0];
-    const int r1 = sh.found[1];                          // the k_q-th largest is the r1-th largest inside b1
-    for (int ci = tid; ci < n_loc; ci += kSelThreads) {  // the clear cases, one thread each
-      const unsigned long long mine = cand_local[ci];
-      if ((uint32_t)(mine >> (32 + shift2)) - base2 > b1) {
-        const int n = atomicAdd(&sh.n_sel_local, 1);
-        sel_pos[n] = (int)(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
-      }
-    }
-    for (int ci = warp; ci < n_loc; ci += kSelWarps) {   // the border cases, one warp each
-      const unsigned long long mine = cand_local[ci];
-      if ((uint32_t)(mine >> (32 + shift2)) - base2 == b1) {
-        int before = 0;
-        for (int i = lane; i < M; i += 32) {
-          const unsigned long long o = cand_all[i];
-          before += ((uint32_t)(o >> (32 + shift2)) - base2 == b1 && o > mine) ? 1 : 0;
-        }
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
-        if (lane == 0 && before < r1) {
-          const int n = atomicAdd(&sh.n_sel_local, 1);
-          sel_pos[n] = (int)(0xffffffffu - (uint32_t)(mine & 0xffffffffull));
-        }
-      }
-    }
-  }
-  __syncthreads();
-  const int n_sel = sh.n_sel_local;
-  if (tid < c.cs) cluster.map_shared_rank(sh.sel_cnt, tid)[c.rank] = n_sel;
-  cluster.sync();   // last access to a peer's shared memory
-  int offset = 0;
-  for (int r = 0; r < c.rank; ++r) offset += sh.sel_cnt[r];
-
-  // 5. output slots in ascending position: offset + number of kept positions of this CTA below one's own.
-  int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
-  const int n_words = (c.n_local + 31) >> 5;
-  if (n_sel > 128 && (size_t)n_words * 4 <= (size_t)c.cand_cap * 8) {
-    // many kept rows in this CTA (clustered scores): a bitmap of the slice and a popcount prefix, O(n) instead
-    // of the pairwise count.  The candidate list is no longer needed (every CTA is past its ranking).
-    uint32_t *bm = reinterpret_cast<uint32_t *>(cand_all);
-    uint32_t *thread_base = sh.gmax;                     // free since step 2
-    for (int w = tid; w < n_words; w += kSelThreads) bm[w] = 0u;
-    __syncthreads();
-    for (int ci = tid; ci < n_sel; ci += kSelThreads) {
-      const int lp = sel_pos[ci] - c.lo;
-      atomicOr(&bm[lp >> 5], 1u << (lp & 31));
-    }
-    __syncthreads();
-    const int wpt = (n_words + kSelThreads - 1) / kSelThreads;   // words per thread
+    const int per_cta = (p.k_q + c.cs - 1) / c.cs;
+    const int slot_lo = min(p.k_q, c.rank * per_cta), slot_hi = min(p.k_q, slot_lo + per_cta);
+    const int cpt = (M + kSelThreads - 1) / kSelThreads;   // candidates per thread, a contiguous run
+    const int i_lo = min(M, tid * cpt), i_hi = min(M, i_lo + cpt);
     int mine_cnt = 0;
-    for (int w = tid * wpt; w < min(n_words, (tid + 1) * wpt); ++w) mine_cnt += __popc(bm[w]);
-    thread_base[tid] = (uint32_t)block_exclusive_scan(mine_cnt, sh.scan_tmp);
-    __syncthreads();
-    for (int ci = tid; ci < n_sel; ci += kSelThreads) {
-      const int pos = sel_pos[ci], lp = pos - c.lo, w0 = lp >> 5, t = w0 / wpt;
-      int before = (int)thread_base[t];
-      for (int w = t * wpt; w < w0; ++w) before += __popc(bm[w]);
-      before += __popc(bm[w0] & ((1u << (lp & 31)) - 1u));
-      const int slot = offset + before;
-      idx_row[slot] = p.S + pos;
-      if (ci < c.list_cap) c.list[ci] = make_int2(slot, p.S + pos);
-    }
-  } else {
-    int tps = 32;
-    while (tps > 1 && n_sel * tps > kSelThreads) tps >>= 1;
-    const int sub2 = tid & (tps - 1);
-    for (int c0 = 0; c0 < n_sel; c0 += kSelThreads / tps) {
-      const int ci = c0 + tid / tps;
-      const bool valid = ci < n_sel;
-      const int mine = valid ? sel_pos[ci] : 0;
-      int before = 0;
-      if (valid)
-        for (int i = sub2; i < n_sel; i += tps) before += sel_pos[i] < mine ? 1 : 0;
-      for (int off = 1; off < tps; off <<= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
-      if (valid && sub2 == 0) {
-        const int slot = offset + before;
-        idx_row[slot] = p.S + mine;
-        if (ci < c.list_cap) c.list[ci] = make_int2(slot, p.S + mine);
+    for (int i = i_lo; i < i_hi; ++i) mine_cnt += flag[i];
+    int slot = block_exclusive_scan(mine_cnt, sh.scan_tmp);
+    int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
+    for (int i = i_lo; i < i_hi; ++i) {
+      if (flag[i]) {
+        if (slot >= slot_lo && slot < slot_hi) {
+          const int pos = p.S + (int)(0xffffffffu - (uint32_t)(cand_all[i] & 0xffffffffull));
+          idx_row[slot] = pos;
+          c.list[slot - slot_lo] = make_int2(slot, pos);
+        }
+        ++slot;
       }
     }
+    if (tid == 0) sh.list_count = slot_hi - slot_lo;
   }
-  // When the kept rows sit in few CTAs (clustered scores) the gather is re-dealt evenly: the positions are
-  // in idx by now, so after one more cluster barrier every CTA copies an equal range of slots.
-  int most = 0;
-  for (int r = 0; r < c.cs; ++r) most = max(most, sh.sel_cnt[r]);
-  const bool redeal = c.cs > 1 && most > 2 * (p.k_q / c.cs) + 64;   // same answer in every CTA
-  if (tid == 0) sh.list_count = redeal ? -1 : n_sel;
   __syncthreads();
-  if (redeal) cluster.sync();                            // every CTA's idx entries are written (and visible in the cluster)
   return true;
 }
 
@@ -401,6 +464,8 @@ __device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const 
   uint32_t *hist_local = reinterpret_cast<uint32_t *>(c.scratch) + 3 * kMaxBins;
   const float *data = c.data;
   const int n_local = c.n_local;
+  asm volatile("cp.async.wait_all;" ::: "memory");       // the staged slice: every thread reads all of it here
+  __syncthreads();
   for (int i = tid; i < kMaxBins; i += kSelThreads) {
     hist_local[i] = 0;
     hist_merged[0][i] = 0; hist_merged[1][i] = 0; hist_merged[2][i] = 0;
@@ -504,7 +569,7 @@ __device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const 
   cluster.sync();   // no CTA moves on (and may exit) while a peer still reads its shared memory
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const SelectParams p, int n_rows, int chunk,
+__global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const SelectParams p, int n_rows, int chunk,
                                                                       int resident, int list_cap, int cand_cap,
                                                                       int try_fast) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -525,9 +590,9 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
   c.cs = cs; c.rank = rank; c.row = cid; c.chunk = chunk;
   c.lo = rank * chunk;
   c.n_local = max(0, min(p.E - c.lo, chunk));
-  c.list = reinterpret_cast<int2 *>(after);
+  c.list = nullptr;           // placed by the path that runs
   c.list_cap = list_cap;
-  c.scratch = after + (((size_t)list_cap * sizeof(int2) + 15) & ~(size_t)15);   // 16-byte aligned
+  c.scratch = after;          // 16-byte aligned
   c.cand_cap = cand_cap;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -538,29 +603,40 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
   sh.hist_fast[tid] = 0;
   c.data = grow;
   if (resident) {
+    // four copy groups per thread, over exactly the vectors the thread works on later (see n_iterations)
     const int n_vec = c.n_local >> 2;
-    for (int v = tid; v < n_vec; v += kSelThreads) {
-      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(staged + 4 * v);
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(grow + 4 * v) : "memory");
+    const int q = n_iterations(n_vec) * 2;
+    for (int g = 0; g < 4; ++g) {
+      for (int k = g * q; k < (g + 1) * q; ++k) {
+        const int v = k * kSelThreads + tid;
+        if (v < n_vec) {
+          const uint32_t dst = (uint32_t)__cvta_generic_to_shared(staged + 4 * v);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(grow + 4 * v) : "memory");
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    for (int i = (n_vec << 2) + tid; i < c.n_local; i += kSelThreads) staged[i] = grow[i];
-    asm volatile("cp.async.wait_all;" ::: "memory");
+    const int tail_i = (n_vec << 2) + tid;
+    if (tail_i < c.n_local) staged[tail_i] = grow[tail_i];
     c.data = staged;
   }
-  __syncthreads();
-  cluster.barrier_wait();
 
+  // The gather list follows the buffers of the path that runs (see select_smem_bytes).
   bool done = false;
-  if (try_fast) done = resident ? fast_select<true>(cluster, sh, p, c) : fast_select<false>(cluster, sh, p, c);
-  if (!done) general_select(cluster, sh, p, c);
+  if (try_fast) {
+    c.list = reinterpret_cast<int2 *>(c.scratch + (size_t)cand_cap * 16 + 16 + (((size_t)cand_cap + 15) & ~(size_t)15));
+    done = resident ? fast_select<true>(cluster, sh, p, c) : fast_select<false>(cluster, sh, p, c);
+  } else {
+    cluster.barrier_wait();
+  }
+  if (!done) {
+    c.list = reinterpret_cast<int2 *>(c.scratch + kGeneralScratch);
+    general_select(cluster, sh, p, c);
+  }
 
-  // gather this CTA's kept rows into head j's segment of the reduced cache: a warp moves four rows at a
+  // gather the rows on this CTA's list into head j's segment of the reduced cache: a warp moves four rows at a
   // time (K in lanes 0-15, V in lanes 16-31), all loads issued before the stores
-  const bool redeal = sh.list_count < 0;                 // take slots [rank, rank+1) * k_q / cs, positions from idx
-  const int per_cta = (p.k_q + cs - 1) / cs;
-  const int slot_lo = redeal ? min(p.k_q, rank * per_cta) : 0;
-  const int n_list = redeal ? min(p.k_q, slot_lo + per_cta) - slot_lo : min(sh.list_count, list_cap);
-  const int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
+  const int n_list = min(sh.list_count, list_cap);
   const uint16_t *src_base = (lane < 16 ? p.K : p.V) + (int64_t)b * p.ks.batch_stride + (int64_t)kvh * p.ks.head_stride +
                              (lane & 15) * 8;
   uint16_t *dst_base = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
@@ -570,8 +646,7 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
     int slot[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int e = min(e0 + u, n_list - 1);
-      const int2 sp = redeal ? make_int2(slot_lo + e, __ldcg(idx_row + slot_lo + e)) : c.list[e];
+      const int2 sp = c.list[min(e0 + u, n_list - 1)];
       slot[u] = sp.x;
       v[u] = ld_stream_v4(src_base + (int64_t)sp.y * p.ks.token_stride);
     }
@@ -579,13 +654,17 @@ __global__ void __launch_bounds__(kSelThreads) select_compact_kernel(const Selec
     for (int u = 0; u < 4; ++u)
       if (e0 + u < n_list) st_v4(dst_base + (int64_t)slot[u] * p.cs.token_stride, v[u]);
   }
+  if (done) cluster.barrier_wait();   // fast path: a peer may still have been copying this CTA's candidates
 }
 
-static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, bool resident) {
-  size_t scratch = (size_t)cand_cap * (8 + 8) + 16 + (size_t)list_cap * 4;   // candidates (own, all) and kept positions
-  if (scratch < (size_t)kGeneralScratch) scratch = kGeneralScratch;
-  return sizeof(SelShared) + (((size_t)list_cap * sizeof(int2) + 15) & ~(size_t)15) + scratch +
-         (resident ? (size_t)chunk * sizeof(float) : 0);
+static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, int share, bool resident) {
+  // fast path: candidates (own, all), one keep flag per candidate, the gather list of the CTA's share of the slots;
+  // general path: the histograms, then the gather list (as long as the slice, or k_q)
+  size_t scratch = (size_t)cand_cap * (8 + 8) + 16 + (((size_t)cand_cap + 15) & ~(size_t)15) + (size_t)share * sizeof(int2);
+  const size_t general = (size_t)kGeneralScratch + (size_t)list_cap * sizeof(int2);
+  if (scratch < general) scratch = general;
+  scratch = (scratch + 15) & ~(size_t)15;
+  return sizeof(SelShared) + scratch + (resident ? (size_t)chunk * sizeof(float) : 0);
 }
 
 cudaError_t select_compact_setup() {
@@ -603,10 +682,12 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   if (chunk < 4) chunk = 4;
   const int list_cap = chunk < p.k_q ? chunk : (p.k_q > 0 ? p.k_q : 1);
   // the prefilter needs at least 2*k_q thread maxima; its buffers hold 1.5*k_q + 256 candidates
-  const int try_fast = select && 2 * (int64_t)p.k_q <= (int64_t)cs * kSelThreads;
+  // (and its per-row hit table, kept where the candidate copies go later, holds 16 iterations of 4096 vectors)
+  const int try_fast = select && 2 * (int64_t)p.k_q <= (int64_t)cs * kSelThreads && chunk <= 16 * 8 * kSelThreads * 4;
   const int cand_cap = try_fast ? (p.k_q + p.k_q / 2 + 256) & ~1 : 0;
-  const bool resident = select_smem_bytes(chunk, list_cap, cand_cap, true) <= (size_t)kSelSmemLimit;
-  const size_t smem = select_smem_bytes(chunk, list_cap, cand_cap, resident);
+  const int share = (p.k_q + cs - 1) / cs;              // slots a CTA writes and gathers on the fast path
+  const bool resident = select_smem_bytes(chunk, list_cap, cand_cap, share, true) <= (size_t)kSelSmemLimit;
+  const size_t smem = select_smem_bytes(chunk, list_cap, cand_cap, share, resident);
 
   const int static_items = p.B * p.H_kv * (p.S + p.R + 1);
   int copy_clusters = (static_items + cs * kSelWarps * 2 - 1) / (cs * kSelWarps * 2);

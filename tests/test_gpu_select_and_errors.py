@@ -78,17 +78,19 @@ def test_select_ties_lowest_position_wins(B):
         assert np.array_equal(idx, O.select(rows, k_q, 3))
 
 
-def test_select_tie_group_straddles_the_cut_in_the_prefilter_path(B):
+@pytest.mark.parametrize("k_q,winners,ties", [(300, 280, 40), (500, 300, 420), (600, 400, 700)])
+def test_select_tie_group_straddles_the_cut_in_the_prefilter_path(B, k_q, winners, ties):
     """Few enough equal scores that the prefilter path is taken, placed so that the k-th score lies inside
-    the group: exactly the lowest positions of the group must be kept."""
-    E, k_q = 60000, 300
+    the group: exactly the lowest positions of the group must be kept.  The three sizes end in the exact
+    ranking of a small group, of one that takes several rounds, and in the hand-over to the general path."""
+    E = 60000
     rng = np.random.default_rng(11)
     rows = (rng.random((4, E), dtype=np.float32) * 0.5).astype(np.float32)
     for h in range(4):
-        top = rng.choice(E, 280, replace=False)               # 280 clear winners
-        rows[h, top] = 0.9 + 0.05 * rng.random(280, dtype=np.float32)
+        top = rng.choice(E, winners, replace=False)           # clear winners
+        rows[h, top] = 0.9 + 0.05 * rng.random(winners, dtype=np.float32)
         rest = np.setdiff1d(np.arange(E), top)
-        tie = rng.choice(rest, 40, replace=False)             # 40 equal scores: 20 of them make the cut
+        tie = rng.choice(rest, ties, replace=False)           # equal scores: k_q - winners of them make the cut
         rows[h, tie] = 0.75
     idx = run_select(B, rows, k_q, H_kv=2)
     want = O.select(rows, k_q, 3)
@@ -96,7 +98,21 @@ def test_select_tie_group_straddles_the_cut_in_the_prefilter_path(B):
     for h in range(4):
         tie_pos = np.sort(np.nonzero(rows[h] == np.float32(0.75))[0]) + 3
         kept = np.intersect1d(idx[h], tie_pos)
-        assert np.array_equal(kept, tie_pos[:20])
+        assert np.array_equal(kept, tie_pos[:k_q - winners])
+
+
+def test_select_large_scores_in_contiguous_runs(B):
+    """Winners that sit next to each other (whole vectors and whole warps of hits) and a run that crosses the
+    border between two CTAs' slices: the candidate lists must still come out in position order."""
+    E, k_q = 60000, 500
+    rng = np.random.default_rng(12)
+    rows = (rng.random((4, E), dtype=np.float32) * 0.5).astype(np.float32)
+    slice_len = (E + 7) // 8
+    for h in range(4):
+        for start in (1234 + 97 * h, slice_len * 3 - 70, 41000 + h):
+            rows[h, start:start + 150] = 0.8 + 0.1 * rng.random(150, dtype=np.float32)
+        rows[h, rng.choice(E, 100, replace=False)] += 0.6
+    assert np.array_equal(run_select(B, rows, k_q, H_kv=2), O.select(rows, k_q, 3))
 
 
 def test_select_threshold_differs_only_in_low_bits(B):
