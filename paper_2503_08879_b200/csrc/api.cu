@@ -65,7 +65,7 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   ctx->max_chunks = (int)((max_ctx + kScoreChunk - 1) / kScoreChunk);
   {
     int cs, n_warps, smem;
-    decode_geometry(max_len, &ctx->max_splits, &cs, &n_warps, &smem);   // clusters per head at the largest L
+    decode_geometry(max_len, 0, &ctx->max_splits, &cs, &n_warps, &smem);   // clusters per head at the largest L
   }
   const size_t n_rows = (size_t)shape->batch * shape->n_q_heads;
   const size_t n_heads = (size_t)shape->batch * shape->n_kv_heads;

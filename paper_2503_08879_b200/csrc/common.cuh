@@ -70,7 +70,7 @@ struct DecodeParams {
 };
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream);
 cudaError_t decode_setup();           // one-time function attributes
-void decode_geometry(int L, int *n_clusters, int *cluster_size, int *n_warps, int *smem_bytes);
+void decode_geometry(int L, int heads, int *n_clusters, int *cluster_size, int *n_warps, int *smem_bytes);
 
 // ---- device helpers --------------------------------------------------------
 #if defined(__CUDACC__)

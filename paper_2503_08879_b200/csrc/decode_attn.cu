@@ -61,7 +61,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
 template <bool kPasses>
 __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char stage[];          // tiles: [K 4 KB | V 4 KB] each
-  __shared__ __align__(16) float inbox_o[kMaxGroup * kHeadDim];     // [source CTA][head][my columns], pushed by the peers
+  __shared__ __align__(16) float inbox_o[kMaxGroup * (kHeadDim + 16)];   // [source CTA][head][my columns], pushed by the peers; cluster size x columns <= 144
   __shared__ float2 inbox_ml[kDecodeMaxCluster * kMaxGroup];        // [source CTA][head] (max, sum)
   __shared__ float sm_m[kDecodeMaxWarps][kMaxGroup], sm_l[kDecodeMaxWarps][kMaxGroup];
   __shared__ int sm_last;
@@ -294,7 +294,7 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
 
   // ---- push this CTA's result to the peers: the owner of a column slice receives it from every CTA.
   // One thread sums four neighbouring columns of one head over the warps and sends them as one 16-byte store.
-  const int cols = kHeadDim / cs;                        // columns each CTA of the cluster finishes (a multiple of 4)
+  const int cols = ((kHeadDim + cs - 1) / cs + 3) & ~3;  // columns each CTA of the cluster finishes: a multiple of 4, the last CTA may get fewer
   // A warp's 32 items are 8 column groups (g) x 4 heads at one (piece, e): their exchange addresses g*8 + h
   // fall into 32 different banks.
   for (int item = tid; item < 8 * 32; item += blockDim.x) {
@@ -330,6 +330,7 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   float *part = p.partials + ((int64_t)bk * n_clusters + cl) * kResFloats;
   for (int item = tid; item < p.G * cols; item += blockDim.x) {
     const int h = item / cols, lc = item - h * cols, col = rank * cols + lc;
+    if (col >= kHeadDim) continue;
     float M = -INFINITY;
     for (int r = 0; r < cs; ++r) M = fmaxf(M, inbox_ml[r * kMaxGroup + h].x);
     float o = 0.f, l = 0.f;
@@ -394,38 +395,87 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   }
 }
 
+// How many clusters of each size can be resident at once when a CTA takes a whole SM (a cluster must fit into
+// one GPC, so this is not n_sm / size: on this part 15 clusters of 8 but 22 of 6).  Filled by decode_setup.
+static int g_cluster_cap[kDecodeMaxCluster + 1];
+
 // Clusters of 8 CTAs, the portable limit.  (16-CTA clusters were tried: too few of them are co-resident on
 // this part, so the grid ran in two waves.)
 cudaError_t decode_setup() {
   cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kDecodeMaxTiles * 2 * kTileBytes);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              kDecodeMaxTiles * 2 * kTileBytes);
+  e = cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kDecodeMaxTiles * 2 * kTileBytes);
+  if (e != cudaSuccess) return e;
+  for (int c = 4; c <= kDecodeMaxCluster; ++c) {
+    if (c == 7) continue;                                // never chosen (no more of them fit than of 8)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(c * 64), 1, 1);
+    cfg.blockDim = dim3(kDecodeMaxWarps * 32, 1, 1);
+    cfg.dynamicSmemBytes = kDecodeMaxTiles * 2 * kTileBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = c;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, decode_attn_kernel<false>, &cfg) != cudaSuccess) {
+      (void)cudaGetLastError();
+      n = 0;                                             // unknown: this size is then not considered
+    }
+    g_cluster_cap[c] = n;
+  }
+  return cudaSuccess;
+}
+
+// Warps and staging bytes of a CTA that gets per_cta tiles
+static void decode_cta_shape(int per_cta, int *n_warps, int *smem_bytes) {
+  int w = (per_cta + 1) / 2;                                                     // two tiles per warp and pass
+  if (per_cta > 2 * 9) w = kDecodeMaxTiles / 2;                                  // several passes: use every slot
+  else if (w > 9) w = 9;
+  if (w < 1) w = 1;
+  *n_warps = w;
+  *smem_bytes = (per_cta < 2 * w ? per_cta : 2 * w) * 2 * kTileBytes;
 }
 
 // Launch geometry for a reduced cache of L rows: one cluster per KV head whose CTAs go through their
 // tiles in passes of (two tiles per warp); more clusters per head only beyond kDecodeMaxPasses passes.
-void decode_geometry(int L, int *n_clusters, int *cs, int *n_warps, int *smem_bytes) {
+// heads = batch x KV heads of the launch (0: not known).  When a CTA needs a whole SM and the heads do not fit
+// at once as clusters of 8, smaller clusters are weighed: more of them are resident, each takes longer
+// (measured on this part at L = 2049 and 4097: about 4.5 us + 0.1 us per tile of a CTA + 1 us per extra pass).
+void decode_geometry(int L, int heads, int *n_clusters, int *cs, int *n_warps, int *smem_bytes) {
   const int n_tiles = (L + 15) / 16;
   int c = 1;
   while (c < kDecodeMaxCluster && c * 2 <= n_tiles) c <<= 1;                     // cluster size 1, 2, 4 or 8
   const int per_pass = kDecodeMaxTiles;                                          // tiles a CTA can stage at once
   const int nc = (n_tiles + c * per_pass * kDecodeMaxPasses - 1) / (c * per_pass * kDecodeMaxPasses);
-  const int per_cta = (n_tiles + c * nc - 1) / (c * nc);                         // most tiles a CTA gets
-  int w = (per_cta + 1) / 2;                                                     // two tiles per warp and pass
-  if (per_cta > 2 * 9) w = kDecodeMaxTiles / 2;                                  // several passes: use every slot
-  else if (w > 9) w = 9;
-  if (w < 1) w = 1;
+  int per_cta = (n_tiles + c * nc - 1) / (c * nc);                               // most tiles a CTA gets
+  decode_cta_shape(per_cta, n_warps, smem_bytes);
+  if (c == kDecodeMaxCluster && nc == 1 && *smem_bytes > 12 * 2 * kTileBytes && heads > g_cluster_cap[c] &&
+      g_cluster_cap[c] > 0) {
+    float best = 0.f;
+    int best_c = c;
+    for (int cand = kDecodeMaxCluster; cand >= 4; --cand) {
+      const int cap = g_cluster_cap[cand];
+      if (cap <= 0 || n_tiles > cand * per_pass * kDecodeMaxPasses) continue;
+      const int per = (n_tiles + cand - 1) / cand, passes = (per + per_pass - 1) / per_pass;
+      const float cost = (float)((heads + cap - 1) / cap) * (4.5f + 0.1f * (float)per + (float)(passes - 1));
+      if (cand == kDecodeMaxCluster || cost < best) { best = cost; best_c = cand; }
+    }
+    c = best_c;
+    per_cta = (n_tiles + c - 1) / c;
+    decode_cta_shape(per_cta, n_warps, smem_bytes);
+  }
   *n_clusters = nc;
   *cs = c;
-  *n_warps = w;
-  *smem_bytes = (per_cta < 2 * w ? per_cta : 2 * w) * 2 * kTileBytes;
 }
 
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream) {
   int n_clusters, cs, n_warps, smem;
-  decode_geometry(p.L, &n_clusters, &cs, &n_warps, &smem);
+  decode_geometry(p.L, p.B * p.H_kv, &n_clusters, &cs, &n_warps, &smem);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(n_clusters * cs), (unsigned)p.H_kv, (unsigned)p.B);
   cfg.blockDim = dim3((unsigned)(n_warps * 32), 1, 1);
