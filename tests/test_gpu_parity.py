@@ -146,6 +146,10 @@ def test_c1_full_config(B):
     ("C3-4096", dict(n_ctx=30000, budget=12600), 2),
     # clustered heavy tokens with a large budget: hundreds of kept rows in one CTA of the select cluster
     ("C5-8192", dict(n_ctx=60000, budget=4096, n_recent_min=64), 2),
+    # more (batch, KV head) pairs than clusters of 8 fit at once: decode runs with clusters of 6 (20 pairs) and
+    # of 5 (24 pairs), whose CTAs finish unequal shares of the 128 output columns
+    ("C4-b1", dict(n_ctx=6000, batch=5), 2),
+    ("C4-b1", dict(n_ctx=6000, batch=6), 2),
 ])
 def test_scaled_configs(B, name, kw, n_decode):
     w = synth.workload(name).with_(n_layers=1, **kw)
