@@ -22,7 +22,7 @@
 // scores): three-digit radix select (11 + 11 + 10 bits) with histograms merged in CTA 0's shared memory by
 // distributed-shared-memory atomics, then a ballot/popcount ranking in row order.
 // The rows on a CTA's list are then copied into the head's segment of the reduced cache (general path: the
-// CTA that owns a kept element copies it), and a few extra clusters copy the sink, recent and last rows.
+// CTA that owns a kept element copies it), together with a share of the KV head's sink, recent and last rows.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -641,19 +641,38 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
                              (lane & 15) * 8;
   uint16_t *dst_base = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
                        ((int64_t)p.S + (int64_t)j * p.k_q) * p.cs.token_stride + (lane & 15) * 8;
-  for (int e0 = warp * 4; e0 < n_list; e0 += kSelWarps * 4) {
-    uint4 v[4];
+  // The sink, recent and last rows of the KV head (positions known without the scores) are shared out over the
+  // warps of the head's G clusters, at most one row per warp per round, loaded together with the first batch.
+  const int n_static = p.S + p.R + 1;
+  const int static_stride = p.G * cs * kSelWarps;
+  int sr = (j * cs + rank) * kSelWarps + warp;           // this warp's first static row
+  for (int e0 = warp * 4; e0 < n_list || sr < n_static; e0 += kSelWarps * 4) {
+    uint4 v[4], vs = make_uint4(0u, 0u, 0u, 0u);
     int slot[4];
+    const bool has_static = sr < n_static;
+    if (has_static) {
+      const int64_t src_tok = sr < p.S ? sr : (int64_t)p.E + sr;                 // S + E + (sr - S)
+      vs = ld_stream_v4(src_base + src_tok * p.ks.token_stride);
+    }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int2 sp = c.list[min(e0 + u, n_list - 1)];
-      slot[u] = sp.x;
-      v[u] = ld_stream_v4(src_base + (int64_t)sp.y * p.ks.token_stride);
+      if (e0 < n_list) {
+        const int2 sp = c.list[min(e0 + u, n_list - 1)];
+        slot[u] = sp.x;
+        v[u] = ld_stream_v4(src_base + (int64_t)sp.y * p.ks.token_stride);
+      }
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
       if (e0 + u < n_list) st_v4(dst_base + (int64_t)slot[u] * p.cs.token_stride, v[u]);
+    if (has_static) {
+      // dst_base points at the head's segment S + j*k_q; static rows are addressed from row 0 of the KV head
+      const int64_t dst_row = sr < p.S ? sr : (int64_t)p.G * p.k_q + sr;         // S + G*k_q + (sr - S)
+      st_v4(dst_base + (dst_row - ((int64_t)p.S + (int64_t)j * p.k_q)) * p.cs.token_stride, vs);
+      sr += static_stride;
+    }
   }
+  if (cid == 0 && rank == 0 && tid == 0) *p.d_step = 0;
   if (done) cluster.barrier_wait();   // fast path: a peer may still have been copying this CTA's candidates
 }
 
@@ -689,11 +708,16 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   const bool resident = select_smem_bytes(chunk, list_cap, cand_cap, share, true) <= (size_t)kSelSmemLimit;
   const size_t smem = select_smem_bytes(chunk, list_cap, cand_cap, share, resident);
 
-  const int static_items = p.B * p.H_kv * (p.S + p.R + 1);
-  int copy_clusters = (static_items + cs * kSelWarps * 2 - 1) / (cs * kSelWarps * 2);
-  if (copy_clusters < 1) copy_clusters = 1;
-  const int cap = (n_sm + cs - 1) / cs;
-  if (copy_clusters > cap) copy_clusters = cap;
+  // Without a selection (k_q = 0 or an empty eviction region) there are no row clusters: plain copy clusters
+  // move the sink, recent and last rows.  Otherwise the row clusters copy them along with the kept rows.
+  int copy_clusters = 0;
+  if (!select) {
+    const int static_items = p.B * p.H_kv * (p.S + p.R + 1);
+    copy_clusters = (static_items + cs * kSelWarps * 2 - 1) / (cs * kSelWarps * 2);
+    if (copy_clusters < 1) copy_clusters = 1;
+    const int cap = (n_sm + cs - 1) / cs;
+    if (copy_clusters > cap) copy_clusters = cap;
+  }
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((n_rows + copy_clusters) * cs), 1, 1);
