@@ -390,7 +390,9 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
     cand_all[i] = cluster.map_shared_rank(cand_local, r)[i - start[r]];
   }
   __syncthreads();
-  cluster.barrier_arrive();   // this CTA is done with its peers' shared memory; waited for before the kernel ends
+  // This CTA is done with its peers' shared memory (the values it read are stored and past a barrier); the
+  // arrival is waited for before the kernel ends.  It orders no data, so it need not be a release.
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 
   // 4. which candidates are kept (every CTA decides for all of them).  A 512-bin histogram of the candidate
   //    keys over [T0, row maximum] locates the bin b1 holding the k_q-th largest: higher bins are kept, lower
