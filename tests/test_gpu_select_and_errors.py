@@ -115,6 +115,27 @@ def test_select_large_scores_in_contiguous_runs(B):
     assert np.array_equal(run_select(B, rows, k_q, H_kv=2), O.select(rows, k_q, 3))
 
 
+def test_cache_rows_read_from_pinned_host_memory(B):
+    """K and V may stay in pinned host memory (addressable from the device): the gather then pulls only the
+    kept rows over the bus.  Same indices and the same reduced cache as with device-resident K and V."""
+    E, k_q, S, R = 20000, 200, 4, 16
+    rows = np.random.default_rng(21).random((4, E), dtype=np.float32) ** 6
+    N = S + E + R + 1
+    g = torch.Generator(device="cuda").manual_seed(77)
+    K = torch.randn(1, 2, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    V = torch.randn(1, 2, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    scores = torch.from_numpy(rows).cuda()
+    sk = B.SageKV(4, 2, 128, 1, max_ctx=N, max_len=S + 2 * k_q + R + 1)
+    on_device = sk.select_compact(scores, K, V, S, R, 2 * k_q)
+    in_place = sk.select_compact(scores, K.cpu().pin_memory(), V.cpu().pin_memory(), S, R, 2 * k_q)
+    torch.cuda.synchronize()
+    assert torch.equal(on_device.indices(), in_place.indices())
+    assert np.array_equal(on_device.indices()[0].cpu().numpy(), O.select(rows, k_q, S))
+    for a, b in zip(on_device.cache(), in_place.cache()):
+        assert torch.equal(a, b)
+    sk.close()
+
+
 def test_select_threshold_differs_only_in_low_bits(B):
     E = 20000
     base = np.float32(0.001)
