@@ -97,19 +97,20 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
 
   // ---- issue the copies of this warp's first two tiles (its later tiles reuse the same two slots) ----
   const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(stage);
-  auto issue_tile = [&](int i) {   // i-th tile of this warp -> slot i & 1
+  auto issue_half = [&](int i, const uint16_t *src, uint32_t half) {   // K (half 0) or V (half 1) of this warp's i-th tile -> slot i & 1
     const int row0 = (first_tile + warp + i * n_warps) << 4;
-    const uint32_t tk = stage_base + (warp + (i & 1) * n_warps) * 2 * kTileBytes, tv = tk + kTileBytes;
+    const uint32_t dst = stage_base + (warp + (i & 1) * n_warps) * 2 * kTileBytes + half * kTileBytes;
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const int flat = u * 32 + lane, row = flat >> 4, piece = flat & 15;
       const int r = min(row0 + row, p.L - 1);
-      const uint32_t off = row * 256 + ((piece ^ swz(row)) << 4);
-      cp_async16(tk + off, Kh + (int64_t)r * p.cs.token_stride + piece * 8);
-      cp_async16(tv + off, Vh + (int64_t)r * p.cs.token_stride + piece * 8);
+      cp_async16(dst + row * 256 + ((piece ^ swz(row)) << 4), src + (int64_t)r * p.cs.token_stride + piece * 8);
     }
   };
-  for (int i = 0; i < min(n_mine, 2); ++i) issue_tile(i);
+  for (int i = 0; i < min(n_mine, 2); ++i) {
+    issue_half(i, Kh, 0u);
+    issue_half(i, Vh, 1u);
+  }
   asm volatile("cp.async.commit_group;" ::: "memory");
 
   if (p.pdl_mode >= 2) {
@@ -157,12 +158,15 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
   // when the partition is longer than the staging area, goes through its tiles in passes of two.
   for (int i0 = 0; i0 < (kPasses ? n_mine : min(n_mine, 2)); i0 += 2) {
     const int nt = min(2, n_mine - i0);                    // tiles of this pass
-    if (kPasses && i0 > 0) {                                          // the slots are free: this warp alone used them
-      __syncwarp();
-      for (int i = i0; i < i0 + nt; ++i) issue_tile(i);
-      asm volatile("cp.async.commit_group;" ::: "memory");
+    // Later passes refill the warp's own two slots, K and V as separate copy groups: K as soon as the pass before
+    // has taken its first product, V after its second.  Here the K rows are needed; the V group, committed
+    // after them, may still be on its way.
+    const bool more = kPasses && i0 + 2 < n_mine;          // a pass follows this one
+    if (kPasses && i0 > 0) {
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncwarp();
     uint32_t tk[2], tv[2];
     int base[2];
@@ -171,10 +175,10 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
       base[t] = (first_tile + warp + (i0 + (t < nt ? t : 0)) * n_warps) << 4;
       tk[t] = stage_base + (warp + (t < nt ? t : 0) * n_warps) * 2 * kTileBytes;
       tv[t] = tk[t] + kTileBytes;
-      if (t < nt && slot >= base[t] && slot < base[t] + 16) {   // the staged copy of the replaced row is stale: patch it
+      if (t < nt && slot >= base[t] && slot < base[t] + 16 && lane < 16) {   // the staged copy of the replaced row is stale: patch it (K here, V below)
         const int row = slot - base[t], piece = lane & 15;
-        const uint4 nv = ld_v4((lane < 16 ? kn : vn) + piece * 8);
-        const uint32_t dst = (lane < 16 ? tk[t] : tv[t]) + row * 256 + ((piece ^ swz(row)) << 4);
+        const uint4 nv = ld_v4(kn + piece * 8);
+        const uint32_t dst = tk[t] + row * 256 + ((piece ^ swz(row)) << 4);
         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(nv.x), "r"(nv.y), "r"(nv.z), "r"(nv.w) : "memory");
       }
     }
@@ -202,6 +206,11 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
           }
         }
       }
+    }
+    if (more) {                                            // the K rows are in registers' past: refill them for the next pass
+      __syncwarp();
+      for (int i = i0 + 2; i < min(n_mine, i0 + 4); ++i) issue_half(i, Kh, 0u);
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
     float tile_max = -INFINITY;
 #pragma unroll
@@ -237,6 +246,24 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
                (__uint_as_float(pb[t][1] << 16) + __uint_as_float(pb[t][1] & 0xffff0000u));
     }
     // ---- O^T += V^T P: rows 2c, 2c+1, 2c+8, 2c+9 at columns 8g..8g+7 and 64+8g..64+8g+7 ----
+    if (kPasses && i0 > 0) {                               // this pass's V group; the next pass's K group may stay pending
+      if (more) {
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+      } else {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+      }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      if (t < nt && slot >= base[t] && slot < base[t] + 16 && lane >= 16) {
+        const int row = slot - base[t], piece = lane & 15;
+        const uint4 nv = ld_v4(vn + piece * 8);
+        const uint32_t dst = tv[t] + row * 256 + ((piece ^ swz(row)) << 4);
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(nv.x), "r"(nv.y), "r"(nv.z), "r"(nv.w) : "memory");
+      }
+    }
+    __syncwarp();
     int vs[4];
     uint32_t voff[4];
 #pragma unroll
@@ -263,6 +290,11 @@ __global__ void __launch_bounds__(kDecodeMaxWarps * 32) decode_attn_kernel(const
           }
         }
       }
+    }
+    if (more) {
+      __syncwarp();
+      for (int i = i0 + 2; i < min(n_mine, i0 + 4); ++i) issue_half(i, Vh, 1u);
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
   }
 
