@@ -121,6 +121,10 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
  *           (Step 3: C = Concat(S, E_topk, R, P_N)).  Rows are bit-exact copies.
  *   state   host struct, filled on return; state->d_step must already point to
  *           a device int32, which is set to 0 on the stream.
+ *   K, V    bf16 [batch, H_kv, n_ctx, 128] through `ks`.  Only the kept, sink,
+ *           recent and last rows are read, so K and V may also be left in
+ *           pinned (device-addressable) host memory: the gather then moves
+ *           just those rows over the bus.
  * Scores are compared as IEEE numbers (-0 equals +0); they must not be NaN.
  * Errors: INVALID (null, k < 0, k % G != 0, bad partition), ALIGN,
  * UNSUPPORTED (L above the context's max_len), CUDA. */
