@@ -45,6 +45,9 @@ enum {
   SAGEKV_ERR_TOO_LARGE = -6    /* problem exceeds the fixed scratch of sagekv_score_static */
 };
 
+#define SAGEKV_SKETCH_ROOM 4100   /* floats behind a score row for sagekv_score's group maxima */
+#define SAGEKV_SKETCH_MIN_E 14337 /* shortest eviction region for which they are written          */
+
 typedef struct sagekv_ctx sagekv_ctx; /* opaque; owns only its scratch memory */
 
 typedef struct {
@@ -102,6 +105,14 @@ int sagekv_budget_split(int32_t B, int32_t G, int32_t *n_init, int32_t *k_q, int
  *   scores  fp32 [batch*H_q rows], row r at scores + r*scores_row_stride;
  *           scores_row_stride >= E and a multiple of 4, base 16-byte aligned.
  * bf16 products are accumulated in fp32.  E == 0 writes nothing.
+ * Optional hint for Step 2's second half (no counterpart in the paper; it
+ * changes no result): when E >= SAGEKV_SKETCH_MIN_E and scores_row_stride >=
+ * round_up(E,4) + SAGEKV_SKETCH_ROOM, the call also writes, behind the E scores
+ * of every row, the maxima of 4096 groups of that row's scores and two tag
+ * words; the buffer must then span all of batch*H_q * scores_row_stride
+ * floats.  sagekv_select_compact, given the same buffer and stride, starts from
+ * those maxima instead of computing them (it verifies the outcome, so scores
+ * changed in between still select correctly, only slower).
  * Errors: INVALID (null, n_init+n_recent+1 > n_ctx, stride < E), ALIGN,
  * UNSUPPORTED (n_ctx above the context's max_ctx), CUDA. */
 int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_strides ks,
@@ -125,6 +136,10 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
  *           recent and last rows are read, so K and V may also be left in
  *           pinned (device-addressable) host memory: the gather then moves
  *           just those rows over the bus.
+ *   scores  as written by sagekv_score.  With a row stride that leaves
+ *           SAGEKV_SKETCH_ROOM floats behind the scores (see sagekv_score) those
+ *           floats are read, whoever wrote the scores: the buffer must span
+ *           batch*H_q * scores_row_stride floats.
  * Scores are compared as IEEE numbers (-0 equals +0); they must not be NaN.
  * Errors: INVALID (null, k < 0, k % G != 0, bad partition), ALIGN,
  * UNSUPPORTED (L above the context's max_len), CUDA. */

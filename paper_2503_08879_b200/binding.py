@@ -24,6 +24,7 @@ lib = C.CDLL(_LIB_PATH)
 
 OK, ERR_INVALID, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
 ERR_TOO_LARGE = -6
+SKETCH_ROOM, SKETCH_MIN_E = 4100, 14337   # SAGEKV_SKETCH_ROOM, SAGEKV_SKETCH_MIN_E of include/sagekv.h
 
 
 class Shape(C.Structure):
@@ -183,7 +184,10 @@ class SageKV:
 
     @staticmethod
     def score_stride(E: int) -> int:
-        return max(4, (E + 3) // 4 * 4)
+        """Row stride of a score buffer: E rounded up to 4, plus, for rows long enough for it, the room in which
+        sagekv_score leaves the group maxima that speed up sagekv_select_compact (see include/sagekv.h)."""
+        stride = max(4, (E + 3) // 4 * 4)
+        return stride + SKETCH_ROOM if E >= SKETCH_MIN_E else stride
 
     def new_scores(self, E: int) -> torch.Tensor:
         Hq, _, _, B = self.shape

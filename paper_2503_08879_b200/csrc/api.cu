@@ -129,6 +129,7 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
   p.scores = scores;
   p.row_stride = scores_row_stride;
   p.partials = ctx->score_partials;
+  p.sketch = true;
   p.n_chunks = (int)((E + kScoreChunk - 1) / kScoreChunk);
   p.E = (int)E;
   p.S = n_init;

@@ -28,8 +28,27 @@ struct ScoreParams {
   int n_chunks;
   int E, S, G, H_q, H_kv, B;
   float scale_log2;        // softmax scale * log2(e)
+  bool sketch = false;     // leave the group maxima behind each row that has room for them
 };
 cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream);
+
+// ---- the group maxima the score step can leave behind each row for the select step ----------------------
+// A row of E scores is cut into 8 slices of sketch_chunk(E) elements (the select step's cluster CTAs) and each
+// slice into 512 groups (the CTA's threads: 16-byte vector v of the slice belongs to group v % 512, the last
+// E % 4 elements to groups 0..2).  If the row has room for it, the maximum of every group is stored at
+// [sketch_offset(E), +4096) of the row, followed by two tag words (a constant and E).  The select step reads
+// them only as a hint: any threshold that leaves at least k_q candidates is a valid one.
+constexpr int kSketchSlices = 8;
+constexpr int kSketchGroups = 512;
+constexpr int kSketchFloats = kSketchSlices * kSketchGroups;
+constexpr int kSketchRoom = kSketchFloats + 4;                 // with the tag, padded to 16 bytes
+constexpr uint32_t kSketchMagic = 0x53414745u;
+constexpr int kSketchMinE = 7 * 2048 + 1;                      // rows the select step gives to clusters of 8
+inline __host__ __device__ int64_t sketch_offset(int64_t E) { return (E + 3) & ~(int64_t)3; }
+inline __host__ __device__ int sketch_chunk(int64_t E) { return (int)((((E + kSketchSlices - 1) / kSketchSlices) + 3) & ~(int64_t)3); }
+inline __host__ __device__ bool sketch_fits(int64_t E, int64_t row_stride) {
+  return E >= kSketchMinE && row_stride >= sketch_offset(E) + kSketchRoom;
+}
 
 // ---- select + compact ------------------------------------------------------
 struct SelectParams {

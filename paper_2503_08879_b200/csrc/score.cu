@@ -153,6 +153,69 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_finalize_kernel(const 
   }
 }
 
+// The normalisation pass for rows that have room for the group maxima (see common.cuh): one CTA per slice of a
+// row, its threads on the vectors the select step's threads will work on, so a thread's running maximum of
+// what it stores is the group's maximum.
+constexpr int kSketchThreads = kSketchGroups;
+
+__global__ void __launch_bounds__(kSketchThreads) score_finalize_sketch_kernel(const ScoreParams p, int chunk) {
+  const int row = blockIdx.y, slice = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float m = -INFINITY, l = 0.f;
+  const float2 *part = p.partials + (int64_t)row * p.n_chunks;
+  for (int i = tid; i < p.n_chunks; i += kSketchThreads) {
+    const float2 v = part[i];
+    merge_ml(m, l, v.x, v.y);
+  }
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1)
+    merge_ml(m, l, __shfl_xor_sync(0xffffffffu, m, off), __shfl_xor_sync(0xffffffffu, l, off));
+  __shared__ float sm_m[kSketchThreads / 32], sm_l[kSketchThreads / 32];
+  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+  __syncthreads();
+  m = sm_m[0]; l = sm_l[0];
+#pragma unroll
+  for (int w = 1; w < kSketchThreads / 32; ++w) merge_ml(m, l, sm_m[w], sm_l[w]);
+  const float inv = 1.f / l;
+
+  float *rowp = p.scores + (int64_t)row * p.row_stride;
+  const int lo = slice * chunk;
+  const int n_local = max(0, min(p.E - lo, chunk));
+  const int n_vec = n_local >> 2;
+  float *base = rowp + lo;
+  float fm = -INFINITY;
+  for (int v0 = 0; v0 < n_vec; v0 += 8 * kSketchThreads) {
+    float4 x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int v = v0 + u * kSketchThreads + tid;
+      if (v < n_vec) x[u] = *reinterpret_cast<const float4 *>(base + 4 * v);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int v = v0 + u * kSketchThreads + tid;
+      if (v < n_vec) {
+        x[u].x = fast_exp2(x[u].x - m) * inv; x[u].y = fast_exp2(x[u].y - m) * inv;
+        x[u].z = fast_exp2(x[u].z - m) * inv; x[u].w = fast_exp2(x[u].w - m) * inv;
+        *reinterpret_cast<float4 *>(base + 4 * v) = x[u];
+        fm = fmaxf(fmaxf(fm, x[u].x), fmaxf(x[u].y, fmaxf(x[u].z, x[u].w)));
+      }
+    }
+  }
+  const int tail_i = (n_vec << 2) + tid;
+  if (tail_i < n_local) {
+    const float y = fast_exp2(base[tail_i] - m) * inv;
+    base[tail_i] = y;
+    fm = fmaxf(fm, y);
+  }
+  float *sketch = rowp + sketch_offset(p.E);
+  sketch[slice * kSketchGroups + tid] = fm;              // -inf: the group is empty
+  if (slice == 0 && tid == 0) {
+    sketch[kSketchFloats] = __uint_as_float(kSketchMagic);
+    sketch[kSketchFloats + 1] = __int_as_float(p.E);
+  }
+}
+
 cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream) {
   if (p.E <= 0) return cudaSuccess;
   dim3 grid(p.n_chunks, p.H_kv, p.B);
@@ -160,6 +223,10 @@ cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream) {
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
   const int rows = p.B * p.H_q;
+  if (p.sketch && sketch_fits(p.E, p.row_stride)) {
+    score_finalize_sketch_kernel<<<dim3(kSketchSlices, rows), kSketchThreads, 0, stream>>>(p, sketch_chunk(p.E));
+    return cudaGetLastError();
+  }
   int slices = (n_sm * 4 + rows - 1) / rows;
   const int max_slices = (p.E + 1023) / 1024;
   if (slices > max_slices) slices = max_slices;

@@ -183,8 +183,17 @@ __device__ __forceinline__ void cp_async_wait() {
 // nothing has been written to global memory in that case.
 // With kStaged the slice arrives through the four cp.async groups the kernel body has issued; every thread
 // reads only the vectors it copied itself, so it waits for its own groups and needs no barrier.
-template <bool kStaged>
-__device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c) {
+// kSketch: the group maxima of the whole row come from the sketch the score step left behind the row (gm_hint,
+// loaded by the caller before the staging copies): steps 1 and 2 need no pass over the data and no exchange.
+// The sketch is only a hint (the scores may have changed since): too few candidates send the row back here
+// without it.  entered: the cluster's entry barrier has been waited for already.
+// Returns kFastDone, kFastRetry / kFastRetryEntered (sketch variant: run the other variant; the entry barrier
+// has / has not been waited for yet) or kFastGeneral (take the general path).
+constexpr int kFastDone = 1, kFastRetry = 0, kFastRetryEntered = -1, kFastGeneral = -2;
+
+template <bool kStaged, bool kSketch>
+__device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c,
+                           const uint32_t (&gm_hint)[kMaxCluster], bool entered) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned long long *cand_local = reinterpret_cast<unsigned long long *>(c.scratch);
   unsigned long long *cand_all = cand_local + c.cand_cap;            // 16-byte aligned: cand_cap is even
@@ -194,6 +203,27 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   const int tail_i = (n_vec << 2) + tid;                 // the slice's last (n_local % 4) elements: threads 0..2
   const bool has_tail = tail_i < c.n_local;
 
+  uint32_t gm[kMaxCluster];
+  uint32_t kmin = 0xffffffffu, kmax = 0u, n_ne = 0u;
+  if (kSketch) {
+    // 1'. statistics of the row's 8 x 512 group maxima, which this thread holds 8 of
+    uint32_t tmin = 0xffffffffu, tmx = 0u, tcnt = 0u;
+#pragma unroll
+    for (int r = 0; r < kMaxCluster; ++r) {
+      gm[r] = gm_hint[r];
+      if (gm[r] != 0u) { tmin = min(tmin, gm[r]); tmx = max(tmx, gm[r]); ++tcnt; }
+    }
+    tmin = __reduce_min_sync(0xffffffffu, tmin);
+    tmx = __reduce_max_sync(0xffffffffu, tmx);
+    tcnt = __reduce_add_sync(0xffffffffu, tcnt);
+    if (lane == 0) { sh.red[0][warp] = tmin; sh.red[1][warp] = tmx; sh.red[2][warp] = tcnt; }
+    if (tid == 0) sh.n_border = 0;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) {
+      kmin = min(kmin, sh.red[0][w]); kmax = max(kmax, sh.red[1][w]); n_ne += sh.red[2][w];
+    }
+  } else {
   // 1. thread maxima (float order equals key order, so one fmaxf per element and one key per thread)
   uint32_t tmax = 0;   // 0 is below the key of every number: "no element"
   {
@@ -234,7 +264,7 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   }
   if (tid == 0) sh.n_border = 0;
   __syncthreads();
-  cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs
+  if (!entered) cluster.barrier_wait();                  // pairs with the arrive at kernel entry: every peer runs
   if (warp == 0) {   // (min, max, count) of this CTA's maxima, pushed into every peer's gstat table
     uint32_t mn = lane < kSelWarps ? sh.red[0][lane] : 0xffffffffu;
     uint32_t mx = lane < kSelWarps ? sh.red[1][lane] : 0u;
@@ -250,8 +280,6 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   cluster.sync();
 
   // 2. all maxima of the cluster -> T0 (512 bins laid over [kmin, kmax])
-  uint32_t gm[kMaxCluster];
-  uint32_t kmin = 0xffffffffu, kmax = 0u, n_ne = 0u;
 #pragma unroll
   for (int r = 0; r < kMaxCluster; ++r) {
     gm[r] = 0u;
@@ -260,7 +288,8 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
       kmin = min(kmin, sh.gstat[r][0]); kmax = max(kmax, sh.gstat[r][1]); n_ne += sh.gstat[r][2];
     }
   }
-  if ((int)n_ne < 2 * p.k_q) return false;              // too few groups for a tight bound (same answer in every CTA)
+  }
+  if ((int)n_ne < 2 * p.k_q) return kSketch ? kFastRetry : kFastGeneral;   // too few groups for a tight bound (same answer in every CTA)
   const uint32_t diff = kmax ^ kmin;
   const int hi = diff ? 31 - __clz(diff) : -1;           // highest bit in which the maxima differ
   const int shift = hi > 8 ? hi - 8 : 0;                 // (kmax >> shift) - (kmin >> shift) < 512
@@ -278,6 +307,7 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   //    (score desc, position asc), written in position order.  A thread's hits of one iteration are a 32-bit
   //    mask (bit 4u + e: element e of its vector u); a row is the 512 vectors of one (it, u).  Pass A leaves the
   //    hits of every (row, warp) in a byte table, pass B turns the table into offsets and writes.
+  if (kSketch && kStaged) cp_async_wait<0>();            // no pass over the slice so far: this thread's copies must have landed
   auto hit_mask = [&](int it) {
     float4 x[8];
     load8<kStaged>(c.data, n_vec, it, x);
@@ -313,6 +343,7 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   int n_loc = sh.wsum[0];
   for (int it = 0; it < n_it; ++it)                      // lane l holds row l/4, warps 4*(l%4) .. +3 of the iteration's table
     n_loc += (int)__reduce_add_sync(0xffffffffu, byte_sum(reinterpret_cast<const uint32_t *>(table)[it * 32 + lane]));
+  if (kSketch) cluster.barrier_wait();                   // pairs with the arrive at kernel entry: every peer runs
   if (tid < c.cs) cluster.map_shared_rank(sh.cand_cnt, tid)[c.rank] = n_loc;
   if (n_loc <= c.cand_cap) {
     int run_base = 0;                                    // hits of the iterations before this one
@@ -381,7 +412,9 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
     start[r + 1] = start[r] + n;
   }
   const int M = start[kMaxCluster];
-  if (overflow || M > c.cand_cap) return false;         // same counts in every CTA: the whole cluster falls back
+  // same counts in every CTA: the whole cluster takes the same way out
+  if (overflow || M > c.cand_cap) return kSketch ? kFastRetryEntered : kFastGeneral;
+  if (kSketch && M < p.k_q) return kFastRetryEntered;    // the sketch did not describe these scores
   // every CTA takes a copy of all candidates, in CTA order: the list is sorted by position
   for (int i = tid; i < M; i += kSelThreads) {
     int r = 0;
@@ -401,15 +434,16 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   const int hb = d2 ? 31 - __clz(d2) : -1;
   const int shift2 = hb > 8 ? hb - 8 : 0;
   const uint32_t base2 = T0 >> shift2;
+  // (a stale sketch may have understated the row maximum: keys above it share the top bin)
   for (int i = tid; i < M; i += kSelThreads)
-    atomicAdd(&sh.hist_fast[(uint32_t)(cand_all[i] >> (32 + shift2)) - base2], 1u);
+    atomicAdd(&sh.hist_fast[min((uint32_t)(cand_all[i] >> (32 + shift2)) - base2, (uint32_t)kSelThreads - 1u)], 1u);
   __syncthreads();
   find_bin_from_top(sh.hist_fast, kSelThreads, p.k_q, sh);
   const uint32_t b1 = (uint32_t)sh.found[0];
   const int r1 = sh.found[1];                            // the k_q-th largest is the r1-th largest inside b1
   uint32_t *border = sh.gmax;                            // free: every peer is past step 2
   for (int i = tid; i < M; i += kSelThreads) {
-    const uint32_t bin = (uint32_t)(cand_all[i] >> (32 + shift2)) - base2;
+    const uint32_t bin = min((uint32_t)(cand_all[i] >> (32 + shift2)) - base2, (uint32_t)kSelThreads - 1u);
     flag[i] = bin > b1 ? 1 : 0;
     if (bin == b1) {
       const int n = atomicAdd(&sh.n_border, 1);
@@ -420,7 +454,7 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
   const int nb = sh.n_border;
   if (nb > kSelThreads) {                                // a large group of near-equal scores at the cut
     cluster.barrier_wait();
-    return false;
+    return kFastGeneral;
   }
   for (int j = warp; j < nb; j += kSelWarps) {           // one warp per candidate of the border bin
     const uint32_t i = border[j];
@@ -456,7 +490,7 @@ __device__ bool fast_select(cg::cluster_group &cluster, SelShared &sh, const Sel
     if (tid == 0) sh.list_count = slot_hi - slot_lo;
   }
   __syncthreads();
-  return true;
+  return kFastDone;
 }
 
 // ---- general path -------------------------------------------------------------------------------
@@ -573,7 +607,7 @@ __device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const 
 
 __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const SelectParams p, int n_rows, int chunk,
                                                                       int resident, int list_cap, int cand_cap,
-                                                                      int try_fast) {
+                                                                      int try_fast, int64_t sketch_off) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   cg::cluster_group cluster = cg::this_cluster();
   const int cs = cluster.num_blocks();
@@ -604,6 +638,21 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
 
   sh.hist_fast[tid] = 0;
   c.data = grow;
+  // the row's group maxima, if the score step left them behind the row: requested ahead of the slice itself
+  uint32_t gm_hint[kMaxCluster], tag0 = 0u, tag1 = 0u;
+#pragma unroll
+  for (int r = 0; r < kMaxCluster; ++r) gm_hint[r] = 0u;
+  if (sketch_off >= 0) {
+    const float *sk = p.scores + (int64_t)c.row * p.row_stride + sketch_off;
+    float v[kSketchSlices];
+#pragma unroll
+    for (int r = 0; r < kSketchSlices; ++r)
+      asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v[r]) : "l"(sk + r * kSketchGroups + tid));
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(tag0) : "l"(sk + kSketchFloats));
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(tag1) : "l"(sk + kSketchFloats + 1));
+#pragma unroll
+    for (int r = 0; r < kSketchSlices; ++r) gm_hint[r] = v[r] == -INFINITY ? 0u : score_key(v[r]);
+  }
   if (resident) {
     // four copy groups per thread, over exactly the vectors the thread works on later (see n_iterations)
     const int n_vec = c.n_local >> 2;
@@ -627,7 +676,14 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   bool done = false;
   if (try_fast) {
     c.list = reinterpret_cast<int2 *>(c.scratch + (size_t)cand_cap * 16 + 16 + (((size_t)cand_cap + 15) & ~(size_t)15));
-    done = resident ? fast_select<true>(cluster, sh, p, c) : fast_select<false>(cluster, sh, p, c);
+    int code = kFastRetry;
+    if (sketch_off >= 0 && tag0 == kSketchMagic && tag1 == (uint32_t)p.E)   // the same words in every CTA of the row
+      code = resident ? fast_select<true, true>(cluster, sh, p, c, gm_hint, false)
+                      : fast_select<false, true>(cluster, sh, p, c, gm_hint, false);
+    if (code == kFastRetry || code == kFastRetryEntered)
+      code = resident ? fast_select<true, false>(cluster, sh, p, c, gm_hint, code == kFastRetryEntered)
+                      : fast_select<false, false>(cluster, sh, p, c, gm_hint, code == kFastRetryEntered);
+    done = code == kFastDone;
   } else {
     cluster.barrier_wait();
   }
@@ -733,8 +789,11 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  // the group maxima behind each row (see common.cuh), laid out for clusters of 8 over slices of this length
+  const int64_t sketch_off = try_fast && cs == kSketchSlices && sketch_fits(p.E, p.row_stride) &&
+                                     chunk == sketch_chunk(p.E) ? sketch_offset(p.E) : (int64_t)-1;
   return cudaLaunchKernelEx(&cfg, select_compact_kernel, p, n_rows, chunk, (int)resident, list_cap, cand_cap,
-                            try_fast);
+                            try_fast, sketch_off);
 }
 
 }  // namespace sagekv

@@ -136,6 +136,91 @@ def test_cache_rows_read_from_pinned_host_memory(B):
     sk.close()
 
 
+@pytest.mark.parametrize("sketch", ["true maxima", "far too high", "far too low", "garbage", "wrong tag"])
+def test_group_maxima_behind_the_rows_are_only_a_hint(B, sketch):
+    """The floats behind a long score row may hold the row's group maxima (written by sagekv_score): whatever
+    they hold, the selection is the oracle's.  Understated maxima give too many candidates, overstated ones too
+    few; both send the row through the path that computes the maxima itself."""
+    E, k_q, S, R = 60000, 300, 3, 5
+    rng = np.random.default_rng(31)
+    rows = (rng.random((4, E), dtype=np.float32) ** 6).astype(np.float32)
+    E4 = (E + 3) // 4 * 4
+    stride = E4 + B.SKETCH_ROOM
+    buf = torch.zeros(4, stride, dtype=torch.float32, device="cuda")
+    buf[:, :E] = torch.from_numpy(rows).cuda()
+    chunk = ((E + 7) // 8 + 3) // 4 * 4
+    sk_host = np.full((4, 8, 512), -np.inf, dtype=np.float32)
+    for h in range(4):
+        for r in range(8):
+            sl = rows[h, r * chunk:min(E, (r + 1) * chunk)]
+            n_vec = len(sl) // 4
+            v = sl[:n_vec * 4].reshape(n_vec, 4).max(axis=1)
+            for t in range(min(512, n_vec)):
+                sk_host[h, r, t] = v[t::512].max()
+            for t in range(len(sl) - n_vec * 4):
+                sk_host[h, r, t] = max(sk_host[h, r, t], sl[n_vec * 4 + t])
+    if sketch == "far too high":
+        sk_host[:] = 1e9
+    elif sketch == "far too low":
+        sk_host[:] = 1e-30
+    elif sketch == "garbage":
+        sk_host = rng.standard_normal(sk_host.shape).astype(np.float32) * 1e3
+        sk_host[0, 0, :7] = np.nan
+    buf[:, E4:E4 + 4096] = torch.from_numpy(sk_host.reshape(4, 4096)).cuda()
+    tag = np.array([0x53414745, E if sketch != "wrong tag" else E + 1], dtype=np.int32).view(np.float32)
+    buf[:, E4 + 4096:E4 + 4098] = torch.from_numpy(tag).cuda()
+    N = S + E + R + 1
+    g = torch.Generator(device="cuda").manual_seed(5)
+    K = torch.randn(1, 2, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    V = torch.randn(1, 2, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    sk = B.SageKV(4, 2, 128, 1, max_ctx=N, max_len=S + 2 * k_q + R + 1)
+    before = buf.clone()
+    layer = sk.select_compact(buf, K, V, S, R, 2 * k_q)
+    torch.cuda.synchronize()
+    assert torch.equal(before.view(torch.int32), buf.view(torch.int32))      # read-only, hint included
+    idx = layer.indices()[0].cpu().numpy()
+    assert np.array_equal(idx, O.select(rows, k_q, S))
+    Kc_ref, Vc_ref = O.compact(bits(K[0]), bits(V[0]), idx, S, R)
+    Kc, Vc = layer.cache()
+    assert np.array_equal(bits(Kc[0]), Kc_ref) and np.array_equal(bits(Vc[0]), Vc_ref)
+    sk.close()
+
+
+def test_score_leaves_the_group_maxima_when_the_rows_have_room(B):
+    """sagekv_score with the wider row stride: scores as without it, and behind each row the maxima of the
+    groups (vector v of slice r belongs to group v % 512) and the tag."""
+    Hq, Hkv, N, S, R = 4, 2, 20000, 4, 16
+    E = N - 1 - S - R
+    g = torch.Generator(device="cuda").manual_seed(9)
+    q = torch.randn(1, Hq, 128, generator=g, device="cuda").to(torch.bfloat16)
+    K = torch.randn(1, Hkv, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    sk = B.SageKV(Hq, Hkv, 128, 1, max_ctx=N, max_len=64)
+    E4 = (E + 3) // 4 * 4
+    narrow = torch.zeros(Hq, E4, dtype=torch.float32, device="cuda")
+    wide = torch.zeros(Hq, E4 + B.SKETCH_ROOM, dtype=torch.float32, device="cuda")
+    sk.score(q, K, S, R, scores=narrow)
+    sk.score(q, K, S, R, scores=wide)
+    torch.cuda.synchronize()
+    assert torch.equal(narrow[:, :E], wide[:, :E])
+    rows = wide[:, :E].cpu().numpy()
+    got = wide[:, E4:E4 + 4096].cpu().numpy().reshape(Hq, 8, 512)
+    chunk = ((E + 7) // 8 + 3) // 4 * 4
+    for h in range(Hq):
+        for r in range(8):
+            sl = rows[h, r * chunk:min(E, (r + 1) * chunk)]
+            n_vec = len(sl) // 4
+            want = np.full(512, -np.inf, dtype=np.float32)
+            v = sl[:n_vec * 4].reshape(n_vec, 4).max(axis=1)
+            for t in range(min(512, n_vec)):
+                want[t] = v[t::512].max()
+            for t in range(len(sl) - n_vec * 4):
+                want[t] = max(want[t], sl[n_vec * 4 + t])
+            assert np.array_equal(got[h, r], want)
+    tag = wide[:, E4 + 4096:E4 + 4098].cpu().numpy().view(np.int32)
+    assert (tag[:, 0] == 0x53414745).all() and (tag[:, 1] == E).all()
+    sk.close()
+
+
 def test_select_threshold_differs_only_in_low_bits(B):
     E = 20000
     base = np.float32(0.001)
