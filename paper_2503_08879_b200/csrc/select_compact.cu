@@ -751,19 +751,24 @@ cudaError_t select_compact_setup() {
 cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t stream) {
   const bool select = p.k_q > 0 && p.E > 0;
   const int n_rows = select ? p.B * p.H_q : 0;
+  // The rows may carry the group maxima of the score step (see common.cuh): then the threshold bound costs no
+  // pass over the data, the slice is read straight from global memory (no staging: it is needed once), and with
+  // many rows smaller clusters pay, because two CTAs per SM times the SM count is all that runs at once.
+  const bool sketch = select && sketch_fits(p.E, p.row_stride);
   // cluster size: slices of at least 2048 scores, at most 8 CTAs (the portable limit)
   int cs = 1;
-  while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E) cs <<= 1;
+  while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E && (!sketch || (int64_t)n_rows * cs * 2 <= 2 * (int64_t)n_sm)) cs <<= 1;
   int chunk = (p.E + cs - 1) / cs;
   chunk = (chunk + 3) & ~3;
   if (chunk < 4) chunk = 4;
   const int list_cap = chunk < p.k_q ? chunk : (p.k_q > 0 ? p.k_q : 1);
   // the prefilter needs at least 2*k_q thread maxima; its buffers hold 1.5*k_q + 256 candidates
   // (and its per-row hit table, kept where the candidate copies go later, holds 16 iterations of 4096 vectors)
-  const int try_fast = select && 2 * (int64_t)p.k_q <= (int64_t)cs * kSelThreads && chunk <= 16 * 8 * kSelThreads * 4;
+  const int try_fast = select && chunk <= 16 * 8 * kSelThreads * 4 &&
+                       (2 * (int64_t)p.k_q <= (int64_t)cs * kSelThreads || (sketch && 2 * p.k_q <= kSketchFloats));
   const int cand_cap = try_fast ? (p.k_q + p.k_q / 2 + 256) & ~1 : 0;
   const int share = (p.k_q + cs - 1) / cs;              // slots a CTA writes and gathers on the fast path
-  const bool resident = select_smem_bytes(chunk, list_cap, cand_cap, share, true) <= (size_t)kSelSmemLimit;
+  const bool resident = !sketch && select_smem_bytes(chunk, list_cap, cand_cap, share, true) <= (size_t)kSelSmemLimit;
   const size_t smem = select_smem_bytes(chunk, list_cap, cand_cap, share, resident);
 
   // Without a selection (k_q = 0 or an empty eviction region) there are no row clusters: plain copy clusters
@@ -789,9 +794,7 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  // the group maxima behind each row (see common.cuh), laid out for clusters of 8 over slices of this length
-  const int64_t sketch_off = try_fast && cs == kSketchSlices && sketch_fits(p.E, p.row_stride) &&
-                                     chunk == sketch_chunk(p.E) ? sketch_offset(p.E) : (int64_t)-1;
+  const int64_t sketch_off = try_fast && sketch ? sketch_offset(p.E) : (int64_t)-1;
   return cudaLaunchKernelEx(&cfg, select_compact_kernel, p, n_rows, chunk, (int)resident, list_cap, cand_cap,
                             try_fast, sketch_off);
 }

@@ -150,6 +150,10 @@ def test_c1_full_config(B):
     # of 5 (24 pairs), whose CTAs finish unequal shares of the 128 output columns
     ("C4-b1", dict(n_ctx=6000, batch=5), 2),
     ("C4-b1", dict(n_ctx=6000, batch=6), 2),
+    # many score rows (112) that carry the score step's group maxima: select runs with clusters of 2, unstaged
+    ("C4-b1", dict(n_ctx=20000, batch=4), 1),
+    # and 56 rows: clusters of 4
+    ("C4-b1", dict(n_ctx=20000, batch=2), 1),
 ])
 def test_scaled_configs(B, name, kw, n_decode):
     w = synth.workload(name).with_(n_layers=1, **kw)
