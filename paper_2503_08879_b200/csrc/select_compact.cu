@@ -653,6 +653,10 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
 #pragma unroll
     for (int r = 0; r < kSketchSlices; ++r) gm_hint[r] = v[r] == -INFINITY ? 0u : score_key(v[r]);
   }
+  if (!resident && sketch_off >= 0 && tid == 0 && c.n_local >= 4) {
+    // not staged: ask for the slice to be brought into L2 while the threshold bound is worked out from the hint
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(grow), "r"((uint32_t)(c.n_local >> 2) * 16u) : "memory");
+  }
   if (resident) {
     // four copy groups per thread, over exactly the vectors the thread works on later (see n_iterations)
     const int n_vec = c.n_local >> 2;
