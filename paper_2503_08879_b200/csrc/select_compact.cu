@@ -3,11 +3,14 @@
 //
 // One thread-block cluster (up to 8 CTAs) owns one score row.  Each CTA stages its contiguous slice of
 // the row in shared memory once (cp.async, 16 bytes per request); every later step works on that copy, so
-// the scores cross the memory system a single time.
+// the scores cross the memory system a single time.  When the row carries the group maxima of the score
+// step (see common.cuh) the slice is needed only once: it is not staged but requested into L2 with one bulk
+// prefetch and read from there, and the cluster shrinks when there are more rows than cluster slots.
 //
 // Fast path (k_q small against the row, the normal case): a prefilter instead of a full radix select.
 //   1. every thread takes the maximum of its elements; the cluster's thread maxima are exchanged over
-//      distributed shared memory.  The k_q-th largest of these maxima is a lower bound T0 of the k_q-th
+//      distributed shared memory (or all of the row's group maxima are read from behind the row: a hint that
+//      is checked by its outcome, see fast_select).  The k_q-th largest of these maxima is a lower bound T0 of the k_q-th
 //      largest score (k_q distinct elements are >= it), and it is tight: about k_q * (1 + few %) scores
 //      are >= T0.  T0 is taken as the lower edge of the histogram bin (512 bins laid over the actual
 //      range of the maxima) in which that maximum falls.
