@@ -108,11 +108,13 @@ int sagekv_budget_split(int32_t B, int32_t G, int32_t *n_init, int32_t *k_q, int
  * Optional hint for Step 2's second half (no counterpart in the paper; it
  * changes no result): when E >= SAGEKV_SKETCH_MIN_E and scores_row_stride >=
  * round_up(E,4) + SAGEKV_SKETCH_ROOM, the call also writes, behind the E scores
- * of every row, the maxima of 4096 groups of that row's scores and two tag
- * words; the buffer must then span all of batch*H_q * scores_row_stride
- * floats.  sagekv_select_compact, given the same buffer and stride, starts from
- * those maxima instead of computing them (it verifies the outcome, so scores
- * changed in between still select correctly, only slower).
+ * of every row, a 512-bin histogram of the maxima of 4096 groups of that row's
+ * scores and four tag words (516 32-bit words; the rest of the room is left
+ * alone); the buffer must then span all of batch*H_q * scores_row_stride
+ * floats.  sagekv_select_compact, given the same buffer and stride, takes its
+ * first threshold bound from that histogram instead of a pass over the scores
+ * (it verifies the outcome, so scores changed in between still select
+ * correctly, only slower).
  * Errors: INVALID (null, n_init+n_recent+1 > n_ctx, stride < E), ALIGN,
  * UNSUPPORTED (n_ctx above the context's max_ctx), CUDA. */
 int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_strides ks,

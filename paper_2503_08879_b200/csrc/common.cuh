@@ -28,22 +28,28 @@ struct ScoreParams {
   int n_chunks;
   int E, S, G, H_q, H_kv, B;
   float scale_log2;        // softmax scale * log2(e)
-  bool sketch = false;     // leave the group maxima behind each row that has room for them
+  bool sketch = false;     // leave the histogram of the group maxima behind each row that has room for it
+  int64_t sketch_off = -1; // set by launch_score: where in a row it goes, or -1
 };
 cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream);
 
-// ---- the group maxima the score step can leave behind each row for the select step ----------------------
-// A row of E scores is cut into 8 slices of sketch_chunk(E) elements (the select step's cluster CTAs) and each
-// slice into 512 groups (the CTA's threads: 16-byte vector v of the slice belongs to group v % 512, the last
-// E % 4 elements to groups 0..2).  If the row has room for it, the maximum of every group is stored at
-// [sketch_offset(E), +4096) of the row, followed by two tag words (a constant and E).  The select step reads
-// them only as a hint: any threshold that leaves at least k_q candidates is a valid one.
+// ---- what the score step can leave behind each row for the select step -----------------------------------
+// A row of E scores is cut into 8 slices of sketch_chunk(E) elements and each slice into 512 groups (16-byte
+// vector v of the slice belongs to group v % 512, the last E % 4 elements to groups 0..2).  If the row has room
+// for it, a histogram of the 4096 group maxima is stored at [sketch_offset(E), +512) of the row as 32-bit counts:
+// 16 bins per octave, the top bin holding the row maximum, 32 octaves in all, lower maxima in bin 0.  Four
+// words follow: a constant, E, the key of bin 0's lower edge >> kSketchShift, the key of the row maximum.  The
+// k-th largest group maximum is a lower bound of the k-th largest score, so the select step finds its
+// threshold bound by a scan of 512 counts.  It takes them only as a hint: any threshold that leaves at least
+// k_q candidates is a valid one, and it checks.
 constexpr int kSketchSlices = 8;
 constexpr int kSketchGroups = 512;
-constexpr int kSketchFloats = kSketchSlices * kSketchGroups;
-constexpr int kSketchRoom = kSketchFloats + 4;                 // with the tag, padded to 16 bytes
+constexpr int kSketchBins = 512;
+constexpr int kSketchShift = 19;                               // key bits below a bin: 2^23 keys per octave / 16
+constexpr int kSketchFloats = kSketchSlices * kSketchGroups;   // groups per row
+constexpr int kSketchRoom = 4100;                              // floats reserved behind a row (SAGEKV_SKETCH_ROOM)
 constexpr uint32_t kSketchMagic = 0x53414745u;
-constexpr int kSketchMinE = 7 * 2048 + 1;                      // rows the select step gives to clusters of 8
+constexpr int kSketchMinE = 7 * 2048 + 1;                      // rows long enough for clusters of 8 in the select step
 inline __host__ __device__ int64_t sketch_offset(int64_t E) { return (E + 3) & ~(int64_t)3; }
 inline __host__ __device__ int sketch_chunk(int64_t E) { return (int)((((E + kSketchSlices - 1) / kSketchSlices) + 3) & ~(int64_t)3); }
 inline __host__ __device__ bool sketch_fits(int64_t E, int64_t row_stride) {
@@ -137,6 +143,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
+}
+
+// order-preserving 32-bit key of a score: larger float <=> larger unsigned key; -0 and +0 share a key
+__device__ __forceinline__ uint32_t score_key(float x) {
+  const uint32_t u = __float_as_uint(x + 0.0f);         // -0 becomes +0: the two compare equal as numbers
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
 // merge two (max, sum) pairs of a running softmax kept in log2 units

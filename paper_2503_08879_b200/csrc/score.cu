@@ -17,6 +17,12 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_logits_kernel(const Sc
   const int chunk = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, c = lane & 3;
+  if (chunk == 0 && p.sketch_off >= 0) {   // the rows' histograms are filled by atomic adds in the second pass
+    for (int i = threadIdx.x; i < p.G * (kSketchBins + 4); i += kScoreWarps * 32) {
+      const int h = i / (kSketchBins + 4);
+      reinterpret_cast<uint32_t *>(p.scores + ((int64_t)b * p.H_q + kvh * p.G + h) * p.row_stride + p.sketch_off)[i - h * (kSketchBins + 4)] = 0u;
+    }
+  }
 
   // B fragments: query head (kvh*G + g) for n = g, zero padding for n >= G
   uint4 qf[4];
@@ -153,9 +159,9 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_finalize_kernel(const 
   }
 }
 
-// The normalisation pass for rows that have room for the group maxima (see common.cuh): one CTA per slice of a
-// row, its threads on the vectors the select step's threads will work on, so a thread's running maximum of
-// what it stores is the group's maximum.
+// The normalisation pass for rows that have room for the histogram of the group maxima (see common.cuh): one
+// CTA per slice of a row, a thread per group, so a thread's running maximum of what it stores is the group's
+// maximum.  The row maximum is exp2(0) / l exactly, so every CTA of the row lays the same bins.
 constexpr int kSketchThreads = kSketchGroups;
 
 __global__ void __launch_bounds__(kSketchThreads) score_finalize_sketch_kernel(const ScoreParams p, int chunk) {
@@ -208,22 +214,36 @@ __global__ void __launch_bounds__(kSketchThreads) score_finalize_sketch_kernel(c
     base[tail_i] = y;
     fm = fmaxf(fm, y);
   }
-  float *sketch = rowp + sketch_offset(p.E);
-  sketch[slice * kSketchGroups + tid] = fm;              // -inf: the group is empty
+  __shared__ uint32_t sm_hist[kSketchBins];
+  sm_hist[tid] = 0u;
+  __syncthreads();
+  const uint32_t kmax = score_key(inv);
+  const uint32_t bin0 = (kmax >> kSketchShift) - (uint32_t)(kSketchBins - 1);
+  if (tid < n_vec || tail_i < n_local) {                  // the group is not empty
+    const uint32_t q = score_key(fm) >> kSketchShift;
+    atomicAdd(&sm_hist[q > bin0 ? min(q - bin0, (uint32_t)kSketchBins - 1u) : 0u], 1u);
+  }
+  __syncthreads();
+  uint32_t *sketch = reinterpret_cast<uint32_t *>(rowp + p.sketch_off);
+  if (sm_hist[tid] != 0u) atomicAdd(&sketch[tid], sm_hist[tid]);
   if (slice == 0 && tid == 0) {
-    sketch[kSketchFloats] = __uint_as_float(kSketchMagic);
-    sketch[kSketchFloats + 1] = __int_as_float(p.E);
+    sketch[kSketchBins] = kSketchMagic;
+    sketch[kSketchBins + 1] = (uint32_t)p.E;
+    sketch[kSketchBins + 2] = bin0;
+    sketch[kSketchBins + 3] = kmax;
   }
 }
 
-cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream) {
-  if (p.E <= 0) return cudaSuccess;
+cudaError_t launch_score(const ScoreParams &p_in, int n_sm, cudaStream_t stream) {
+  if (p_in.E <= 0) return cudaSuccess;
+  ScoreParams p = p_in;
+  p.sketch_off = p.sketch && sketch_fits(p.E, p.row_stride) ? sketch_offset(p.E) : (int64_t)-1;
   dim3 grid(p.n_chunks, p.H_kv, p.B);
   score_logits_kernel<<<grid, kScoreWarps * 32, 0, stream>>>(p);
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
   const int rows = p.B * p.H_q;
-  if (p.sketch && sketch_fits(p.E, p.row_stride)) {
+  if (p.sketch_off >= 0) {
     score_finalize_sketch_kernel<<<dim3(kSketchSlices, rows), kSketchThreads, 0, stream>>>(p, sketch_chunk(p.E));
     return cudaGetLastError();
   }

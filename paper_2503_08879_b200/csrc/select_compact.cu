@@ -58,11 +58,6 @@ struct SelShared {
 };
 static_assert(sizeof(SelShared) % 16 == 0, "staged scores must stay 16-byte aligned");
 
-__device__ __forceinline__ uint32_t score_key(float x) {
-  const uint32_t u = __float_as_uint(x + 0.0f);         // -0 becomes +0: the two compare equal as numbers
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);   // larger float <=> larger unsigned key
-}
-
 __device__ __forceinline__ float key_to_score(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
@@ -186,17 +181,24 @@ __device__ __forceinline__ void cp_async_wait() {
 // nothing has been written to global memory in that case.
 // With kStaged the slice arrives through the four cp.async groups the kernel body has issued; every thread
 // reads only the vectors it copied itself, so it waits for its own groups and needs no barrier.
-// kSketch: the group maxima of the whole row come from the sketch the score step left behind the row (gm_hint,
-// loaded by the caller before the staging copies): steps 1 and 2 need no pass over the data and no exchange.
-// The sketch is only a hint (the scores may have changed since): too few candidates send the row back here
-// without it.  entered: the cluster's entry barrier has been waited for already.
+// kSketch: the bound comes from the histogram of the row's group maxima that the score step left behind the
+// row (hint, loaded by the caller ahead of everything else): steps 1 and 2 are a scan of 512 counts, with no
+// pass over the data and no exchange.  It is only a hint (the scores may have changed since): too few or too
+// many candidates send the row back here without it.  entered: the cluster's entry barrier has been waited
+// for already.
 // Returns kFastDone, kFastRetry / kFastRetryEntered (sketch variant: run the other variant; the entry barrier
 // has / has not been waited for yet) or kFastGeneral (take the general path).
 constexpr int kFastDone = 1, kFastRetry = 0, kFastRetryEntered = -1, kFastGeneral = -2;
 
+struct SketchHint {
+  uint32_t cnt;    // count of bin kSketchBins - 1 - threadIdx.x of the row's histogram
+  uint32_t bin0;   // key >> kSketchShift of bin 0's lower edge
+  uint32_t kmax;   // key of the row maximum
+};
+
 template <bool kStaged, bool kSketch>
 __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c,
-                           const uint32_t (&gm_hint)[kMaxCluster], bool entered) {
+                           const SketchHint &hint, bool entered) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned long long *cand_local = reinterpret_cast<unsigned long long *>(c.scratch);
   unsigned long long *cand_all = cand_local + c.cand_cap;            // 16-byte aligned: cand_cap is even
@@ -206,26 +208,34 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
   const int tail_i = (n_vec << 2) + tid;                 // the slice's last (n_local % 4) elements: threads 0..2
   const bool has_tail = tail_i < c.n_local;
 
-  uint32_t gm[kMaxCluster];
-  uint32_t kmin = 0xffffffffu, kmax = 0u, n_ne = 0u;
+  uint32_t T0 = 0u, kmax = 0u;      // key of the threshold bound, key of the row maximum
   if (kSketch) {
-    // 1'. statistics of the row's 8 x 512 group maxima, which this thread holds 8 of
-    uint32_t tmin = 0xffffffffu, tmx = 0u, tcnt = 0u;
+    // 1', 2'. the bin of the k_q-th largest group maximum, counted from the top of the row's histogram
+    const int cnt = (int)hint.cnt;
+    int inc = cnt;
 #pragma unroll
-    for (int r = 0; r < kMaxCluster; ++r) {
-      gm[r] = gm_hint[r];
-      if (gm[r] != 0u) { tmin = min(tmin, gm[r]); tmx = max(tmx, gm[r]); ++tcnt; }
+    for (int off = 1; off < 32; off <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, inc, off);
+      if (lane >= off) inc += n;
     }
-    tmin = __reduce_min_sync(0xffffffffu, tmin);
-    tmx = __reduce_max_sync(0xffffffffu, tmx);
-    tcnt = __reduce_add_sync(0xffffffffu, tcnt);
-    if (lane == 0) { sh.red[0][warp] = tmin; sh.red[1][warp] = tmx; sh.red[2][warp] = tcnt; }
-    if (tid == 0) sh.n_border = 0;
+    if (lane == 31) sh.scan_tmp[warp] = inc;
+    if (tid == 0) { sh.n_border = 0; sh.found[0] = 0; }
     __syncthreads();
+    int above = inc - cnt, total = 0;
 #pragma unroll
     for (int w = 0; w < kSelWarps; ++w) {
-      kmin = min(kmin, sh.red[0][w]); kmax = max(kmax, sh.red[1][w]); n_ne += sh.red[2][w];
+      const int t = sh.scan_tmp[w];
+      if (w < warp) above += t;
+      total += t;
     }
+    if (total < 2 * p.k_q || total > kSketchFloats) return kFastRetry;   // (the same answer in every CTA, here and below)
+    if (above < p.k_q && above + cnt >= p.k_q) sh.found[0] = kSketchBins - 1 - tid;
+    __syncthreads();
+    const uint32_t b = (uint32_t)sh.found[0];
+    if (b == 0u) return kFastRetry;                      // bin 0 also holds everything below the histogram's range
+    T0 = (hint.bin0 + b) << kSketchShift;
+    kmax = hint.kmax;
+    if (kmax < T0) return kFastRetry;
   } else {
   // 1. thread maxima (float order equals key order, so one fmaxf per element and one key per thread)
   uint32_t tmax = 0;   // 0 is below the key of every number: "no element"
@@ -283,6 +293,8 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
   cluster.sync();
 
   // 2. all maxima of the cluster -> T0 (512 bins laid over [kmin, kmax])
+  uint32_t gm[kMaxCluster];
+  uint32_t kmin = 0xffffffffu, n_ne = 0u;
 #pragma unroll
   for (int r = 0; r < kMaxCluster; ++r) {
     gm[r] = 0u;
@@ -291,8 +303,7 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
       kmin = min(kmin, sh.gstat[r][0]); kmax = max(kmax, sh.gstat[r][1]); n_ne += sh.gstat[r][2];
     }
   }
-  }
-  if ((int)n_ne < 2 * p.k_q) return kSketch ? kFastRetry : kFastGeneral;   // too few groups for a tight bound (same answer in every CTA)
+  if ((int)n_ne < 2 * p.k_q) return kFastGeneral;       // too few groups for a tight bound (same answer in every CTA)
   const uint32_t diff = kmax ^ kmin;
   const int hi = diff ? 31 - __clz(diff) : -1;           // highest bit in which the maxima differ
   const int shift = hi > 8 ? hi - 8 : 0;                 // (kmax >> shift) - (kmin >> shift) < 512
@@ -302,9 +313,10 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
     if (gm[r] != 0u) atomicAdd(&sh.hist_fast[(gm[r] >> shift) - base], 1u);
   __syncthreads();
   find_bin_from_top(sh.hist_fast, kSelThreads, p.k_q, sh);
-  const uint32_t T0 = (base + (uint32_t)sh.found[0]) << shift;
-  const float T0f = key_to_score(T0);
+  T0 = (base + (uint32_t)sh.found[0]) << shift;
   sh.hist_fast[tid] = 0;                                 // reused in step 4 (barriers in between)
+  }
+  const float T0f = key_to_score(T0);
 
   // 3. candidates: scores >= T0 as (key, position), packed so that a larger value precedes in
   //    (score desc, position asc), written in position order.  A thread's hits of one iteration are a 32-bit
@@ -641,20 +653,16 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
 
   sh.hist_fast[tid] = 0;
   c.data = grow;
-  // the row's group maxima, if the score step left them behind the row: requested ahead of the slice itself
-  uint32_t gm_hint[kMaxCluster], tag0 = 0u, tag1 = 0u;
-#pragma unroll
-  for (int r = 0; r < kMaxCluster; ++r) gm_hint[r] = 0u;
+  // the histogram of the row's group maxima, if the score step left it behind the row: requested first
+  SketchHint hint = {0u, 0u, 0u};
+  uint32_t tag0 = 0u, tag1 = 0u;
   if (sketch_off >= 0) {
-    const float *sk = p.scores + (int64_t)c.row * p.row_stride + sketch_off;
-    float v[kSketchSlices];
-#pragma unroll
-    for (int r = 0; r < kSketchSlices; ++r)
-      asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v[r]) : "l"(sk + r * kSketchGroups + tid));
-    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(tag0) : "l"(sk + kSketchFloats));
-    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(tag1) : "l"(sk + kSketchFloats + 1));
-#pragma unroll
-    for (int r = 0; r < kSketchSlices; ++r) gm_hint[r] = v[r] == -INFINITY ? 0u : score_key(v[r]);
+    const uint32_t *sk = reinterpret_cast<const uint32_t *>(p.scores + (int64_t)c.row * p.row_stride + sketch_off);
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(hint.cnt) : "l"(sk + kSketchBins - 1 - tid));
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(tag0) : "l"(sk + kSketchBins));
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(tag1) : "l"(sk + kSketchBins + 1));
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(hint.bin0) : "l"(sk + kSketchBins + 2));
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(hint.kmax) : "l"(sk + kSketchBins + 3));
   }
   if (!resident && sketch_off >= 0 && tid == 0 && c.n_local >= 4) {
     // not staged: ask for the slice to be brought into L2 while the threshold bound is worked out from the hint
@@ -685,11 +693,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     c.list = reinterpret_cast<int2 *>(c.scratch + (size_t)cand_cap * 16 + 16 + (((size_t)cand_cap + 15) & ~(size_t)15));
     int code = kFastRetry;
     if (sketch_off >= 0 && tag0 == kSketchMagic && tag1 == (uint32_t)p.E)   // the same words in every CTA of the row
-      code = resident ? fast_select<true, true>(cluster, sh, p, c, gm_hint, false)
-                      : fast_select<false, true>(cluster, sh, p, c, gm_hint, false);
+      code = resident ? fast_select<true, true>(cluster, sh, p, c, hint, false)
+                      : fast_select<false, true>(cluster, sh, p, c, hint, false);
     if (code == kFastRetry || code == kFastRetryEntered)
-      code = resident ? fast_select<true, false>(cluster, sh, p, c, gm_hint, code == kFastRetryEntered)
-                      : fast_select<false, false>(cluster, sh, p, c, gm_hint, code == kFastRetryEntered);
+      code = resident ? fast_select<true, false>(cluster, sh, p, c, hint, code == kFastRetryEntered)
+                      : fast_select<false, false>(cluster, sh, p, c, hint, code == kFastRetryEntered);
     done = code == kFastDone;
   } else {
     cluster.barrier_wait();

@@ -50,7 +50,7 @@ def test_random_cases_match_the_oracle(B, seed):
             np.testing.assert_allclose(got[b, :, :E].astype(np.float64), ref, rtol=SCORE_RTOL, atol=1e-30, err_msg=str(what))
             np.testing.assert_allclose(got[b, :, :E].astype(np.float64).sum(axis=1), 1.0, atol=1e-4, err_msg=str(what))
         if wide:
-            assert (got[:, :, E4 + 4098:] == 7.5).all() and (got[:, :, E:E4] == 7.5).all(), what
+            assert (got[:, :, E4 + 516:] == 7.5).all() and (got[:, :, E:E4] == 7.5).all(), what
         else:
             assert (got[:, :, E:] == 7.5).all(), what
         sk.close()

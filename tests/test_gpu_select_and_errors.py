@@ -136,39 +136,65 @@ def test_cache_rows_read_from_pinned_host_memory(B):
     sk.close()
 
 
-@pytest.mark.parametrize("sketch", ["true maxima", "far too high", "far too low", "garbage", "wrong tag"])
-def test_group_maxima_behind_the_rows_are_only_a_hint(B, sketch):
-    """The floats behind a long score row may hold the row's group maxima (written by sagekv_score): whatever
-    they hold, the selection is the oracle's.  Understated maxima give too many candidates, overstated ones too
-    few; both send the row through the path that computes the maxima itself."""
+def score_keys(x):
+    """Order-preserving 32-bit keys of float32 values (the kernels' comparison key)."""
+    u = (np.asarray(x, dtype=np.float32) + np.float32(0.0)).view(np.uint32)
+    return np.where(u & np.uint32(0x80000000), ~u, u | np.uint32(0x80000000)).astype(np.uint32)
+
+
+def hint_of(rows, E):
+    """What sagekv_score leaves behind rows of E scores: per row the 512-bin histogram of the maxima of the
+    8 x 512 groups (16 bins per octave below the row maximum) and the four tag words, as uint32 [H, 516]."""
+    H = rows.shape[0]
+    chunk = ((E + 7) // 8 + 3) // 4 * 4
+    out = np.zeros((H, 516), dtype=np.uint32)
+    for h in range(H):
+        gm = []
+        for r in range(8):
+            sl = rows[h, r * chunk:min(E, (r + 1) * chunk)]
+            n_vec = len(sl) // 4
+            g = np.full(512, -np.inf, dtype=np.float32)
+            if n_vec:
+                v = sl[:n_vec * 4].reshape(n_vec, 4).max(axis=1)
+                pad = (-n_vec) % 512
+                g = np.concatenate([v, np.full(pad, -np.inf, np.float32)]).reshape(-1, 512).max(axis=0)
+            for t in range(len(sl) - n_vec * 4):
+                g[t] = max(g[t], sl[n_vec * 4 + t])
+            gm.append(g)
+        gm = np.concatenate(gm)
+        gm = gm[gm > -np.inf]
+        kmax = int(score_keys(rows[h, :E].max()))
+        bin0 = (kmax >> 19) - 511
+        bins = np.clip((score_keys(gm) >> 19).astype(np.int64) - bin0, 0, 511)
+        out[h, :512] = np.bincount(bins, minlength=512).astype(np.uint32)
+        out[h, 512:] = [0x53414745, E, bin0, kmax]
+    return out
+
+
+@pytest.mark.parametrize("hint", ["true", "far too high", "far too low", "garbage", "wrong tag"])
+def test_histogram_behind_the_rows_is_only_a_hint(B, hint):
+    """The floats behind a long score row may hold the histogram of the row's group maxima (written by
+    sagekv_score): whatever they hold, the selection is the oracle's.  A bound that is too low gives too many
+    candidates, one that is too high too few; both send the row through the path that takes the maxima itself."""
     E, k_q, S, R = 60000, 300, 3, 5
     rng = np.random.default_rng(31)
     rows = (rng.random((4, E), dtype=np.float32) ** 6).astype(np.float32)
     E4 = (E + 3) // 4 * 4
-    stride = E4 + B.SKETCH_ROOM
-    buf = torch.zeros(4, stride, dtype=torch.float32, device="cuda")
+    buf = torch.zeros(4, E4 + B.SKETCH_ROOM, dtype=torch.float32, device="cuda")
     buf[:, :E] = torch.from_numpy(rows).cuda()
-    chunk = ((E + 7) // 8 + 3) // 4 * 4
-    sk_host = np.full((4, 8, 512), -np.inf, dtype=np.float32)
-    for h in range(4):
-        for r in range(8):
-            sl = rows[h, r * chunk:min(E, (r + 1) * chunk)]
-            n_vec = len(sl) // 4
-            v = sl[:n_vec * 4].reshape(n_vec, 4).max(axis=1)
-            for t in range(min(512, n_vec)):
-                sk_host[h, r, t] = v[t::512].max()
-            for t in range(len(sl) - n_vec * 4):
-                sk_host[h, r, t] = max(sk_host[h, r, t], sl[n_vec * 4 + t])
-    if sketch == "far too high":
-        sk_host[:] = 1e9
-    elif sketch == "far too low":
-        sk_host[:] = 1e-30
-    elif sketch == "garbage":
-        sk_host = rng.standard_normal(sk_host.shape).astype(np.float32) * 1e3
-        sk_host[0, 0, :7] = np.nan
-    buf[:, E4:E4 + 4096] = torch.from_numpy(sk_host.reshape(4, 4096)).cuda()
-    tag = np.array([0x53414745, E if sketch != "wrong tag" else E + 1], dtype=np.int32).view(np.float32)
-    buf[:, E4 + 4096:E4 + 4098] = torch.from_numpy(tag).cuda()
+    words = hint_of(rows, E)
+    if hint == "far too high":
+        words[:, :512] = 0
+        words[:, 511] = 4096                                  # every group maximum claimed to be near the row maximum
+    elif hint == "far too low":
+        words[:, 514] -= 40 * 16                              # bins laid 40 octaves lower: the bound lands far below
+        words[:, 515] = words[:, 514] + 511 << 19
+    elif hint == "garbage":
+        words[:, :512] = rng.integers(0, 2 ** 32, (4, 512), dtype=np.uint64).astype(np.uint32)
+        words[:, 514:] = rng.integers(0, 2 ** 32, (4, 2), dtype=np.uint64).astype(np.uint32)
+    elif hint == "wrong tag":
+        words[:, 513] += 1
+    buf[:, E4:E4 + 516] = torch.from_numpy(words.view(np.float32)).cuda()
     N = S + E + R + 1
     g = torch.Generator(device="cuda").manual_seed(5)
     K = torch.randn(1, 2, N, 128, generator=g, device="cuda").to(torch.bfloat16)
@@ -186,9 +212,9 @@ def test_group_maxima_behind_the_rows_are_only_a_hint(B, sketch):
     sk.close()
 
 
-def test_score_leaves_the_group_maxima_when_the_rows_have_room(B):
-    """sagekv_score with the wider row stride: scores as without it, and behind each row the maxima of the
-    groups (vector v of slice r belongs to group v % 512) and the tag."""
+def test_score_leaves_the_histogram_when_the_rows_have_room(B):
+    """sagekv_score with the wider row stride: scores as without it, and behind each row the histogram of the
+    group maxima with its tag; the floats after those 516 words stay untouched."""
     Hq, Hkv, N, S, R = 4, 2, 20000, 4, 16
     E = N - 1 - S - R
     g = torch.Generator(device="cuda").manual_seed(9)
@@ -197,27 +223,15 @@ def test_score_leaves_the_group_maxima_when_the_rows_have_room(B):
     sk = B.SageKV(Hq, Hkv, 128, 1, max_ctx=N, max_len=64)
     E4 = (E + 3) // 4 * 4
     narrow = torch.zeros(Hq, E4, dtype=torch.float32, device="cuda")
-    wide = torch.zeros(Hq, E4 + B.SKETCH_ROOM, dtype=torch.float32, device="cuda")
+    wide = torch.full((Hq, E4 + B.SKETCH_ROOM), 7.5, dtype=torch.float32, device="cuda")
     sk.score(q, K, S, R, scores=narrow)
-    sk.score(q, K, S, R, scores=wide)
+    for _ in range(2):                                           # the second call starts from the first one's counts
+        sk.score(q, K, S, R, scores=wide)
     torch.cuda.synchronize()
     assert torch.equal(narrow[:, :E], wide[:, :E])
-    rows = wide[:, :E].cpu().numpy()
-    got = wide[:, E4:E4 + 4096].cpu().numpy().reshape(Hq, 8, 512)
-    chunk = ((E + 7) // 8 + 3) // 4 * 4
-    for h in range(Hq):
-        for r in range(8):
-            sl = rows[h, r * chunk:min(E, (r + 1) * chunk)]
-            n_vec = len(sl) // 4
-            want = np.full(512, -np.inf, dtype=np.float32)
-            v = sl[:n_vec * 4].reshape(n_vec, 4).max(axis=1)
-            for t in range(min(512, n_vec)):
-                want[t] = v[t::512].max()
-            for t in range(len(sl) - n_vec * 4):
-                want[t] = max(want[t], sl[n_vec * 4 + t])
-            assert np.array_equal(got[h, r], want)
-    tag = wide[:, E4 + 4096:E4 + 4098].cpu().numpy().view(np.int32)
-    assert (tag[:, 0] == 0x53414745).all() and (tag[:, 1] == E).all()
+    got = wide[:, E4:E4 + 516].cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, hint_of(wide[:, :E].cpu().numpy(), E))
+    assert (wide[:, E4 + 516:] == 7.5).all() and (wide[:, E:E4] == 7.5).all()
     sk.close()
 
 

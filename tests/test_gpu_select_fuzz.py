@@ -1,6 +1,6 @@
 """Seeded random cases for select + compact: shapes, budgets, score distributions (skewed, few distinct values,
-contiguous runs, signed, softmax-like) and what lies behind the rows (nothing, the true group maxima, the maxima
-of other scores, noise).  Every case must give the oracle's indices and a bit-exact reduced cache."""
+contiguous runs, signed, softmax-like) and what lies behind the rows (nothing, the true histogram of the group
+maxima, that of other scores, noise).  Every case must give the oracle's indices and a bit-exact reduced cache."""
 
 import numpy as np
 import pytest
@@ -17,22 +17,40 @@ def B():
     return binding
 
 
-def sketch_of(rows, E):
+def score_keys(x):
+    """Order-preserving 32-bit keys of float32 values (the kernels' comparison key)."""
+    u = (np.asarray(x, dtype=np.float32) + np.float32(0.0)).view(np.uint32)
+    return np.where(u & np.uint32(0x80000000), ~u, u | np.uint32(0x80000000)).astype(np.uint32)
+
+
+def hint_of(rows, E):
+    """What sagekv_score leaves behind rows of E scores: per row the 512-bin histogram of the maxima of the
+    8 x 512 groups (16 bins per octave below the row maximum) and the four tag words, as uint32 [H, 516]."""
     H = rows.shape[0]
     chunk = ((E + 7) // 8 + 3) // 4 * 4
-    sk = np.full((H, 8, 512), -np.inf, dtype=np.float32)
+    out = np.zeros((H, 516), dtype=np.uint32)
     for h in range(H):
+        gm = []
         for r in range(8):
             sl = rows[h, r * chunk:min(E, (r + 1) * chunk)]
             n_vec = len(sl) // 4
+            g = np.full(512, -np.inf, dtype=np.float32)
             if n_vec:
                 v = sl[:n_vec * 4].reshape(n_vec, 4).max(axis=1)
                 pad = (-n_vec) % 512
-                vv = np.concatenate([v, np.full(pad, -np.inf, np.float32)]).reshape(-1, 512).max(axis=0)
-                sk[h, r] = vv
+                g = np.concatenate([v, np.full(pad, -np.inf, np.float32)]).reshape(-1, 512).max(axis=0)
             for t in range(len(sl) - n_vec * 4):
-                sk[h, r, t] = max(sk[h, r, t], sl[n_vec * 4 + t])
-    return sk.reshape(H, 4096)
+                g[t] = max(g[t], sl[n_vec * 4 + t])
+            gm.append(g)
+        gm = np.concatenate(gm)
+        gm = gm[gm > -np.inf]
+        kmax = int(score_keys(rows[h, :E].max()))
+        bin0 = (kmax >> 19) - 511
+        bins = np.clip((score_keys(gm) >> 19).astype(np.int64) - bin0, 0, 511)
+        out[h, :512] = np.bincount(bins, minlength=512).astype(np.uint32)
+        out[h, 512:] = [0x53414745, E, bin0, kmax]
+    return out
+
 
 def gen_rows(rng, H, E, kind):
     if kind == 0: r = rng.random((H, E), dtype=np.float32) ** rng.integers(1, 12)
@@ -65,21 +83,20 @@ def test_random_cases_match_the_oracle(B, seed):
         kind = int(rng.integers(0, 5))
         rows = gen_rows(rng, H, E, kind)
         E4 = (E + 3) // 4 * 4
-        # behind the rows: 0 nothing, 1 the true group maxima, 2 those of other scores, 3 noise
+        # behind the rows: 0 nothing, 1 the true histogram of the group maxima, 2 that of other scores, 3 noise
         mode = int(rng.integers(0, 4)) if E >= B.SKETCH_MIN_E else 0
         stride = E4 + (B.SKETCH_ROOM if mode else int(rng.integers(0, 3)) * 4)
         buf = torch.zeros(H, stride, dtype=torch.float32, device="cuda")
         buf[:, :E] = torch.from_numpy(rows).cuda()
         if mode:
             if mode == 1:
-                sk = sketch_of(rows, E)
+                words = hint_of(rows, E)
             elif mode == 2:
-                sk = sketch_of(gen_rows(rng, H, E, int(rng.integers(0, 5))), E)
+                words = hint_of(gen_rows(rng, H, E, int(rng.integers(0, 5))), E)
             else:
-                sk = (rng.standard_normal((H, 4096)) * 10.0 ** float(rng.integers(-6, 6))).astype(np.float32)
-            buf[:, E4:E4 + 4096] = torch.from_numpy(sk).cuda()
-            tag = np.array([0x53414745, E], dtype=np.int32).view(np.float32)
-            buf[:, E4 + 4096:E4 + 4098] = torch.from_numpy(tag).cuda()
+                words = rng.integers(0, 2 ** 32, (H, 516), dtype=np.uint64).astype(np.uint32)
+                words[:, 512:514] = [0x53414745, E]
+            buf[:, E4:E4 + 516] = torch.from_numpy(words.view(np.float32)).cuda()
         N = S + E + R + 1
         K = torch.randn(1, Hkv, N, 128, generator=gen, device="cuda").to(torch.bfloat16)
         V = torch.randn(1, Hkv, N, 128, generator=gen, device="cuda").to(torch.bfloat16)
