@@ -214,7 +214,7 @@ def run_cuda(args, w):
     for l in range(n_layers):
         lay = synth.make_layer(w, l, dev)
         lay.pop("heavy")
-        lay["scores"] = sk.new_scores(w.E)
+        lay["scores"] = sk.new_scores(w.n_ctx, w.n_init, w.n_recent)
         lay["cache"] = sk.new_layer(w.n_init, w.n_recent, w.n_sel)
         lay["out"] = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
         lay["dec"] = [synth.make_decode_inputs(w, l, t, dev) for t in range(graph_steps)]

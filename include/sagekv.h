@@ -25,6 +25,9 @@
  *   - Return value: SAGEKV_OK (0) or a negative SAGEKV_ERR_* code.  Argument
  *     errors are found on the host before anything is launched.
  *   - A query head h reads KV head h / G, G = n_q_heads / n_kv_heads <= 8.
+ *   - A context belongs to the device that was current in sagekv_create; every
+ *     later call on it must find the same device current (SAGEKV_ERR_DEVICE
+ *     otherwise).
  */
 #ifndef SAGEKV_H_
 #define SAGEKV_H_
@@ -42,11 +45,11 @@ enum {
   SAGEKV_ERR_UNSUPPORTED = -3, /* head_dim != 128, G > 8, size beyond the context's max  */
   SAGEKV_ERR_CUDA = -4,        /* a CUDA runtime call failed (see sagekv_last_cuda_error) */
   SAGEKV_ERR_NOMEM = -5,       /* scratch allocation failed in sagekv_create             */
-  SAGEKV_ERR_TOO_LARGE = -6    /* problem exceeds the fixed scratch of sagekv_score_static */
+  SAGEKV_ERR_TOO_LARGE = -6,   /* problem exceeds the fixed scratch of sagekv_score_static */
+  SAGEKV_ERR_TIMEOUT = -7,     /* sagekv_status: a bounded wait inside a kernel ran out  */
+  SAGEKV_ERR_BOUNDS = -8,      /* sagekv_status, checked build: an out-of-range index was skipped */
+  SAGEKV_ERR_DEVICE = -9       /* the context was created on another device than the current one */
 };
-
-#define SAGEKV_SKETCH_ROOM 4100   /* floats behind a score row for sagekv_score's group maxima */
-#define SAGEKV_SKETCH_MIN_E 14337 /* shortest eviction region for which they are written          */
 
 typedef struct sagekv_ctx sagekv_ctx; /* opaque; owns only its scratch memory */
 
@@ -94,8 +97,8 @@ int sagekv_destroy(sagekv_ctx *ctx);
  * Errors: INVALID for B < 4, G < 1 or a null pointer. */
 int sagekv_budget_split(int32_t B, int32_t G, int32_t *n_init, int32_t *k_q, int32_t *n_recent);
 
-/* Step 2, first half ("attention scores between the last token of the input
- * sequence and the evicted tokens").  For every batch entry b, query head h and
+/* Section 2, Step 2, first half: the last token's query scores every token of
+ * the eviction region.  For every batch entry b, query head h and
  * eviction-region offset i in [0,E):
  *     s = scale * <q_last[b,h,:], K[b, h/G, S+i, :]>
  *     scores[b,h,i] = exp(s - max_j s_j) / sum_j exp(s_j - max_j s_j),  j in [0,E)
@@ -104,27 +107,20 @@ int sagekv_budget_split(int32_t B, int32_t G, int32_t *n_init, int32_t *k_q, int
  *   K       bf16 [batch, H_kv, n_ctx, 128] addressed through `ks`.
  *   scores  fp32 [batch*H_q rows], row r at scores + r*scores_row_stride;
  *           scores_row_stride >= E and a multiple of 4, base 16-byte aligned.
- * bf16 products are accumulated in fp32.  E == 0 writes nothing.
- * Optional hint for Step 2's second half (no counterpart in the paper; it
- * changes no result): when E >= SAGEKV_SKETCH_MIN_E and scores_row_stride >=
- * round_up(E,4) + SAGEKV_SKETCH_ROOM, the call also writes, behind the E scores
- * of every row, a 512-bin histogram of the maxima of 4096 groups of that row's
- * scores and four tag words (516 32-bit words; the rest of the room is left
- * alone); the buffer must then span all of batch*H_q * scores_row_stride
- * floats.  sagekv_select_compact, given the same buffer and stride, takes its
- * first threshold bound from that histogram instead of a pass over the scores
- * (it verifies the outcome, so scores changed in between still select
- * correctly, only slower).
+ * bf16 products are accumulated in fp32.  E == 0 writes nothing.  Nothing
+ * outside the E scores of each row is written, unless the caller has asked for
+ * a hint with sagekv_set_select_hint (see there).
  * Errors: INVALID (null, n_init+n_recent+1 > n_ctx, stride < E), ALIGN,
  * UNSUPPORTED (n_ctx above the context's max_ctx), CUDA. */
 int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_strides ks,
                  int64_t n_ctx, int32_t n_init, int32_t n_recent,
                  float *scores, int64_t scores_row_stride, void *stream);
 
-/* Step 2, second half, and Step 3.  `k` is the number of selected slots per KV
- * head; it must be a multiple of G and every query head keeps k_q = min(k/G, E)
- * tokens ("this yields H_q groups of the top-k"; Appendix A.2 counts G*k
- * selected slots in the budget).  Per score row the k_q largest scores are
+/* Section 2, Step 2, second half, and Step 3.  `k` is the number of selected
+ * slots per KV head; it must be a multiple of G and every query head keeps
+ * k_q = min(k/G, E) tokens (Step 2 selects per query head, one group of kept
+ * tokens for each of the H_q heads; Appendix A.2 counts G*k selected slots in
+ * the budget).  Per score row the k_q largest scores are
  * kept; of equal scores the lower position wins; the kept positions are written
  * in ascending order (token order is maintained, Appendix A.2).
  *   idx     int32 [batch, H_q, k_q] contiguous: absolute positions in [S,S+E).
@@ -138,10 +134,9 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
  *           recent and last rows are read, so K and V may also be left in
  *           pinned (device-addressable) host memory: the gather then moves
  *           just those rows over the bus.
- *   scores  as written by sagekv_score.  With a row stride that leaves
- *           SAGEKV_SKETCH_ROOM floats behind the scores (see sagekv_score) those
- *           floats are read, whoever wrote the scores: the buffer must span
- *           batch*H_q * scores_row_stride floats.
+ *   scores  fp32 rows as written by sagekv_score (any finite numbers select
+ *           correctly).  Only the E scores of each row are read, unless the
+ *           caller has asked for a hint with sagekv_set_select_hint.
  * Scores are compared as IEEE numbers (-0 equals +0); they must not be NaN.
  * Errors: INVALID (null, k < 0, k % G != 0, bad partition), ALIGN,
  * UNSUPPORTED (L above the context's max_len), CUDA. */
@@ -151,8 +146,9 @@ int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_r
                           int32_t *idx, void *Kc, void *Vc, sagekv_strides cs,
                           sagekv_cache_state *state, void *stream);
 
-/* Step 4 ("each new token's KV pair is added to the recent window R, evicting
- * the oldest entry in R to maintain its size").  With t = *state->d_step:
+/* Section 2, Step 4: decoding on the reduced cache, the recent window rolling
+ * (a new token's key and value take the place of the window's oldest entry, so
+ * the cache keeps its length).  With t = *state->d_step:
  * if k_new / v_new are non-NULL they overwrite row S + n_sel + (t mod ring_len)
  * of every KV head (row S + n_sel is the oldest recent token after compaction)
  * and *d_step becomes t+1; with both NULL nothing is appended.  Then
@@ -188,6 +184,52 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
  *      are still read after the wait.
  * Errors: INVALID for a null context or a mode outside 0..2. */
 int sagekv_set_overlap(sagekv_ctx *ctx, int mode);
+
+/* Optional hint from the score step to the select step (no counterpart in the
+ * paper; it changes no result).  Off by default: sagekv_score then writes, and
+ * sagekv_select_compact reads, nothing but the E scores of each row, whatever
+ * the row stride, so rows may be interleaved with other data of the caller.
+ *   mode 0  off.
+ *   mode 1  for rows of at least 14337 scores sagekv_score also writes, behind
+ *           the E scores of every row (from float round_up(E,4) on), a 512-bin
+ *           histogram of the maxima of 4096 groups of that row's scores and four
+ *           tag words (516 32-bit words), and sagekv_select_compact takes its
+ *           first threshold bound from that histogram instead of a pass over
+ *           the scores.  It verifies the outcome, so scores changed in between,
+ *           or any other content of those words, still select correctly, only
+ *           slower.  The caller must give both calls a row stride of at least
+ *           sagekv_scores_row_stride() and a buffer that spans
+ *           batch*H_q * stride floats; both calls use the words only when the
+ *           stride leaves room for them.
+ * `k` is reserved for hints that depend on the later call's k (pass the k that
+ * sagekv_select_compact will get, or 0).  The setting applies to later calls on
+ * the context.  Errors: INVALID (null context, unknown mode, k < 0). */
+int sagekv_set_select_hint(sagekv_ctx *ctx, int mode, int32_t k);
+
+/* Smallest scores_row_stride (in floats, a multiple of 4) that holds a row of
+ * E = n_ctx - 1 - n_init - n_recent scores plus whatever the context's hint
+ * mode keeps behind it.  Host-only.  Negative: SAGEKV_ERR_INVALID. */
+int64_t sagekv_scores_row_stride(const sagekv_ctx *ctx, int64_t n_ctx, int32_t n_init, int32_t n_recent);
+
+/* Device-side status of the context.  The kernels never trap: a wait on a copy
+ * that does not arrive within its (generous) bound, or, in a library built
+ * with -DSAGEKV_CHECKS, a global-memory index outside the extent the call was
+ * given (the access is skipped), sets a bit in one int32 of context-owned device
+ * memory and the kernel runs to its end.  This call copies that word to
+ * *device_status (may be NULL), clears it, and returns sagekv_status_code() of
+ * it.  It synchronises (a blocking 4-byte copy): call it after synchronising
+ * the streams the context was used on, never inside a stream capture.
+ * Errors: INVALID (null context), DEVICE, CUDA, or the word's own code. */
+int sagekv_status(sagekv_ctx *ctx, int32_t *device_status);
+
+/* The return code that belongs to a status word: SAGEKV_OK for 0,
+ * SAGEKV_ERR_TIMEOUT if bit 0 is set, else SAGEKV_ERR_BOUNDS if bit 1 is set.
+ * Host-only, needs no device. */
+int sagekv_status_code(int32_t device_status);
+
+/* 1 if the library was built with -DSAGEKV_CHECKS (index checks in every
+ * kernel, slower), else 0. */
+int sagekv_checked_build(void);
 
 /* The score step without any allocation (the paper has no counterpart: this is
  * a deployment variant of sagekv_score, same arithmetic, same kernels, same

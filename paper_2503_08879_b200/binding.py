@@ -15,7 +15,8 @@ import os
 
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsagekv.so")
+# SAGEKV_LIB selects another build of the same interface (the checked build, libsagekv_checked.so)
+_LIB_PATH = os.environ.get("SAGEKV_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsagekv.so")
 if not os.path.exists(_LIB_PATH):
     raise ImportError(
         f"{_LIB_PATH} is missing: build it with `python -m paper_2503_08879_b200.build` "
@@ -23,8 +24,7 @@ if not os.path.exists(_LIB_PATH):
 lib = C.CDLL(_LIB_PATH)
 
 OK, ERR_INVALID, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
-ERR_TOO_LARGE = -6
-SKETCH_ROOM, SKETCH_MIN_E = 4100, 14337   # SAGEKV_SKETCH_ROOM, SAGEKV_SKETCH_MIN_E of include/sagekv.h
+ERR_TOO_LARGE, ERR_TIMEOUT, ERR_BOUNDS, ERR_DEVICE = -6, -7, -8, -9
 
 
 class Shape(C.Structure):
@@ -53,6 +53,16 @@ lib.sagekv_score_static.argtypes = [C.POINTER(Shape), _vp, _vp, Strides, _i64, _
 lib.sagekv_score_static.restype = C.c_int
 lib.sagekv_set_overlap.argtypes = [_vp, C.c_int]
 lib.sagekv_set_overlap.restype = C.c_int
+lib.sagekv_set_select_hint.argtypes = [_vp, C.c_int, _i32]
+lib.sagekv_set_select_hint.restype = C.c_int
+lib.sagekv_scores_row_stride.argtypes = [_vp, _i64, _i32, _i32]
+lib.sagekv_scores_row_stride.restype = _i64
+lib.sagekv_status.argtypes = [_vp, C.POINTER(_i32)]
+lib.sagekv_status.restype = C.c_int
+lib.sagekv_status_code.argtypes = [_i32]
+lib.sagekv_status_code.restype = C.c_int
+lib.sagekv_checked_build.argtypes = []
+lib.sagekv_checked_build.restype = C.c_int
 lib.sagekv_strerror.argtypes = [C.c_int]
 lib.sagekv_strerror.restype = C.c_char_p
 lib.sagekv_last_cuda_error.argtypes = [_vp]
@@ -117,6 +127,28 @@ def sagekv_set_overlap(ctx, mode: int):
     _check(lib.sagekv_set_overlap(ctx, mode), "sagekv_set_overlap", ctx)
 
 
+def sagekv_set_select_hint(ctx, mode: int, k: int = 0):
+    _check(lib.sagekv_set_select_hint(ctx, mode, k), "sagekv_set_select_hint", ctx)
+
+
+def sagekv_scores_row_stride(ctx, n_ctx: int, n_init: int, n_recent: int) -> int:
+    r = lib.sagekv_scores_row_stride(ctx, n_ctx, n_init, n_recent)
+    if r < 0:
+        _check(int(r), "sagekv_scores_row_stride", ctx)
+    return int(r)
+
+
+def sagekv_status(ctx) -> int:
+    """The context's device status word (0 = clean); raises SagekvError if any bit is set."""
+    bits = _i32(0)
+    code = lib.sagekv_status(ctx, C.byref(bits))
+    if code != OK:
+        e = SagekvError(code, "sagekv_status (word %d)" % bits.value, lib.sagekv_last_cuda_error(ctx))
+        e.bits = bits.value
+        raise e
+    return bits.value
+
+
 def sagekv_score_static(shape: Shape, q_last, K, n_ctx: int, n_init: int, n_recent: int, scores,
                         scores_row_stride: int):
     """sagekv_score without a context or any allocation: the partials live in the library's fixed array."""
@@ -171,6 +203,12 @@ class SageKV:
     def set_overlap(self, mode: int):
         sagekv_set_overlap(self.ctx, mode)
 
+    def set_select_hint(self, mode: int, k: int = 0):
+        sagekv_set_select_hint(self.ctx, mode, k)
+
+    def status(self) -> int:
+        return sagekv_status(self.ctx)
+
     def close(self):
         if self.ctx is not None:
             sagekv_destroy(self.ctx)
@@ -182,26 +220,24 @@ class SageKV:
         except Exception:
             pass
 
-    @staticmethod
-    def score_stride(E: int) -> int:
-        """Row stride of a score buffer: E rounded up to 4, plus, for rows long enough for it, the room in which
-        sagekv_score leaves the group maxima that speed up sagekv_select_compact (see include/sagekv.h)."""
-        stride = max(4, (E + 3) // 4 * 4)
-        return stride + SKETCH_ROOM if E >= SKETCH_MIN_E else stride
+    def score_stride(self, n_ctx: int, n_init: int, n_recent: int) -> int:
+        """Row stride of a score buffer for this context's hint mode (sagekv_scores_row_stride)."""
+        return sagekv_scores_row_stride(self.ctx, n_ctx, n_init, n_recent)
 
-    def new_scores(self, E: int) -> torch.Tensor:
+    def new_scores(self, n_ctx: int, n_init: int, n_recent: int) -> torch.Tensor:
         Hq, _, _, B = self.shape
-        return torch.empty(B * Hq, self.score_stride(E), dtype=torch.float32, device=self.device)
+        return torch.empty(B * Hq, self.score_stride(n_ctx, n_init, n_recent), dtype=torch.float32,
+                           device=self.device)
 
-    def new_layer(self, n_init: int, n_recent: int, k: int) -> Layer:
+    def new_layer(self, n_init: int, n_recent: int, k: int, spare_rows: int = 0) -> Layer:
+        """Buffers for a reduced cache of L = n_init + k + n_recent + 1 rows (plus `spare_rows` unused ones)."""
         Hq, Hkv, d, B = self.shape
-        return Layer(B, Hq, Hkv, d, n_init + k + n_recent + 1, k // self.G, self.device)
+        return Layer(B, Hq, Hkv, d, n_init + k + n_recent + 1 + spare_rows, k // self.G, self.device)
 
     def score(self, q_last, K, n_init, n_recent, scores=None):
         n_ctx = K.shape[2]
-        E = n_ctx - 1 - n_init - n_recent
         if scores is None:
-            scores = self.new_scores(E)
+            scores = self.new_scores(n_ctx, n_init, n_recent)
         sagekv_score(self.ctx, q_last, K, n_ctx, n_init, n_recent, scores, scores.stride(0))
         return scores
 

@@ -1,5 +1,6 @@
 // The C interface (include/sagekv.h): argument checks on the host, then the kernel launches.
 #include <math.h>
+#include <mutex>
 #include <new>
 
 #include "common.cuh"
@@ -11,15 +12,19 @@ struct sagekv_ctx {
   int G;
   int64_t max_ctx;
   int32_t max_len;
-  int n_sm;
+  int device;               // the device the context was created on; every call must find it current
+  const DeviceInfo *dev;    // that device's one-time set-up
   float scale;
   float2 *score_partials;   // [B*H_q, ceil(max_ctx / kScoreChunk)]
   int max_chunks;
   float *decode_partials;   // [B*H_kv, max_splits (clusters per head), kPartialStride]
   int max_splits;
-  int32_t *tickets;         // [B*H_kv + 1], zero between launches
+  int32_t *tickets;         // [B*H_kv + 1], zero between launches; the status word follows them
+  int32_t *status;          // one int32: kStatus* bits raised by the kernels
   int last_cuda_error;
   int overlap;              // 0, 1 or 2: see sagekv_set_overlap
+  int hint;                 // 0, 1: see sagekv_set_select_hint
+  int32_t hint_k;
 };
 
 namespace {
@@ -31,6 +36,32 @@ bool strides_ok(const sagekv_strides &s) {
 int cuda_fail(sagekv_ctx *ctx, cudaError_t e) {
   if (ctx) ctx->last_cuda_error = (int)e;
   return SAGEKV_ERR_CUDA;
+}
+
+// One-time set-up per device (function attributes, SM count, cluster capacities), done with that device current.
+constexpr int kMaxDevices = 64;
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_dev_mutex;
+
+cudaError_t device_setup(int dev, const DeviceInfo **out) {
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_dev_mutex);
+  DeviceInfo &d = g_dev[dev];
+  if (!d.ready) {
+    cudaError_t e = cudaDeviceGetAttribute(&d.n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = select_compact_setup();
+    if (e == cudaSuccess) e = decode_setup(&d);
+    if (e != cudaSuccess) return e;
+    d.ready = true;
+  }
+  *out = &d;
+  return cudaSuccess;
+}
+
+// false: another device is current than the one the context belongs to
+bool on_own_device(const sagekv_ctx *ctx) {
+  int cur = -1;
+  return cudaGetDevice(&cur) == cudaSuccess && cur == ctx->device;
 }
 
 }  // namespace
@@ -55,27 +86,28 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   ctx->scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.0f / sqrtf((float)shape->head_dim);
   ctx->last_cuda_error = 0;
   ctx->overlap = 0;
+  ctx->hint = 0;
+  ctx->hint_k = 0;
   int dev = 0;
-  cudaDeviceProp prop;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+  if (cudaGetDevice(&dev) != cudaSuccess || device_setup(dev, &ctx->dev) != cudaSuccess) {
     delete ctx;
+    (void)cudaGetLastError();
     return SAGEKV_ERR_CUDA;
   }
-  ctx->n_sm = prop.multiProcessorCount;
+  ctx->device = dev;
   ctx->max_chunks = (int)((max_ctx + kScoreChunk - 1) / kScoreChunk);
   {
-    int cs, n_warps, smem;
-    decode_geometry(max_len, 0, &ctx->max_splits, &cs, &n_warps, &smem);   // clusters per head at the largest L
+    int cs, resident, smem;
+    decode_geometry(max_len, 0, nullptr, &ctx->max_splits, &cs, &resident, &smem);   // clusters per head at the largest L
   }
   const size_t n_rows = (size_t)shape->batch * shape->n_q_heads;
   const size_t n_heads = (size_t)shape->batch * shape->n_kv_heads;
   cudaError_t e = cudaMalloc(&ctx->score_partials, n_rows * ctx->max_chunks * sizeof(float2));
   if (e == cudaSuccess)
     e = cudaMalloc(&ctx->decode_partials, n_heads * ctx->max_splits * kPartialStride * sizeof(float));
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->tickets, (n_heads + 1) * sizeof(int32_t));
-  if (e == cudaSuccess) e = cudaMemset(ctx->tickets, 0, (n_heads + 1) * sizeof(int32_t));
-  if (e == cudaSuccess) e = select_compact_setup();
-  if (e == cudaSuccess) e = decode_setup();
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->tickets, (n_heads + 2) * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(ctx->tickets, 0, (n_heads + 2) * sizeof(int32_t));
+  if (e == cudaSuccess) ctx->status = ctx->tickets + n_heads + 1;
   if (e != cudaSuccess) {
     cudaFree(ctx->score_partials);
     cudaFree(ctx->decode_partials);
@@ -118,6 +150,7 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
   if (ctx == nullptr || q_last == nullptr || K == nullptr || scores == nullptr) return SAGEKV_ERR_INVALID;
   if (n_init < 0 || n_recent < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx) return SAGEKV_ERR_INVALID;
   if (n_ctx > ctx->max_ctx) return SAGEKV_ERR_UNSUPPORTED;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
   const int64_t E = n_ctx - 1 - n_init - n_recent;
   if (scores_row_stride < E || ks.token_stride < kHeadDim) return SAGEKV_ERR_INVALID;
   if (!aligned16(q_last) || !aligned16(K) || !aligned16(scores) || !strides_ok(ks) || scores_row_stride % 4 != 0)
@@ -129,7 +162,8 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
   p.scores = scores;
   p.row_stride = scores_row_stride;
   p.partials = ctx->score_partials;
-  p.sketch = true;
+  p.sketch = ctx->hint == 1;
+  p.status = ctx->status;
   p.n_chunks = (int)((E + kScoreChunk - 1) / kScoreChunk);
   p.E = (int)E;
   p.S = n_init;
@@ -138,7 +172,7 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
   p.H_kv = ctx->shape.n_kv_heads;
   p.B = ctx->shape.batch;
   p.scale_log2 = ctx->scale * kLog2e;
-  const cudaError_t e = launch_score(p, ctx->n_sm, static_cast<cudaStream_t>(stream));
+  const cudaError_t e = launch_score(p, ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
 }
 
@@ -153,6 +187,7 @@ int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_r
       k % ctx->G != 0)
     return SAGEKV_ERR_INVALID;
   if (n_ctx > ctx->max_ctx) return SAGEKV_ERR_UNSUPPORTED;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
   const int64_t E = n_ctx - 1 - n_init - n_recent;
   int64_t k_q = k / ctx->G;
   if (k_q > E) k_q = E;
@@ -183,7 +218,9 @@ int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_r
   p.H_q = ctx->shape.n_q_heads;
   p.H_kv = ctx->shape.n_kv_heads;
   p.B = ctx->shape.batch;
-  const cudaError_t e = launch_select_compact(p, ctx->n_sm, static_cast<cudaStream_t>(stream));
+  p.status = ctx->status;
+  p.sketch = ctx->hint == 1;
+  const cudaError_t e = launch_select_compact(p, ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   state->n_init = n_init;
   state->k_q = (int32_t)k_q;
@@ -205,6 +242,7 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
       cs.token_stride < kHeadDim)
     return SAGEKV_ERR_INVALID;
   if (state->len > ctx->max_len) return SAGEKV_ERR_UNSUPPORTED;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
   if (!aligned16(q) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(out) || !strides_ok(cs) ||
       (k_new != nullptr && (!aligned16(k_new) || !aligned16(v_new))))
     return SAGEKV_ERR_ALIGN;
@@ -220,6 +258,7 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
   p.partials = ctx->decode_partials;
   p.tickets = ctx->tickets;
   p.d_step = state->d_step;
+  p.status = ctx->status;
   p.S = state->n_init;
   p.k_q = state->k_q;
   p.n_sel = state->n_sel;
@@ -231,7 +270,7 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
   p.B = ctx->shape.batch;
   p.scale_log2 = ctx->scale * kLog2e;
   p.pdl_mode = ctx->overlap;
-  const cudaError_t e = launch_decode(p, static_cast<cudaStream_t>(stream));
+  const cudaError_t e = launch_decode(p, *ctx->dev, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
 }
 
@@ -239,6 +278,48 @@ int sagekv_set_overlap(sagekv_ctx *ctx, int mode) {
   if (ctx == nullptr || mode < 0 || mode > 2) return SAGEKV_ERR_INVALID;
   ctx->overlap = mode;
   return SAGEKV_OK;
+}
+
+int sagekv_set_select_hint(sagekv_ctx *ctx, int mode, int32_t k) {
+  if (ctx == nullptr || mode < 0 || mode > 1 || k < 0) return SAGEKV_ERR_INVALID;
+  ctx->hint = mode;
+  ctx->hint_k = k;
+  return SAGEKV_OK;
+}
+
+int64_t sagekv_scores_row_stride(const sagekv_ctx *ctx, int64_t n_ctx, int32_t n_init, int32_t n_recent) {
+  if (ctx == nullptr || n_init < 0 || n_recent < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx)
+    return SAGEKV_ERR_INVALID;
+  const int64_t E = n_ctx - 1 - n_init - n_recent;
+  int64_t stride = (E + 3) & ~(int64_t)3;
+  if (stride < 4) stride = 4;
+  if (ctx->hint == 1 && E >= kSketchMinE) stride += kSketchRoom;
+  return stride;
+}
+
+int sagekv_status_code(int32_t bits) {
+  if (bits & kStatusWaitTimeout) return SAGEKV_ERR_TIMEOUT;
+  if (bits & kStatusBounds) return SAGEKV_ERR_BOUNDS;
+  return SAGEKV_OK;
+}
+
+int sagekv_status(sagekv_ctx *ctx, int32_t *device_status) {
+  if (ctx == nullptr) return SAGEKV_ERR_INVALID;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
+  int32_t bits = 0;
+  cudaError_t e = cudaMemcpy(&bits, ctx->status, sizeof(bits), cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && bits != 0) e = cudaMemset(ctx->status, 0, sizeof(bits));
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  if (device_status != nullptr) *device_status = bits;
+  return sagekv_status_code(bits);
+}
+
+int sagekv_checked_build(void) {
+#if defined(SAGEKV_CHECKS)
+  return 1;
+#else
+  return 0;
+#endif
 }
 
 const char *sagekv_strerror(int code) {
@@ -250,6 +331,9 @@ const char *sagekv_strerror(int code) {
     case SAGEKV_ERR_CUDA: return "CUDA runtime error";
     case SAGEKV_ERR_NOMEM: return "out of memory";
     case SAGEKV_ERR_TOO_LARGE: return "problem larger than the fixed scratch array";
+    case SAGEKV_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case SAGEKV_ERR_BOUNDS: return "checked build: an index outside its buffer was skipped";
+    case SAGEKV_ERR_DEVICE: return "the context belongs to another device than the current one";
     default: return "unknown error code";
   }
 }

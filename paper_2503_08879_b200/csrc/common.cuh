@@ -30,6 +30,7 @@ struct ScoreParams {
   float scale_log2;        // softmax scale * log2(e)
   bool sketch = false;     // leave the histogram of the group maxima behind each row that has room for it
   int64_t sketch_off = -1; // set by launch_score: where in a row it goes, or -1
+  int32_t *status = nullptr;   // status word of the context, or null (see kStatus*)
 };
 cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream);
 
@@ -47,7 +48,7 @@ constexpr int kSketchGroups = 512;
 constexpr int kSketchBins = 512;
 constexpr int kSketchShift = 19;                               // key bits below a bin: 2^23 keys per octave / 16
 constexpr int kSketchFloats = kSketchSlices * kSketchGroups;   // groups per row
-constexpr int kSketchRoom = 4100;                              // floats reserved behind a row (SAGEKV_SKETCH_ROOM)
+constexpr int kSketchRoom = kSketchBins + 8;                   // 32-bit words reserved behind a row: the bins, four tag words, padding
 constexpr uint32_t kSketchMagic = 0x53414745u;
 constexpr int kSketchMinE = 7 * 2048 + 1;                      // rows long enough for clusters of 8 in the select step
 inline __host__ __device__ int64_t sketch_offset(int64_t E) { return (E + 3) & ~(int64_t)3; }
@@ -67,15 +68,18 @@ struct SelectParams {
   int32_t *idx;            // [B, H_q, k_q]
   int32_t *d_step;
   int E, S, R, N, k_q, G, H_q, H_kv, B;
+  int32_t *status = nullptr;   // status word of the context, or null
+  bool sketch = false;         // the caller asked for the histograms behind the rows to be used (sagekv_set_select_hint)
 };
 cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t stream);
 cudaError_t select_compact_setup();   // one-time function attributes
 
 // ---- decode attention ------------------------------------------------------
-constexpr int kDecodeMaxWarps = 12;                                    // warps per CTA, one or two 16-row tiles each
+constexpr int kDecodeWarps = 8;                                        // warps per CTA
 constexpr int kDecodeMaxCluster = 8;                                   // CTAs per cluster (the portable limit)
-constexpr int kDecodeMaxPasses = 4;                                    // passes over the staging area before a head gets more clusters
-constexpr int kDecodeMaxTiles = 24;                                    // 16-row tiles (K and V) a CTA can stage: 192 KB
+constexpr int kDecodeMaxResident = 24;                                 // 16-row tiles (K and V) a CTA holds at once: 192 KB
+constexpr int kDecodeRoundTiles = 12;                                  // tiles per round when the partition is longer (two buffers)
+constexpr int kDecodeMaxRounds = 8;                                    // rounds before a head gets more clusters
 constexpr int kPartialStride = kMaxGroup * kHeadDim + 2 * kMaxGroup;   // floats per cluster result: O[8][128], m[8], l[8]
 
 struct DecodeParams {
@@ -89,16 +93,43 @@ struct DecodeParams {
   float *partials;         // [B*H_kv, clusters per head, kPartialStride]; used only with several clusters per head
   int32_t *tickets;        // [B*H_kv] arrival counters + [1] finished-heads counter, all 0 between launches
   int32_t *d_step;
+  int32_t *status;         // the context's status word (see kStatus*)
   int S, k_q, n_sel, ring_len, L, G, H_q, H_kv, B;
   float scale_log2;
-  int pdl_mode;            // 0 plain launch, 1 programmatic dependent launch, 2 also prefetch the cache before the wait
+  int pdl_mode;            // 0 plain launch, 1 programmatic dependent launch, 2 also fetch the cache before the wait
 };
-cudaError_t launch_decode(const DecodeParams &p, cudaStream_t stream);
-cudaError_t decode_setup();           // one-time function attributes
-void decode_geometry(int L, int heads, int *n_clusters, int *cluster_size, int *n_warps, int *smem_bytes);
+
+// What the one-time set-up of a device leaves behind (function attributes are set as a side effect).
+struct DeviceInfo {
+  int n_sm;
+  int cluster_cap[kDecodeMaxCluster + 1];   // decode clusters of each size that can be resident at once
+  bool ready;
+};
+cudaError_t launch_decode(const DecodeParams &p, const DeviceInfo &dev, cudaStream_t stream);
+cudaError_t decode_setup(DeviceInfo *dev);   // one-time, with the device current
+void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, int *cluster_size, int *resident_tiles,
+                     int *smem_bytes);
+
+// ---- status word -------------------------------------------------------------
+// One int32 in device memory per context, OR-ed into by the kernels, read by sagekv_status.
+constexpr int kStatusWaitTimeout = 1;   // a bounded wait on a copy barrier gave up
+constexpr int kStatusBounds = 2;        // checked build: an index outside its buffer was found and the access skipped
+
+// In a build with -DSAGEKV_CHECKS every global-memory index of the kernels is compared with the extent the
+// call was given; a violation sets kStatusBounds and the access is skipped (nothing traps).  Otherwise the
+// condition is not evaluated.
+#if defined(SAGEKV_CHECKS)
+#define SAGEKV_OK_INDEX(status, cond) ((cond) ? true : (sagekv::note_bad_index(status), false))
+#else
+#define SAGEKV_OK_INDEX(status, cond) (true)
+#endif
 
 // ---- device helpers --------------------------------------------------------
 #if defined(__CUDACC__)
+
+__device__ __forceinline__ void note_bad_index(int32_t *status) {
+  if (status != nullptr) atomicOr(status, kStatusBounds);
+}
 
 // 16-byte read-only load that does not linger in L1: cache rows are streamed once.
 __device__ __forceinline__ uint4 ld_stream_v4(const void *ptr) {

@@ -47,10 +47,11 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_logits_kernel(const Sc
     const int r1 = min(tok_base + t * 16 + g + 8, last);
     const char *pa = reinterpret_cast<const char *>(Kbase + (int64_t)r0 * p.ks.token_stride) + c * 16;
     const char *pb = reinterpret_cast<const char *>(Kbase + (int64_t)r1 * p.ks.token_stride) + c * 16;
+    const bool ok = SAGEKV_OK_INDEX(p.status, r0 >= 0 && r0 < p.E && r1 >= 0 && r1 < p.E && kvh < p.H_kv && b < p.B);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      ka[t][j] = ld_stream_v4(pa + j * 64);
-      kb[t][j] = ld_stream_v4(pb + j * 64);
+      ka[t][j] = ok ? ld_stream_v4(pa + j * 64) : make_uint4(0u, 0u, 0u, 0u);
+      kb[t][j] = ok ? ld_stream_v4(pb + j * 64) : make_uint4(0u, 0u, 0u, 0u);
     }
   }
 
@@ -71,7 +72,8 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_logits_kernel(const Sc
     const int r0 = tok_base + t * 16 + g, r1 = r0 + 8;
     const float s00 = a0 * p.scale_log2, s01 = a1 * p.scale_log2;   // (r0,h0) (r0,h1)
     const float s10 = a2 * p.scale_log2, s11 = a3 * p.scale_log2;   // (r1,h0) (r1,h1)
-    const bool v0 = r0 < p.E, v1 = r1 < p.E;
+    const bool v0 = r0 < p.E && SAGEKV_OK_INDEX(p.status, r0 >= 0 && (int64_t)r0 < p.row_stride);
+    const bool v1 = r1 < p.E && SAGEKV_OK_INDEX(p.status, r1 >= 0 && (int64_t)r1 < p.row_stride);
     if (h0 < p.G) {
       if (v0) row0[r0] = s00;
       if (v1) row0[r1] = s10;
@@ -107,7 +109,8 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_logits_kernel(const Sc
     float m = sm_m[0][h], l = sm_l[0][h];
 #pragma unroll
     for (int w = 1; w < kScoreWarps; ++w) merge_ml(m, l, sm_m[w][h], sm_l[w][h]);
-    p.partials[((int64_t)b * p.H_q + kvh * p.G + h) * p.n_chunks + chunk] = make_float2(m, l);
+    if (SAGEKV_OK_INDEX(p.status, chunk < p.n_chunks && kvh * p.G + h < p.H_q))
+      p.partials[((int64_t)b * p.H_q + kvh * p.G + h) * p.n_chunks + chunk] = make_float2(m, l);
   }
 }
 
@@ -136,6 +139,7 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_finalize_kernel(const 
   float *rowp = p.scores + (int64_t)row * p.row_stride;
   const int lo = blockIdx.x * per_slice;            // per_slice is a multiple of 4
   const int hi = min(p.E, lo + per_slice);
+  if (!SAGEKV_OK_INDEX(p.status, row < p.B * p.H_q && lo >= 0 && (int64_t)hi <= p.row_stride)) return;
   // eight 16-byte loads in flight per thread before the first store (the row is read and written in place,
   // so the compiler would otherwise keep every load behind the previous store)
   for (int i0 = lo + threadIdx.x * 4; i0 < hi; i0 += kFinalizeThreads * 4 * 8) {
@@ -187,6 +191,8 @@ __global__ void __launch_bounds__(kSketchThreads) score_finalize_sketch_kernel(c
   float *rowp = p.scores + (int64_t)row * p.row_stride;
   const int lo = slice * chunk;
   const int n_local = max(0, min(p.E - lo, chunk));
+  if (!SAGEKV_OK_INDEX(p.status, row < p.B * p.H_q && p.sketch_off >= p.E && p.sketch_off + kSketchBins + 4 <= p.row_stride))
+    return;
   const int n_vec = n_local >> 2;
   float *base = rowp + lo;
   float fm = -INFINITY;

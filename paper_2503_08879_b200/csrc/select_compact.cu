@@ -116,7 +116,9 @@ __device__ __forceinline__ void copy_kv_row(const SelectParams &p, int b, int kv
   uint16_t *dst = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
                   dst_row * p.cs.token_stride;
   const int piece = (lane & 15) * 8;
-  st_v4(dst + piece, ld_stream_v4(src + piece));
+  if (SAGEKV_OK_INDEX(p.status, src_tok >= 0 && src_tok < p.N && dst_row >= 0 &&
+                                    dst_row < (int64_t)p.S + (int64_t)p.G * p.k_q + p.R + 1))
+    st_v4(dst + piece, ld_stream_v4(src + piece));
 }
 
 // sink rows, recent rows and the last token: positions known without the scores
@@ -496,6 +498,7 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
       if (flag[i]) {
         if (slot >= slot_lo && slot < slot_hi) {
           const int pos = p.S + (int)(0xffffffffu - (uint32_t)(cand_all[i] & 0xffffffffull));
+          (void)SAGEKV_OK_INDEX(p.status, pos >= p.S && pos < p.S + p.E && slot - slot_lo < c.list_cap);
           idx_row[slot] = pos;
           c.list[slot - slot_lo] = make_int2(slot, pos);
         }
@@ -609,7 +612,7 @@ __device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const 
     else if (eq && e_here < ties_kept) slot = g_here + e_here;
     if (slot >= 0) {
       const int pos = p.S + c.lo + i;
-      idx_row[slot] = pos;
+      if (SAGEKV_OK_INDEX(p.status, slot < p.k_q && pos < p.S + p.E)) idx_row[slot] = pos;
       const int n = atomicAdd(&sh.list_count, 1);
       if (n < c.list_cap) c.list[n] = make_int2(slot, pos);
     }
@@ -650,6 +653,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   const int b = c.row / p.H_q, h = c.row - b * p.H_q;
   const int kvh = h / p.G, j = h - kvh * p.G;
   const float *grow = p.scores + (int64_t)c.row * p.row_stride + c.lo;   // 16-byte aligned: chunk % 4 == 0
+  (void)SAGEKV_OK_INDEX(p.status, c.row < p.B * p.H_q && (int64_t)c.lo + c.n_local <= p.row_stride && c.lo + c.n_local <= p.E &&
+                                      (sketch_off < 0 || sketch_off + kSketchBins + 4 <= p.row_stride));
 
   sh.hist_fast[tid] = 0;
   c.data = grow;
@@ -725,12 +730,14 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     const bool has_static = sr < n_static;
     if (has_static) {
       const int64_t src_tok = sr < p.S ? sr : (int64_t)p.E + sr;                 // S + E + (sr - S)
+      (void)SAGEKV_OK_INDEX(p.status, src_tok >= 0 && src_tok < p.N);
       vs = ld_stream_v4(src_base + src_tok * p.ks.token_stride);
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       if (e0 < n_list) {
-        const int2 sp = c.list[min(e0 + u, n_list - 1)];
+        int2 sp = c.list[min(e0 + u, n_list - 1)];
+        if (!SAGEKV_OK_INDEX(p.status, sp.x >= 0 && sp.x < p.k_q && sp.y >= p.S && sp.y < p.S + p.E)) sp = make_int2(0, p.S);
         slot[u] = sp.x;
         v[u] = ld_stream_v4(src_base + (int64_t)sp.y * p.ks.token_stride);
       }
@@ -769,7 +776,7 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   // The rows may carry the group maxima of the score step (see common.cuh): then the threshold bound costs no
   // pass over the data, the slice is read straight from global memory (no staging: it is needed once), and with
   // many rows smaller clusters pay, because two CTAs per SM times the SM count is all that runs at once.
-  const bool sketch = select && sketch_fits(p.E, p.row_stride);
+  const bool sketch = select && p.sketch && sketch_fits(p.E, p.row_stride);
   // cluster size: slices of at least 2048 scores, at most 8 CTAs (the portable limit)
   int cs = 1;
   while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E && (!sketch || (int64_t)n_rows * cs * 2 <= 2 * (int64_t)n_sm)) cs <<= 1;

@@ -37,8 +37,35 @@ def test_every_declared_symbol_is_exported(lib):
 def test_strerror(lib):
     lib.sagekv_strerror.restype = ctypes.c_char_p
     assert lib.sagekv_strerror(0) == b"ok"
-    texts = {lib.sagekv_strerror(c) for c in range(-5, 1)}
-    assert len(texts) == 6 and lib.sagekv_strerror(-99) not in texts
+    texts = {lib.sagekv_strerror(c) for c in range(-9, 1)}
+    assert len(texts) == 10 and lib.sagekv_strerror(-99) not in texts
+    assert b"another device" in lib.sagekv_strerror(-9)          # SAGEKV_ERR_DEVICE: context used off its device
+
+
+def test_status_word_maps_to_a_return_code(lib):
+    """Host logic of sagekv_status: which return code a device status word gives (needs no device)."""
+    code = lib.sagekv_status_code
+    code.argtypes, code.restype = [ctypes.c_int32], ctypes.c_int
+    assert code(0) == 0
+    assert code(1) == -7                 # a bounded wait ran out: SAGEKV_ERR_TIMEOUT
+    assert code(2) == -8                 # checked build found an index out of range: SAGEKV_ERR_BOUNDS
+    assert code(3) == -7                 # the timeout is reported first
+    assert lib.sagekv_status(None, None) == -1
+    assert lib.sagekv_checked_build() == 0
+
+
+def test_checked_build_compiles_and_says_so():
+    from paper_2503_08879_b200 import build
+    checked = ctypes.CDLL(build.build(checks=True))
+    assert checked.sagekv_checked_build() == 1
+    for name in declared_symbols():
+        assert getattr(checked, name) is not None, name
+
+
+def test_hint_and_stride_helpers_reject_bad_arguments(lib):
+    lib.sagekv_scores_row_stride.restype = ctypes.c_int64
+    assert lib.sagekv_set_select_hint(None, 1, 0) == -1
+    assert lib.sagekv_scores_row_stride(None, ctypes.c_int64(100), 4, 16) == -1
 
 
 def test_budget_split_host_function_matches_paper_and_oracle(lib):

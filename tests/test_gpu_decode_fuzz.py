@@ -8,6 +8,7 @@ import pytest
 import torch
 
 from oracle import sagekv_oracle as O
+from helpers import bits
 
 pytestmark = pytest.mark.gpu
 OUT_ATOL, OUT_RTOL = 1e-2, 1e-2
@@ -17,10 +18,6 @@ OUT_ATOL, OUT_RTOL = 1e-2, 1e-2
 def B():
     from paper_2503_08879_b200 import binding
     return binding
-
-
-def bits(t):
-    return t.detach().cpu().contiguous().view(torch.uint16).numpy()
 
 
 def f32(a):
@@ -47,11 +44,12 @@ def test_random_cases_match_the_oracle(B, seed):
         buf = torch.zeros(Bt * H, max(4, (E + 3) // 4 * 4), dtype=torch.float32, device="cuda")
         if E:
             buf[:, :E] = torch.from_numpy(rows[:, :E]).cuda()
-        sk = B.SageKV(H, Hkv, 128, Bt, max_ctx=N, max_len=L)
+        sm_scale = float(rng.choice([0.0, 0.0, 0.05, 0.2]))      # softmax scale of the context; 0: the default 1/sqrt(d)
+        sk = B.SageKV(H, Hkv, 128, Bt, max_ctx=N, max_len=L, softmax_scale=sm_scale)
         sk.set_overlap(int(rng.integers(0, 2)))
         layer = sk.select_compact(buf if k_q else None, K, V, S, R, G * k_q)
         torch.cuda.synchronize()
-        what = dict(case=case, G=G, Hkv=Hkv, batch=Bt, S=S, R=R, k_q=k_q, E=E, L=L)
+        what = dict(case=case, G=G, Hkv=Hkv, batch=Bt, S=S, R=R, k_q=k_q, E=E, L=L, softmax_scale=sm_scale)
         caches = []
         for b in range(Bt):
             idx = O.select(rows[b * H:(b + 1) * H, :E], k_q, S) if k_q else np.zeros((H, 0), np.int32)
@@ -66,10 +64,11 @@ def test_random_cases_match_the_oracle(B, seed):
             torch.cuda.synchronize()
             for b in range(Bt):
                 ref, _, steps[b] = O.decode_step(bits(q[b]), bits(kn[b]), bits(vn[b]), caches[b][0], caches[b][1],
-                                                 steps[b], S, k_q, R)
+                                                 steps[b], S, k_q, R, scale=sm_scale if sm_scale > 0 else None)
                 got = f32(bits(out[b])).astype(np.float64)
                 assert np.all(np.abs(got - ref) <= OUT_ATOL + OUT_RTOL * np.abs(ref)), what
         Kc, Vc = layer.cache()
         for b in range(Bt):
             assert np.array_equal(bits(Kc[b]), caches[b][0]) and np.array_equal(bits(Vc[b]), caches[b][1]), what
+        assert sk.status() == 0, what
         sk.close()

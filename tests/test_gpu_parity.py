@@ -14,6 +14,7 @@ import pytest
 import torch
 
 from oracle import sagekv_oracle as O
+from helpers import bits
 from paper_2503_08879_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -29,12 +30,8 @@ def B():
     return binding
 
 
-def bits(t: torch.Tensor) -> np.ndarray:
-    return t.detach().cpu().contiguous().view(torch.uint16).numpy()
-
-
-def check_scores(gpu_scores, lay, w, b):
-    ref = O.score(bits(lay["q_last"][b]), bits(lay["K"][b]), w.n_init, w.n_recent)
+def check_scores(gpu_scores, lay, w, b, scale=None):
+    ref = O.score(bits(lay["q_last"][b]), bits(lay["K"][b]), w.n_init, w.n_recent, scale=scale)
     got = gpu_scores.view(w.batch, w.n_q_heads, -1)[b, :, : w.E].cpu().numpy().astype(np.float64)
     np.testing.assert_allclose(got, ref, rtol=SCORE_RTOL, atol=1e-30)
     if w.E > 0:
@@ -72,8 +69,20 @@ def check_out(out, ref):
     assert np.all(err <= OUT_ATOL + OUT_RTOL * np.abs(ref)), float(err.max())
 
 
-def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0):
-    """All four steps on one layer of workload `w`, every result checked against the oracle."""
+CANARY = 0x5A5A           # bf16 bit pattern in the guard rows of the reduced cache
+GUARD_ROWS = 2
+
+
+def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0, hint=0, scale=0.0, sampled_heads=None):
+    """All four steps on one layer of workload `w`, every result checked against the oracle.
+
+    Every output buffer carries a guard band (rows behind the reduced cache, floats behind each score row, an
+    extra row behind `out`) that must still hold its fill value at the end; score and the first decode step
+    run twice and must repeat bit for bit; the context's status word must stay clean.
+    sampled_heads: check scores and indices for these query heads only (the oracle's select takes seconds per
+    long row); caches and outputs are always checked in full.
+    """
+    oscale = scale if scale > 0 else None
     lay = synth.make_layer(w, 0, device)
     K, V = lay["K"], lay["V"]
     if strided:   # token stride 136 and a gap between heads: exercises the stride arguments
@@ -82,45 +91,80 @@ def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0):
         Kp[:, :, : w.n_ctx, :128] = K
         Vp[:, :, : w.n_ctx, :128] = V
         K, V = Kp[:, :, : w.n_ctx, :128], Vp[:, :, : w.n_ctx, :128]
-    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L, softmax_scale=scale)
     sk.set_overlap(overlap)
-    scores = sk.score(lay["q_last"], K, w.n_init, w.n_recent)
-    layer = sk.select_compact(scores, K, V, w.n_init, w.n_recent, w.n_sel)
+    sk.set_select_hint(hint, w.n_sel)
+    stride = sk.score_stride(w.n_ctx, w.n_init, w.n_recent)
+    n_rows = w.batch * w.n_q_heads
+    buf = torch.full((n_rows, stride + 8), 7.5, dtype=torch.float32, device=device)
+    scores = buf[:, :stride]
+    B.sagekv_score(sk.ctx, lay["q_last"], K, w.n_ctx, w.n_init, w.n_recent, scores, buf.stride(0))
+    first = scores[:, : w.E].clone()
+    B.sagekv_score(sk.ctx, lay["q_last"], K, w.n_ctx, w.n_init, w.n_recent, scores, buf.stride(0))
+    layer = sk.new_layer(w.n_init, w.n_recent, w.n_sel, spare_rows=GUARD_ROWS)
+    layer.Kc.view(torch.int16).fill_(CANARY)
+    layer.Vc.view(torch.int16).fill_(CANARY)
+    sk.select_compact(scores, K, V, w.n_init, w.n_recent, w.n_sel, layer)
     torch.cuda.synchronize()
+    assert torch.equal(first, scores[:, : w.E])                       # the score step repeats bit for bit
+    assert (buf[:, stride:] == 7.5).all()                             # nothing written behind the rows' stride
+    if hint == 0:
+        assert (buf[:, w.E:] == 7.5).all()
     st = layer.state
     k_q = min(w.k_q, w.E)
     assert (st.n_init, st.k_q, st.n_sel, st.n_recent, st.ring_len, st.len) == (
         w.n_init, k_q, w.G * k_q, w.n_recent, w.n_recent + 1, w.n_init + w.G * k_q + w.n_recent + 1)
     assert int(layer.step.item()) == 0
+    heads = list(range(w.n_q_heads)) if sampled_heads is None else list(sampled_heads)
     caches = []
     for b in range(w.batch):
-        ref_scores, got_scores = check_scores(scores, lay, w, b)
         idx_gpu = layer.indices()[b].cpu().numpy()
-        if k_q > 0:
-            check_select(idx_gpu, got_scores, ref_scores, w, k_q)
+        if sampled_heads is None:
+            ref_scores, got_scores = check_scores(scores, lay, w, b, oscale)
+            if k_q > 0:
+                check_select(idx_gpu, got_scores, ref_scores, w, k_q)
+        else:
+            ref_all = O.score(bits(lay["q_last"][b]), bits(lay["K"][b]), w.n_init, w.n_recent, scale=oscale)
+            got_all = scores.view(w.batch, w.n_q_heads, -1)[b, :, : w.E].cpu().numpy().astype(np.float64)
+            np.testing.assert_allclose(got_all, ref_all, rtol=SCORE_RTOL, atol=1e-30)
+            np.testing.assert_allclose(got_all.sum(axis=1), 1.0, atol=1e-4)
+            check_select(idx_gpu[heads], got_all[heads], ref_all[heads], w, k_q)
+            assert np.all(np.diff(idx_gpu, axis=1) > 0) and idx_gpu.min() >= w.n_init and idx_gpu.max() < w.n_init + w.E
         caches.append(list(check_compact(layer, lay, idx_gpu, w, b)))
+    guard_ok = lambda: bool((layer.Kc[:, :, st.len:].view(torch.int16) == CANARY).all()
+                            and (layer.Vc[:, :, st.len:].view(torch.int16) == CANARY).all())
+    assert guard_ok()
     # attention with the last token's query and no append, then decode steps with appends
     lse = torch.empty(w.batch, w.n_q_heads, dtype=torch.float32, device=device)
-    out = sk.decode_attn(lay["q_last"], None, None, layer, lse=lse)
+    outbuf = torch.full((w.batch + 1, w.n_q_heads, w.head_dim), 3.0, dtype=torch.bfloat16, device=device)
+    out = outbuf[: w.batch]
+    sk.decode_attn(lay["q_last"], None, None, layer, out=out, lse=lse)
     torch.cuda.synchronize()
+    again = torch.empty_like(out)
+    sk.decode_attn(lay["q_last"], None, None, layer, out=again)
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), again.view(torch.int16))   # decode repeats bit for bit
     for b in range(w.batch):
         ref, ref_lse, _ = O.decode_step(bits(lay["q_last"][b]), None, None, caches[b][0], caches[b][1], 0,
-                                        w.n_init, k_q, w.n_recent)
+                                        w.n_init, k_q, w.n_recent, scale=oscale)
         check_out(out[b], ref)
         np.testing.assert_allclose(lse[b].cpu().numpy(), ref_lse, rtol=1e-3, atol=1e-3)
     steps = [0] * w.batch
     for t in range(n_decode):
         d = synth.make_decode_inputs(w, 0, t, device)
-        out = sk.decode_attn(d["q"], d["k_new"], d["v_new"], layer)
+        sk.decode_attn(d["q"], d["k_new"], d["v_new"], layer, out=out)
         torch.cuda.synchronize()
         assert int(layer.step.item()) == t + 1
         for b in range(w.batch):
             ref, _, steps[b] = O.decode_step(bits(d["q"][b]), bits(d["k_new"][b]), bits(d["v_new"][b]),
-                                             caches[b][0], caches[b][1], steps[b], w.n_init, k_q, w.n_recent)
+                                             caches[b][0], caches[b][1], steps[b], w.n_init, k_q, w.n_recent,
+                                             scale=oscale)
             check_out(out[b], ref)
     Kc, Vc = layer.cache()
     for b in range(w.batch):   # the window rolled the same way on both sides
         assert np.array_equal(bits(Kc[b]), caches[b][0]) and np.array_equal(bits(Vc[b]), caches[b][1])
+    assert guard_ok() and bool((outbuf[w.batch] == 3.0).all())
+    assert sk.status() == 0
     sk.close()
     return lay, layer
 
@@ -155,9 +199,10 @@ def test_c1_full_config(B):
     # and 56 rows: clusters of 4
     ("C4-b1", dict(n_ctx=20000, batch=2), 1),
 ])
-def test_scaled_configs(B, name, kw, n_decode):
+@pytest.mark.parametrize("hint", [0, 1])
+def test_scaled_configs(B, name, kw, n_decode, hint):
     w = synth.workload(name).with_(n_layers=1, **kw)
-    run_pipeline(B, w, n_decode)
+    run_pipeline(B, w, n_decode, hint=hint)
 
 
 def test_strided_cache(B):
@@ -188,7 +233,33 @@ def test_degenerate_partitions(B, kw):
 def test_full_size_128k_one_layer(B):
     """C3 at budget 2048, one layer, the launch configuration the benchmark times."""
     w = synth.workload("C3-2048")
-    run_pipeline(B, w, 2)
+    run_pipeline(B, w, 2, hint=1)
+
+
+@pytest.mark.parametrize("name,hint", [
+    ("C2", 0),          # 32K context
+    ("C3-1024", 1),     # 128K, the smaller and the larger budget
+    ("C3-2048", 0),
+    ("C3-4096", 0),
+    ("C4-b1", 1),       # Qwen shape, G = 7
+    ("C5-4096", 0),     # 512K: the select step reads its unstaged slice in four rounds, the score grid has 2047 chunks
+    ("C5-4096", 1),
+    ("C5-8192", 1),
+])
+def test_every_workload_at_full_size_one_layer(B, name, hint):
+    """Each workload at its full context and budget, one layer, with and without the hint behind the score
+    rows: scores, indices, reduced cache, two decode steps, all against the oracle."""
+    w = synth.workload(name).with_(n_layers=1)
+    run_pipeline(B, w, 2, hint=hint)
+
+
+@pytest.mark.parametrize("scale", [0.05, 0.2])
+def test_softmax_scale_override(B, scale):
+    """A context created with its own softmax scale instead of 1/sqrt(d): score and decode must both use it."""
+    w = synth.workload("C2").with_(n_ctx=9001, n_layers=1, budget=516)
+    run_pipeline(B, w, 3, scale=scale)
+    w = synth.workload("C4-b1").with_(n_ctx=16500, n_layers=1, batch=2)
+    run_pipeline(B, w, 2, scale=scale, hint=1)
 
 
 def test_full_size_qwen_128k_batch4_sampled(B):
@@ -197,6 +268,7 @@ def test_full_size_qwen_128k_batch4_sampled(B):
     dev = "cuda"
     lay = synth.make_layer(w, 0, dev)
     sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    sk.set_select_hint(1)
     scores = sk.score(lay["q_last"], lay["K"], w.n_init, w.n_recent)
     layer = sk.select_compact(scores, lay["K"], lay["V"], w.n_init, w.n_recent, w.n_sel)
     d = synth.make_decode_inputs(w, 0, 0, dev)

@@ -8,6 +8,7 @@ import pytest
 import torch
 
 from oracle import sagekv_oracle as O
+from helpers import HINT_WORDS, bits, hint_of
 
 pytestmark = pytest.mark.gpu
 
@@ -16,10 +17,6 @@ pytestmark = pytest.mark.gpu
 def B():
     from paper_2503_08879_b200 import binding
     return binding
-
-
-def bits(t):
-    return t.detach().cpu().contiguous().view(torch.uint16).numpy()
 
 
 def run_select(B, rows: np.ndarray, k_q: int, S=3, R=5, H_kv=None, pad=8):
@@ -136,41 +133,6 @@ def test_cache_rows_read_from_pinned_host_memory(B):
     sk.close()
 
 
-def score_keys(x):
-    """Order-preserving 32-bit keys of float32 values (the kernels' comparison key)."""
-    u = (np.asarray(x, dtype=np.float32) + np.float32(0.0)).view(np.uint32)
-    return np.where(u & np.uint32(0x80000000), ~u, u | np.uint32(0x80000000)).astype(np.uint32)
-
-
-def hint_of(rows, E):
-    """What sagekv_score leaves behind rows of E scores: per row the 512-bin histogram of the maxima of the
-    8 x 512 groups (16 bins per octave below the row maximum) and the four tag words, as uint32 [H, 516]."""
-    H = rows.shape[0]
-    chunk = ((E + 7) // 8 + 3) // 4 * 4
-    out = np.zeros((H, 516), dtype=np.uint32)
-    for h in range(H):
-        gm = []
-        for r in range(8):
-            sl = rows[h, r * chunk:min(E, (r + 1) * chunk)]
-            n_vec = len(sl) // 4
-            g = np.full(512, -np.inf, dtype=np.float32)
-            if n_vec:
-                v = sl[:n_vec * 4].reshape(n_vec, 4).max(axis=1)
-                pad = (-n_vec) % 512
-                g = np.concatenate([v, np.full(pad, -np.inf, np.float32)]).reshape(-1, 512).max(axis=0)
-            for t in range(len(sl) - n_vec * 4):
-                g[t] = max(g[t], sl[n_vec * 4 + t])
-            gm.append(g)
-        gm = np.concatenate(gm)
-        gm = gm[gm > -np.inf]
-        kmax = int(score_keys(rows[h, :E].max()))
-        bin0 = (kmax >> 19) - 511
-        bins = np.clip((score_keys(gm) >> 19).astype(np.int64) - bin0, 0, 511)
-        out[h, :512] = np.bincount(bins, minlength=512).astype(np.uint32)
-        out[h, 512:] = [0x53414745, E, bin0, kmax]
-    return out
-
-
 @pytest.mark.parametrize("hint", ["true", "far too high", "far too low", "garbage", "wrong tag"])
 def test_histogram_behind_the_rows_is_only_a_hint(B, hint):
     """The floats behind a long score row may hold the histogram of the row's group maxima (written by
@@ -180,7 +142,12 @@ def test_histogram_behind_the_rows_is_only_a_hint(B, hint):
     rng = np.random.default_rng(31)
     rows = (rng.random((4, E), dtype=np.float32) ** 6).astype(np.float32)
     E4 = (E + 3) // 4 * 4
-    buf = torch.zeros(4, E4 + B.SKETCH_ROOM, dtype=torch.float32, device="cuda")
+    N = S + E + R + 1
+    sk = B.SageKV(4, 2, 128, 1, max_ctx=N, max_len=S + 2 * k_q + R + 1)
+    sk.set_select_hint(1)
+    stride = sk.score_stride(N, S, R)
+    assert stride >= E4 + HINT_WORDS
+    buf = torch.zeros(4, stride, dtype=torch.float32, device="cuda")
     buf[:, :E] = torch.from_numpy(rows).cuda()
     words = hint_of(rows, E)
     if hint == "far too high":
@@ -195,11 +162,9 @@ def test_histogram_behind_the_rows_is_only_a_hint(B, hint):
     elif hint == "wrong tag":
         words[:, 513] += 1
     buf[:, E4:E4 + 516] = torch.from_numpy(words.view(np.float32)).cuda()
-    N = S + E + R + 1
     g = torch.Generator(device="cuda").manual_seed(5)
     K = torch.randn(1, 2, N, 128, generator=g, device="cuda").to(torch.bfloat16)
     V = torch.randn(1, 2, N, 128, generator=g, device="cuda").to(torch.bfloat16)
-    sk = B.SageKV(4, 2, 128, 1, max_ctx=N, max_len=S + 2 * k_q + R + 1)
     before = buf.clone()
     layer = sk.select_compact(buf, K, V, S, R, 2 * k_q)
     torch.cuda.synchronize()
@@ -223,8 +188,10 @@ def test_score_leaves_the_histogram_when_the_rows_have_room(B):
     sk = B.SageKV(Hq, Hkv, 128, 1, max_ctx=N, max_len=64)
     E4 = (E + 3) // 4 * 4
     narrow = torch.zeros(Hq, E4, dtype=torch.float32, device="cuda")
-    wide = torch.full((Hq, E4 + B.SKETCH_ROOM), 7.5, dtype=torch.float32, device="cuda")
+    assert sk.score_stride(N, S, R) == E4                        # hint off: no room asked for
     sk.score(q, K, S, R, scores=narrow)
+    sk.set_select_hint(1)
+    wide = torch.full((Hq, sk.score_stride(N, S, R) + 12), 7.5, dtype=torch.float32, device="cuda")
     for _ in range(2):                                           # the second call starts from the first one's counts
         sk.score(q, K, S, R, scores=wide)
     torch.cuda.synchronize()
@@ -232,6 +199,41 @@ def test_score_leaves_the_histogram_when_the_rows_have_room(B):
     got = wide[:, E4:E4 + 516].cpu().numpy().view(np.uint32)
     assert np.array_equal(got, hint_of(wide[:, :E].cpu().numpy(), E))
     assert (wide[:, E4 + 516:] == 7.5).all() and (wide[:, E:E4] == 7.5).all()
+    sk.close()
+
+
+def test_without_the_hint_nothing_behind_the_rows_is_touched_or_believed(B):
+    """Hint off (the default): score rows may be interleaved with other data of the caller, e.g. one
+    [rows, layers, E] tensor with a row stride of layers * E.  sagekv_score must leave the neighbouring data
+    bit-exact, and sagekv_select_compact must not read it: here it holds words that look like a valid hint
+    claiming every group maximum sits at the row maximum."""
+    Hq, Hkv, N, S, R, k_q, layers = 4, 2, 20000, 4, 16, 200, 3
+    E = N - 1 - S - R
+    E4 = (E + 3) // 4 * 4
+    g = torch.Generator(device="cuda").manual_seed(19)
+    q = torch.randn(1, Hq, 128, generator=g, device="cuda").to(torch.bfloat16)
+    K = torch.randn(1, Hkv, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    V = torch.randn(1, Hkv, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    sk = B.SageKV(Hq, Hkv, 128, 1, max_ctx=N, max_len=S + 2 * k_q + R + 1)
+    tensor = torch.full((Hq, layers, E4), 3.25, dtype=torch.float32, device="cuda")
+    fake = np.zeros((Hq, HINT_WORDS), dtype=np.uint32)
+    fake[:, 511] = 4096
+    fake[:, 512:] = [0x53414745, E, 100, 0x7fffffff]
+    tensor[:, 1, :HINT_WORDS] = torch.from_numpy(fake.view(np.float32)).cuda()      # right behind layer 0's rows
+    before = tensor.clone()
+    rows = tensor[:, 0, :]                                                          # row stride layers * E4
+    B.sagekv_score(sk.ctx, q, K, N, S, R, rows, rows.stride(0))
+    torch.cuda.synchronize()
+    assert torch.equal(tensor[:, 1:].view(torch.int32), before[:, 1:].view(torch.int32))
+    assert (tensor[:, 0, E:] == 3.25).all()
+    layer = sk.new_layer(S, R, 2 * k_q)
+    B.sagekv_select_compact(sk.ctx, rows, rows.stride(0), K, V, N, S, R, 2 * k_q, layer.idx, layer.Kc, layer.Vc,
+                            layer.state)
+    torch.cuda.synchronize()
+    assert torch.equal(tensor[:, 1:].view(torch.int32), before[:, 1:].view(torch.int32))
+    got = rows[:, :E].cpu().numpy()
+    assert np.array_equal(layer.indices()[0].cpu().numpy(), O.select(got, k_q, S))
+    assert sk.status() == 0
     sk.close()
 
 

@@ -1,13 +1,16 @@
 """sagekv_score_static: the score step for callers that cannot allocate device memory (a serving
 process whose cache manager already owns the GPU's memory cannot afford the cudaMalloc, or its
 device-wide synchronisation, that creating a context costs).  The entry point keeps its scratch in a
-fixed array inside the library, so its results must equal those of sagekv_score, call after call,
-although every call reuses the same array.  Collected last on purpose."""
+fixed array inside the library, so its results must equal those of sagekv_score and lie within the score
+tolerance of the CPU oracle, call after call, although every call reuses the same array.  Collected last on
+purpose."""
 
 import numpy as np
 import pytest
 import torch
 
+from oracle import sagekv_oracle as O
+from helpers import bits
 from paper_2503_08879_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -34,6 +37,10 @@ def test_static_score_matches_context_score_on_two_calls_in_a_row():
         a, b = got[:, : w.E].cpu().numpy(), want[:, : w.E].cpu().numpy()
         np.testing.assert_allclose(a, b, rtol=SCORE_RTOL, atol=1e-30)
         np.testing.assert_allclose(a.sum(axis=1), 1.0, atol=1e-4)
+        for bi in range(w.batch):                                # and against the oracle itself, not only the sibling call
+            ref = O.score(bits(lay["q_last"][bi]), bits(lay["K"][bi]), w.n_init, w.n_recent)
+            np.testing.assert_allclose(a.reshape(w.batch, w.n_q_heads, -1)[bi].astype(np.float64), ref,
+                                       rtol=SCORE_RTOL, atol=1e-30)
         assert torch.equal(got[:, w.E:], torch.full_like(got[:, w.E:], -1.0))     # row padding untouched
         sk.close()
 
