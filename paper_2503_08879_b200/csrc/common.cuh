@@ -76,7 +76,7 @@ cudaError_t select_compact_setup();   // one-time function attributes
 
 // ---- decode attention ------------------------------------------------------
 constexpr int kDecodeWarps = 8;                                        // warps per CTA
-constexpr int kDecodeMaxCluster = 8;                                   // CTAs per cluster (the portable limit)
+constexpr int kDecodeMaxCluster = 16;                                  // CTAs per cluster (beyond 8: the non-portable sizes this part allows)
 constexpr int kDecodeMaxResident = 24;                                 // 16-row tiles (K and V) a CTA holds at once: 192 KB
 constexpr int kDecodeRoundTiles = 12;                                  // tiles per round when the partition is longer (two buffers)
 constexpr int kDecodeMaxRounds = 8;                                    // rounds before a head gets more clusters

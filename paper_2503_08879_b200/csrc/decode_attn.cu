@@ -35,20 +35,21 @@ namespace cg = cooperative_groups;
 namespace sagekv {
 
 constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kDecodeBaseCluster = 8;         // the cluster size tried first (the portable limit)
 constexpr int kTileBytes = 2 * 16 * 256;       // 16 rows of K and of V
 constexpr int kHalfBytes = 16 * 128;           // 16 rows x 64 columns: one box of the tensor copy
-constexpr int kPStride = kDecodeMaxResident * 16 + 8;   // bf16 per head row of the weight buffer: 784 bytes, 16 mod 128
+constexpr int kPStride = kDecodeMaxResident * 16 + 8;   // bf16 per head row of the weight buffer: 784 bytes, so that the 32 lanes of a fragment read hit 32 banks
 constexpr uint32_t kWaitLimit = 1u << 22;      // polls of a copy barrier before giving up (each poll already blocks for a while)
 
 struct DecShared {
   unsigned long long bar[4];                                   // K landed [buffer 0, 1], V landed [buffer 0, 1]
-  float warp_m[kDecodeWarps][kMaxGroup];                       // per round: maxima of the warps' rows
-  float warp_l[kDecodeWarps][kMaxGroup];                       // per round: sums of the warps' weights
-  float2 inbox_ml[kDecodeMaxCluster][kMaxGroup];               // [source CTA][head] (max, sum), pushed by the peers
+  unsigned long long inbox_bar;                                // completes when every CTA's share for this CTA's columns has landed
   int last;
-  int pad_[3];
-  float inbox_o[kMaxGroup * (kHeadDim + 4 * kDecodeMaxCluster)];   // [source CTA][head][my columns]; cluster size x columns <= 160
+  int pad_;
+  float warp_m[kDecodeWarps][kMaxGroup];                       // per round: maxima of the warps' rows
+  float2 inbox_ml[kDecodeMaxCluster][kMaxGroup];               // [source CTA][head] (max, sum)
   uint16_t P[kMaxGroup][kPStride];                             // softmax weights of the round, [head][row]
+  float inbox_o[(kHeadDim + 4 * kDecodeMaxCluster) * kMaxGroup];   // [source CTA][my column][head]; cluster size x columns <= 192
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -76,10 +77,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
 }
 
 // one box of a [batch, head, row, column] bf16 tensor -> shared memory; the copy reads this GPU's memory only
-__device__ __forceinline__ void tensor_copy_4d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, int w, uint32_t bar) {
+// (the cache rows are read once per call: they are marked evict-first in L2, so that the small operands every
+// call reads after its dependency wait, q and the step counter, tend to stay there)
+__device__ __forceinline__ void tensor_copy_4d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, int w, uint32_t bar,
+                                               uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar), "l"(policy)
       : "memory");
 }
 
@@ -115,8 +119,8 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   const int ci = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;    // ci: CTA index within the head
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;
+  const int h0 = 2 * c, h1 = 2 * c + 1;                           // the two heads a lane's accumulators belong to
   const bool append = p.k_new != nullptr;
-  cluster.barrier_arrive();                              // waited for just before the first push into a peer
 
   // tiles of this CTA: an even deal of the head's n_tiles over the gridDim.x CTAs, contiguous ranges
   const int n_tiles = (p.L + 15) >> 4;
@@ -125,18 +129,29 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   const int my_tiles = base_n + (ci < rem ? 1 : 0);
   const int n_rounds = kMulti ? (my_tiles + kDecodeRoundTiles - 1) / kDecodeRoundTiles : 1;
 
+  // columns each CTA of the cluster finishes: a multiple of 4, the last CTA may get fewer
+  const int cols = ((kHeadDim + cs - 1) / cs + 3) & ~3;
+  const int my_cols = max(0, min(cols, kHeadDim - rank * cols));   // (cluster sizes that do not divide 128 leave the last CTAs fewer, or none)
+  const int n_pairs = (p.G + 1) >> 1;                             // head pairs in use
+
   const uint32_t bar0 = smem_u32(&sh.bar[0]);
   if (tid == 0) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) mbar_init(bar0 + 8 * i, 1);
+    mbar_init(smem_u32(&sh.inbox_bar), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    // from every CTA of the cluster: 8 bytes per (own column, head pair in use) and 64 bytes of (max, sum) pairs
+    mbar_expect_tx(smem_u32(&sh.inbox_bar), (uint32_t)(cs * (my_cols * n_pairs * 8 + 64)));
   }
   __syncthreads();
+  cluster.barrier_arrive();                              // waited for just before the first store into a peer: its barrier is set up
 
   // the copies of one round, K boxes first: lane i of warp 0 issues requests i, i + 32, ...
+  uint64_t stream_policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
   auto issue_round = [&](int r) {
     const int buf = kMulti ? (r & 1) : 0;
     const int t0 = kMulti ? r * kDecodeRoundTiles : 0;
@@ -152,7 +167,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       const int o2 = is_v ? op - nt * 2 : op;
       const int t = o2 >> 1, half = o2 & 1;
       const uint32_t dst = stage + (uint32_t)((buf * kDecodeRoundTiles + t) * kTileBytes + (is_v ? 2 : 0) * kHalfBytes + half * kHalfBytes);
-      tensor_copy_4d(dst, is_v ? &map_v : &map_k, half * 64, (first_tile + t0 + t) << 4, kvh, b, is_v ? vbar : kbar);
+      tensor_copy_4d(dst, is_v ? &map_v : &map_k, half * 64, (first_tile + t0 + t) << 4, kvh, b, is_v ? vbar : kbar, stream_policy);
     }
   };
 
@@ -169,20 +184,44 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     issue_round(0);
     if (kMulti && n_rounds > 1) issue_round(1);
   }
+
+  // Everything that does not depend on the predecessor's results is worked out before the wait: which of this
+  // lane's score elements are visible to their heads (sink, own segment, window; bit 4i + e for tile i, element
+  // e), and where the finishing stage finds its operands.
+  const int win_lo = p.S + p.n_sel;
+  const int seg0_lo = p.S + h0 * p.k_q, seg0_hi = seg0_lo + p.k_q, seg1_lo = seg0_hi, seg1_hi = seg1_lo + p.k_q;
+  auto visibility = [&](int t0) {
+    uint32_t bits = 0;
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      const int ra = ((first_tile + t0 + warp + kDecodeWarps * i) << 4) + g, rb = ra + 8;
+      const bool va = ra < p.L, vb = rb < p.L;
+      const bool sa = ra < p.S || ra >= win_lo, sb = rb < p.S || rb >= win_lo;
+      bits |= (va && h0 < p.G && (sa || (ra >= seg0_lo && ra < seg0_hi)) ? 1u : 0u) << (4 * i);
+      bits |= (va && h1 < p.G && (sa || (ra >= seg1_lo && ra < seg1_hi)) ? 2u : 0u) << (4 * i);
+      bits |= (vb && h0 < p.G && (sb || (rb >= seg0_lo && rb < seg0_hi)) ? 4u : 0u) << (4 * i);
+      bits |= (vb && h1 < p.G && (sb || (rb >= seg1_lo && rb < seg1_hi)) ? 8u : 0u) << (4 * i);
+    }
+    return bits;
+  };
+  uint32_t vis = visibility(0);
+  // finishing stage: four lanes per output value (own column lc, head fh), lane q of them holds the shares of
+  // source CTAs q and q + 4
+  const int fin_items = my_cols * p.G, fin_q = tid & 3;
+  const int mi = lane >> 3, l8 = lane & 7;
+  const int arow = (mi & 1) * 8 + l8;                     // ldmatrix row of this lane for K fragments
+  const int vrow = (mi >> 1) * 8 + l8, vpiece = 2 * warp + (mi & 1);
+  const uint32_t v_lane_off = 2 * kHalfBytes + tile_offset(vrow, vpiece);
+  const uint16_t *prow = &sh.P[g][2 * c];
+
   if (p.pdl_mode >= 2) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
 
-  int step = 0, slot = -1;
-  if (append) {
-    step = *reinterpret_cast<const volatile int32_t *>(p.d_step);
-    slot = p.S + p.n_sel + step % p.ring_len;
-  }
-  const uint16_t *kn = append ? p.k_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
-  const uint16_t *vn = append ? p.v_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
-  const int slot_tile = append ? (slot >> 4) - first_tile : -1;   // CTA-local tile of the replaced row (if 0 <= . < my_tiles)
-
+  // What the predecessor may have written is read now, all requests issued back to back (query first: the first
+  // product needs it; the step counter last: only the patch of the replaced row needs it), so the round trips to
+  // L2 overlap instead of queueing behind one another.
   // B fragments of Q^T for the first product: lane (g, c) holds head g's dims 16ks + 2c, +1 and 16ks + 8 + 2c, +1
   uint32_t qb[8][2];
 #pragma unroll
@@ -191,21 +230,30 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     const uint16_t *qrow = p.q + ((int64_t)b * p.H_q + kvh * p.G + g) * kHeadDim;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
-      qb[ks][0] = *reinterpret_cast<const uint32_t *>(qrow + 16 * ks + 2 * c);
-      qb[ks][1] = *reinterpret_cast<const uint32_t *>(qrow + 16 * ks + 8 + 2 * c);
+      asm volatile("ld.global.b32 %0, [%1];" : "=r"(qb[ks][0]) : "l"(qrow + 16 * ks + 2 * c));
+      asm volatile("ld.global.b32 %0, [%1];" : "=r"(qb[ks][1]) : "l"(qrow + 16 * ks + 8 + 2 * c));
     }
   }
-  // rows heads 2c and 2c+1 may look at: sink, own segment, the window
-  const int h0 = 2 * c, h1 = 2 * c + 1;
-  const int win_lo = p.S + p.n_sel;
-  const int seg0_lo = p.S + h0 * p.k_q, seg0_hi = seg0_lo + p.k_q, seg1_lo = seg0_hi, seg1_hi = seg1_lo + p.k_q;
+  const uint16_t *kn = append ? p.k_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
+  const uint16_t *vn = append ? p.v_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
+  uint4 new_row = make_uint4(0u, 0u, 0u, 0u);            // lanes 0-15: 16 bytes of k_new, lanes 16-31: of v_new
+  int step = 0, my_ticket = -1;
+  if (append) {
+    new_row = ld_v4((lane < 16 ? kn : vn) + (lane & 15) * 8);
+    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(step) : "l"(p.d_step));
+    // One ticket per CTA, taken once the counter has been read (release: the load is ordered before it), by a
+    // thread of the warp with the fewest tiles.  The answer is looked at only when the CTA is done, long after
+    // it has come back.
+    if (tid == kDecodeThreads - 1)
+      asm volatile("atom.add.release.gpu.global.s32 %0, [%1], 1;" : "=r"(my_ticket) : "l"(p.tickets + p.B * p.H_kv) : "memory");
+  }
 
   float M0 = -INFINITY, M1 = -INFINITY;   // running maxima of heads 2c, 2c+1 over the CTA's rows (log2 units)
   float L0 = 0.f, L1 = 0.f;               // running sums of the (bf16-rounded) weights over the CTA's rows
   float acc[4] = {0.f, 0.f, 0.f, 0.f};    // O^T: (col 16w+g, h0) (col 16w+g, h1) (col 16w+g+8, h0) (col 16w+g+8, h1)
   bool dead = false;                      // a copy never arrived: the CTA contributes nothing
+  int slot = -1, slot_tile = -1;          // the replaced window row and its CTA-local tile, worked out at first use
 
-  const int mi = lane >> 3, l8 = lane & 7;
   for (int r = 0; r < n_rounds; ++r) {
     const int buf = kMulti ? (r & 1) : 0;
     const uint32_t par = kMulti ? (uint32_t)((r >> 1) & 1) : 0u;
@@ -213,21 +261,25 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     const int nt = kMulti ? min(kDecodeRoundTiles, my_tiles - t0) : my_tiles;
     const uint32_t kbar = bar0 + 8 * buf, vbar = bar0 + 16 + 8 * buf;
     const uint32_t buf_base = stage + (uint32_t)(buf * kDecodeRoundTiles * kTileBytes);
+    if (kMulti && r > 0) vis = visibility(t0);
     if (nt > 0 && !dead && !mbar_wait(kbar, par)) dead = true;
 
     // the staged copy of the replaced row is stale: the warp that works on its tile patches K and V
+    if (append && r == 0) {
+      slot = p.S + p.n_sel + step % p.ring_len;
+      slot_tile = (slot >> 4) - first_tile;
+    }
     const int st = slot_tile - t0;                       // tile of this round holding the replaced row, if in [0, nt)
     if (append && st >= 0 && st < nt && (st & (kDecodeWarps - 1)) == warp && !dead) {
       if (!mbar_wait(vbar, par)) dead = true;
       if (!dead) {
         const int row = slot & 15, piece = lane & 15;
-        const uint4 nv = ld_v4((lane < 16 ? kn : vn) + piece * 8);
         const uint32_t dst = buf_base + (uint32_t)(st * kTileBytes + (lane < 16 ? 0 : 2 * kHalfBytes)) + tile_offset(row, piece);
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(nv.x), "r"(nv.y), "r"(nv.z), "r"(nv.w) : "memory");
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(new_row.x), "r"(new_row.y), "r"(new_row.z), "r"(new_row.w) : "memory");
         if (SAGEKV_OK_INDEX(p.status, slot >= 0 && slot < p.L)) {
           uint16_t *gdst = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
                            (int64_t)slot * p.cs.token_stride + piece * 8;
-          st_v4(gdst, nv);
+          st_v4(gdst, new_row);
         }
       }
       __syncwarp();
@@ -235,35 +287,49 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     dead = __any_sync(0xffffffffu, dead);
 
     // ---- S = K Q^T: this warp's tiles of the round are warp, warp + 8, warp + 16 ----
+    // An mma takes far longer than its issue slot, so the work is laid out as many short independent chains:
+    // per tile four accumulators (k-steps j and j + 4), the fragments of all tiles requested ahead of the mmas.
     float sv[3][4];
     float wm0 = -INFINITY, wm1 = -INFINITY;
+    {
+      float ch[3][4][4];
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {
-      const int t = warp + kDecodeWarps * i;
-      sv[i][0] = sv[i][1] = sv[i][2] = sv[i][3] = -INFINITY;
-      if (t < nt && !dead) {
-        const uint32_t tb = buf_base + (uint32_t)(t * kTileBytes);
-        float e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f, o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;   // two chains
-        const int arow = (mi & 1) * 8 + l8;
+      for (int i = 0; i < 3; ++i)
 #pragma unroll
-        for (int ks = 0; ks < 8; ks += 2) {
-          uint32_t a0, a1, a2, a3;
-          ldmatrix_x4(tb + tile_offset(arow, 2 * ks + (mi >> 1)), a0, a1, a2, a3);
-          mma_bf16_16816(e0, e1, e2, e3, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
-          ldmatrix_x4(tb + tile_offset(arow, 2 * ks + 2 + (mi >> 1)), a0, a1, a2, a3);
-          mma_bf16_16816(o0, o1, o2, o3, a0, a1, a2, a3, qb[ks + 1][0], qb[ks + 1][1]);
+        for (int j = 0; j < 4; ++j) ch[i][j][0] = ch[i][j][1] = ch[i][j][2] = ch[i][j][3] = 0.f;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {             // k-steps 0..3, then 4..7: twelve independent mmas each time
+        uint32_t fa[3][4][4];
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+          const int t = warp + kDecodeWarps * i;
+          if (t < nt && !dead) {
+            const uint32_t tb = buf_base + (uint32_t)(t * kTileBytes);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              ldmatrix_x4(tb + tile_offset(arow, 2 * (4 * half + j) + (mi >> 1)), fa[i][j][0], fa[i][j][1], fa[i][j][2], fa[i][j][3]);
+          }
         }
-        const int ra = ((first_tile + t0 + t) << 4) + g, rb = ra + 8;
-        const bool va = ra < p.L, vb = rb < p.L;
-        const bool sa = ra < p.S || ra >= win_lo, sb = rb < p.S || rb >= win_lo;
-        const bool a_h0 = va && h0 < p.G && (sa || (ra >= seg0_lo && ra < seg0_hi));
-        const bool a_h1 = va && h1 < p.G && (sa || (ra >= seg1_lo && ra < seg1_hi));
-        const bool b_h0 = vb && h0 < p.G && (sb || (rb >= seg0_lo && rb < seg0_hi));
-        const bool b_h1 = vb && h1 < p.G && (sb || (rb >= seg1_lo && rb < seg1_hi));
-        sv[i][0] = a_h0 ? (e0 + o0) * p.scale_log2 : -INFINITY;
-        sv[i][1] = a_h1 ? (e1 + o1) * p.scale_log2 : -INFINITY;
-        sv[i][2] = b_h0 ? (e2 + o2) * p.scale_log2 : -INFINITY;
-        sv[i][3] = b_h1 ? (e3 + o3) * p.scale_log2 : -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+          const int t = warp + kDecodeWarps * i;
+          if (t < nt && !dead) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              mma_bf16_16816(ch[i][j][0], ch[i][j][1], ch[i][j][2], ch[i][j][3], fa[i][j][0], fa[i][j][1], fa[i][j][2], fa[i][j][3],
+                             qb[4 * half + j][0], qb[4 * half + j][1]);
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 3; ++i) {
+        const int t = warp + kDecodeWarps * i;
+        const uint32_t vb4 = (t < nt && !dead) ? (vis >> (4 * i)) & 15u : 0u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float x = (ch[i][0][e] + ch[i][1][e]) + (ch[i][2][e] + ch[i][3][e]);
+          sv[i][e] = ((vb4 >> e) & 1u) ? x * p.scale_log2 : -INFINITY;
+        }
         wm0 = fmaxf(wm0, fmaxf(sv[i][0], sv[i][2]));
         wm1 = fmaxf(wm1, fmaxf(sv[i][1], sv[i][3]));
       }
@@ -290,96 +356,123 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       acc[0] *= f0; acc[2] *= f0; acc[1] *= f1; acc[3] *= f1;
     }
     M0 = N0; M1 = N1;
-    // the weights enter the second product as bf16; sum the rounded values so numerator and denominator agree
-    float ws0 = 0.f, ws1 = 0.f;
+    // the weights enter the second product as bf16
 #pragma unroll
     for (int i = 0; i < 3; ++i) {
       const int t = warp + kDecodeWarps * i;
       if (t < nt) {
         const uint32_t p0 = pack_bf16x2(fast_exp2(sv[i][0] - s0), fast_exp2(sv[i][2] - s0));   // head h0: rows g, g + 8
         const uint32_t p1 = pack_bf16x2(fast_exp2(sv[i][1] - s1), fast_exp2(sv[i][3] - s1));   // head h1
-        ws0 += __uint_as_float(p0 << 16) + __uint_as_float(p0 & 0xffff0000u);
-        ws1 += __uint_as_float(p1 << 16) + __uint_as_float(p1 & 0xffff0000u);
         uint16_t *w0 = &sh.P[h0][t * 16 + g], *w1 = &sh.P[h1][t * 16 + g];
         w0[0] = (uint16_t)(p0 & 0xffffu); w0[8] = (uint16_t)(p0 >> 16);
         w1[0] = (uint16_t)(p1 & 0xffffu); w1[8] = (uint16_t)(p1 >> 16);
       }
     }
-#pragma unroll
-    for (int off = 4; off < 32; off <<= 1) {
-      ws0 += __shfl_xor_sync(0xffffffffu, ws0, off);
-      ws1 += __shfl_xor_sync(0xffffffffu, ws1, off);
-    }
-    if (g == 0) { sh.warp_l[warp][h0] = ws0; sh.warp_l[warp][h1] = ws1; }
     if (nt > 0 && !dead && !mbar_wait(vbar, par)) dead = true;
     dead = __any_sync(0xffffffffu, dead);
-    __syncthreads();   // B: weights and sums of the round are in shared memory (and a patched V row is visible)
-#pragma unroll
-    for (int w = 0; w < kDecodeWarps; ++w) { L0 += sh.warp_l[w][h0]; L1 += sh.warp_l[w][h1]; }
+    __syncthreads();   // B: the weights of the round are in shared memory (and a patched V row is visible)
 
     // ---- O^T += V^T P over all rows of the round, columns 16*warp .. 16*warp + 15 ----
+    // Eight tiles per step, each on an accumulator chain of its own; their V fragments and weights are all
+    // requested before the mmas.  The same weights times a fragment of ones give the sums of the rounded
+    // weights per head, in every lane, in the accumulator layout (so numerator and denominator agree, and no
+    // shuffle or shared-memory exchange is needed for them).
     if (!dead) {
-      float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;      // second chain (odd tiles)
-      const int vrow = (mi >> 1) * 8 + l8, vpiece = 2 * warp + (mi & 1);
-      const uint32_t voff = 2 * kHalfBytes + tile_offset(vrow, vpiece);
-      const uint16_t *prow = &sh.P[g][2 * c];
-      int t = 0;
-      for (; t + 1 < nt; t += 2) {
-        uint32_t a0, a1, a2, a3;
-        ldmatrix_x4_trans(buf_base + (uint32_t)(t * kTileBytes) + voff, a0, a1, a2, a3);
-        mma_bf16_16816(acc[0], acc[1], acc[2], acc[3], a0, a1, a2, a3,
-                       *reinterpret_cast<const uint32_t *>(prow + t * 16), *reinterpret_cast<const uint32_t *>(prow + t * 16 + 8));
-        ldmatrix_x4_trans(buf_base + (uint32_t)((t + 1) * kTileBytes) + voff, a0, a1, a2, a3);
-        mma_bf16_16816(x0, x1, x2, x3, a0, a1, a2, a3,
-                       *reinterpret_cast<const uint32_t *>(prow + t * 16 + 16), *reinterpret_cast<const uint32_t *>(prow + t * 16 + 24));
+      float xc[7][4], lc0[4] = {0.f, 0.f, 0.f, 0.f}, lc1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int u = 0; u < 7; ++u) xc[u][0] = xc[u][1] = xc[u][2] = xc[u][3] = 0.f;
+      const uint32_t vbase = buf_base + v_lane_off;
+      const uint32_t ones = 0x3f803f80u;
+      for (int t8 = 0; t8 < nt; t8 += 8) {
+        uint32_t va[8][4], pb[8][2];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (t8 + u < nt) {
+            ldmatrix_x4_trans(vbase + (uint32_t)((t8 + u) * kTileBytes), va[u][0], va[u][1], va[u][2], va[u][3]);
+            pb[u][0] = *reinterpret_cast<const uint32_t *>(prow + (t8 + u) * 16);
+            pb[u][1] = *reinterpret_cast<const uint32_t *>(prow + (t8 + u) * 16 + 8);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (t8 + u < nt) {
+            if (u == 0) mma_bf16_16816(acc[0], acc[1], acc[2], acc[3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
+            else mma_bf16_16816(xc[u - 1][0], xc[u - 1][1], xc[u - 1][2], xc[u - 1][3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
+            if (u & 1) mma_bf16_16816(lc1[0], lc1[1], lc1[2], lc1[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
+            else mma_bf16_16816(lc0[0], lc0[1], lc0[2], lc0[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
+          }
+        }
       }
-      if (t < nt) {
-        uint32_t a0, a1, a2, a3;
-        ldmatrix_x4_trans(buf_base + (uint32_t)(t * kTileBytes) + voff, a0, a1, a2, a3);
-        mma_bf16_16816(acc[0], acc[1], acc[2], acc[3], a0, a1, a2, a3,
-                       *reinterpret_cast<const uint32_t *>(prow + t * 16), *reinterpret_cast<const uint32_t *>(prow + t * 16 + 8));
-      }
-      acc[0] += x0; acc[1] += x1; acc[2] += x2; acc[3] += x3;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        acc[e] += ((xc[0][e] + xc[1][e]) + (xc[2][e] + xc[3][e])) + ((xc[4][e] + xc[5][e]) + xc[6][e]);
+      L0 += lc0[0] + lc1[0];
+      L1 += lc0[1] + lc1[1];
     }
   }
   if (dead && tid == 0) atomicOr(p.status, kStatusWaitTimeout);
 
   // ---- merge the CTAs of the cluster: the owner of a column slice receives it from every CTA ----
-  const int cols = ((kHeadDim + cs - 1) / cs + 3) & ~3;   // columns each CTA finishes: a multiple of 4, the last CTA may get fewer
-  cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs
+  // Every warp sends its 16 columns straight from registers into the owners' inboxes with asynchronous stores
+  // that count their bytes on the owner's barrier: data and signal travel together and nobody waits for an
+  // acknowledgement or for a cluster-wide barrier; a CTA only waits for its own inbox to fill.
+  cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs, its barrier is set up
   {
-    const int col_a = 16 * warp + g, col_b = col_a + 8;
-    const int own_a = col_a / cols, own_b = col_b / cols;
-    float *ia = cluster.map_shared_rank(sh.inbox_o, own_a) + (rank * kMaxGroup) * cols + (col_a - own_a * cols);
-    float *ib = cluster.map_shared_rank(sh.inbox_o, own_b) + (rank * kMaxGroup) * cols + (col_b - own_b * cols);
-    if (h0 < p.G) { ia[h0 * cols] = acc[0]; ib[h0 * cols] = acc[2]; }
-    if (h1 < p.G) { ia[h1 * cols] = acc[1]; ib[h1 * cols] = acc[3]; }
-    if (warp == 0 && g < cs) {                           // lane (g, c) tells CTA g the (max, sum) of heads 2c and 2c+1
-      float2 *ml = &cluster.map_shared_rank(&sh.inbox_ml[0][0], g)[rank * kMaxGroup];
-      ml[h0] = make_float2(M0, L0);
-      ml[h1] = make_float2(M1, L1);
+    auto send2 = [&](uint32_t local_addr, int dst_rank, float x, float y) {
+      uint32_t addr, rbar;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(addr) : "r"(local_addr), "r"(dst_rank));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_u32(&sh.inbox_bar)), "r"(dst_rank));
+      asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+                   ::"r"(addr), "f"(x), "f"(y), "r"(rbar) : "memory");
+    };
+    const uint32_t inbox = smem_u32(sh.inbox_o);
+    if (h0 < p.G) {
+      const int col_a = 16 * warp + g, col_b = col_a + 8;
+      const int own_a = col_a / cols, own_b = col_b / cols;
+      send2(inbox + (uint32_t)(((rank * cols + (col_a - own_a * cols)) * kMaxGroup + h0) * 4), own_a, acc[0], acc[1]);
+      send2(inbox + (uint32_t)(((rank * cols + (col_b - own_b * cols)) * kMaxGroup + h0) * 4), own_b, acc[2], acc[3]);
+    }
+    if (warp < 2 && 8 * warp + g < cs) {                 // lane (g, c) of warps 0, 1 tells CTA 8*warp + g the (max, sum) of heads 2c and 2c+1
+      const uint32_t mlbox = smem_u32(&sh.inbox_ml[rank][0]);
+      send2(mlbox + (uint32_t)h0 * 8u, 8 * warp + g, M0, L0);
+      send2(mlbox + (uint32_t)h1 * 8u, 8 * warp + g, M1, L1);
     }
   }
-  cluster.sync();   // all pushes have landed; no shared memory of a peer is touched after this point
+  if (!mbar_wait(smem_u32(&sh.inbox_bar), 0u) && tid == 0) atomicOr(p.status, kStatusWaitTimeout);
 
-  // ---- finish columns [rank*cols, (rank+1)*cols) of every head from the inbox ----
+  // ---- finish columns [rank*cols, rank*cols + my_cols) of every head from the inbox ----
   const int bk = b * p.H_kv + kvh;
   const int n_clusters = (int)gridDim.x / cs, cl = ci / cs;
   float *part = p.partials + ((int64_t)bk * n_clusters + cl) * kPartialStride;
-  for (int item = tid; item < p.G * cols; item += kDecodeThreads) {
-    const int h = item / cols, lc = item - h * cols, col = rank * cols + lc;
-    if (col >= kHeadDim) continue;
-    float M = -INFINITY;
-    for (int s = 0; s < cs; ++s) M = fmaxf(M, sh.inbox_ml[s][h].x);
-    float o = 0.f, l = 0.f;
-    for (int s = 0; s < cs; ++s) {
-      const float2 ml = sh.inbox_ml[s][h];
-      const float wgt = M == -INFINITY ? 0.f : fast_exp2(ml.x - M);
-      o += sh.inbox_o[(s * kMaxGroup + h) * cols + lc] * wgt;
-      l += ml.y * wgt;
+  for (int base = 0; base < fin_items; base += kDecodeThreads / 4) {   // the same trip count in every lane: shuffles inside
+    const int item = min(base + (tid >> 2), fin_items - 1);
+    const bool real = base + (tid >> 2) < fin_items;
+    const int lc = item / p.G, h = item - lc * p.G, col = rank * cols + lc;
+    float2 ml[4];
+    float ov[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {                        // this lane's source CTAs: fin_q, fin_q + 4, ...
+      const int src = fin_q + 4 * j;
+      ml[j] = src < cs ? sh.inbox_ml[src][h] : make_float2(-INFINITY, 0.f);
+      ov[j] = src < cs ? sh.inbox_o[(src * cols + lc) * kMaxGroup + h] : 0.f;
     }
+    float M = fmaxf(fmaxf(ml[0].x, ml[1].x), fmaxf(ml[2].x, ml[3].x));
+    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));
+    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
+    float o = 0.f, l = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float wgt = M == -INFINITY ? 0.f : fast_exp2(ml[j].x - M);
+      o += ov[j] * wgt;
+      l += ml[j].y * wgt;
+    }
+    o += __shfl_xor_sync(0xffffffffu, o, 1); l += __shfl_xor_sync(0xffffffffu, l, 1);
+    o += __shfl_xor_sync(0xffffffffu, o, 2); l += __shfl_xor_sync(0xffffffffu, l, 2);
+    if (fin_q != 0 || !real) continue;
     if (n_clusters == 1) {
-      const float outv = l > 0.f ? o / l : 0.f;
+      float inv;                                           // the output is rounded to bf16: an approximate reciprocal is ample
+      asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(l));
+      const float outv = l > 0.f ? o * inv : 0.f;
       p.out[((int64_t)b * p.H_q + kvh * p.G + h) * kHeadDim + col] = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
       if (p.lse != nullptr && col == 0)
         p.lse[(int64_t)b * p.H_q + kvh * p.G + h] = l > 0.f ? (M + log2f(l)) * kLn2 : -INFINITY;
@@ -392,15 +485,13 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     }
   }
 
-  bool head_done = rank == 0;                            // one CTA per head reports completion
   if (n_clusters > 1) {
     // ---- several clusters per head: the last CTA to arrive merges the cluster results ----
     __threadfence();
     __syncthreads();
     if (tid == 0) sh.last = atomicAdd(&p.tickets[bk], 1) == (int)gridDim.x - 1;
     __syncthreads();
-    head_done = sh.last != 0;
-    if (head_done) {
+    if (sh.last != 0) {
       __threadfence();
       const float *all = p.partials + (int64_t)bk * n_clusters * kPartialStride;
       for (int item = tid; item < p.G * kHeadDim; item += kDecodeThreads) {
@@ -422,14 +513,10 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       if (tid == 0) p.tickets[bk] = 0;
     }
   }
-  // ---- the last KV head to finish advances the step counter ----
-  // (every CTA read the counter before it got here, so the update cannot reach a reader of this launch)
-  if (append && head_done && tid == 0) {
-    const int n_heads = p.B * p.H_kv;
-    if (atomicAdd(&p.tickets[n_heads], 1) == n_heads - 1) {
-      p.tickets[n_heads] = 0;
-      *p.d_step = step + 1;
-    }
+  // ---- the step counter: whoever took the last ticket of the launch knows that every CTA has read it ----
+  if (append && tid == kDecodeThreads - 1 && my_ticket == (int)(gridDim.x * gridDim.y * gridDim.z) - 1) {
+    p.tickets[p.B * p.H_kv] = 0;
+    *p.d_step = step + 1;
   }
 }
 
@@ -447,9 +534,12 @@ cudaError_t decode_setup(DeviceInfo *dev) {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  if (e != cudaSuccess) return e;
   for (int c = 0; c <= kDecodeMaxCluster; ++c) dev->cluster_cap[c] = 0;
   for (int c = 4; c <= kDecodeMaxCluster; ++c) {
-    if (c == 7) continue;                                // never chosen (no more of them fit than of 8)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(c * 64), 1, 1);
     cfg.blockDim = dim3(kDecodeThreads, 1, 1);
@@ -479,21 +569,21 @@ cudaError_t decode_setup(DeviceInfo *dev) {
 void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, int *cs, int *resident_tiles, int *smem_bytes) {
   const int n_tiles = (L + 15) / 16;
   int c = 1;
-  while (c < kDecodeMaxCluster && c * 2 <= n_tiles) c <<= 1;                     // cluster size 1, 2, 4 or 8
+  while (c < kDecodeBaseCluster && c * 2 <= n_tiles) c <<= 1;                     // cluster size 1, 2, 4 or 8
   const int per_cluster_cta = kDecodeRoundTiles * kDecodeMaxRounds;              // most tiles a CTA goes through
   const int nc = (n_tiles + c * per_cluster_cta - 1) / (c * per_cluster_cta);
   int per_cta = (n_tiles + c * nc - 1) / (c * nc);                               // most tiles a CTA gets
-  if (dev != nullptr && c == kDecodeMaxCluster && nc == 1 && per_cta > 12 && heads > dev->cluster_cap[c] &&
+  if (dev != nullptr && c == kDecodeBaseCluster && nc == 1 && per_cta > 12 && heads > dev->cluster_cap[c] &&
       dev->cluster_cap[c] > 0) {
     float best = 0.f;
     int best_c = c;
-    for (int cand = kDecodeMaxCluster; cand >= 4; --cand) {
+    for (int cand = kDecodeBaseCluster; cand >= 4; --cand) {
       const int cap = dev->cluster_cap[cand];
       if (cap <= 0 || n_tiles > cand * per_cluster_cta) continue;
       const int per = (n_tiles + cand - 1) / cand;
       const int rounds = per <= kDecodeMaxResident ? 1 : (per + kDecodeRoundTiles - 1) / kDecodeRoundTiles;
       const float cost = (float)((heads + cap - 1) / cap) * (4.5f + 0.1f * (float)per + (float)(rounds - 1));
-      if (cand == kDecodeMaxCluster || cost < best) { best = cost; best_c = cand; }
+      if (cand == kDecodeBaseCluster || cost < best) { best = cost; best_c = cand; }
     }
     c = best_c;
     per_cta = (n_tiles + c - 1) / c;
