@@ -48,6 +48,7 @@ cudaError_t device_setup(int dev, const DeviceInfo **out) {
   std::lock_guard<std::mutex> lock(g_dev_mutex);
   DeviceInfo &d = g_dev[dev];
   if (!d.ready) {
+    d.device = dev;
     cudaError_t e = cudaDeviceGetAttribute(&d.n_sm, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess) e = select_compact_setup();
     if (e == cudaSuccess) e = decode_setup(&d);

@@ -75,8 +75,11 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
 cudaError_t select_compact_setup();   // one-time function attributes
 
 // ---- decode attention ------------------------------------------------------
-constexpr int kDecodeWarps = 8;                                        // warps per CTA
-constexpr int kDecodeMaxCluster = 16;                                  // CTAs per cluster (beyond 8: the non-portable sizes this part allows)
+#if !defined(SAGEKV_DECODE_WARPS)
+#define SAGEKV_DECODE_WARPS 8
+#endif
+constexpr int kDecodeWarps = SAGEKV_DECODE_WARPS;                      // warps per CTA: 8, or 16 (two row halves in the second product)
+constexpr int kDecodeMaxCluster = 8;                                   // CTAs per cluster (the portable limit)
 constexpr int kDecodeMaxResident = 24;                                 // 16-row tiles (K and V) a CTA holds at once: 192 KB
 constexpr int kDecodeRoundTiles = 12;                                  // tiles per round when the partition is longer (two buffers)
 constexpr int kDecodeMaxRounds = 8;                                    // rounds before a head gets more clusters
@@ -101,8 +104,8 @@ struct DecodeParams {
 
 // What the one-time set-up of a device leaves behind (function attributes are set as a side effect).
 struct DeviceInfo {
+  int device;
   int n_sm;
-  int cluster_cap[kDecodeMaxCluster + 1];   // decode clusters of each size that can be resident at once
   bool ready;
 };
 cudaError_t launch_decode(const DecodeParams &p, const DeviceInfo &dev, cudaStream_t stream);

@@ -22,7 +22,8 @@
 // The staged copy of the window row that the new token replaces is overwritten in shared memory from
 // k_new / v_new once it has landed, and the CTA owning that row stores the new token into the cache.
 // Every wait on a copy barrier is bounded: a wait that runs out sets kStatusWaitTimeout in the context's status
-// word and the CTA goes on as if it had no rows, so every block and cluster barrier is still reached.
+// word and the CTA runs on with whatever its shared memory holds, so every block and cluster barrier is still
+// reached and the kernel ends; the output of such a launch is meaningless and the status word says so.
 #include <cooperative_groups.h>
 #include <cuda.h>
 
@@ -35,21 +36,25 @@ namespace cg = cooperative_groups;
 namespace sagekv {
 
 constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kDecodeBaseCluster = 8;         // the cluster size tried first (the portable limit)
+constexpr int kDecodeBaseCluster = 8;          // the cluster size tried first (the portable limit)
 constexpr int kTileBytes = 2 * 16 * 256;       // 16 rows of K and of V
 constexpr int kHalfBytes = 16 * 128;           // 16 rows x 64 columns: one box of the tensor copy
-constexpr int kPStride = kDecodeMaxResident * 16 + 8;   // bf16 per head row of the weight buffer: 784 bytes, so that the 32 lanes of a fragment read hit 32 banks
+constexpr int kPHeadWords = 12;                // 32-bit words per (tile, head) of the weight buffer: 8 used, 4 spread the banks
+constexpr int kPTileWords = kMaxGroup * kPHeadWords;
+constexpr int kIssueWarp = kDecodeWarps - 1;   // the warp with the fewest tiles issues the copies
+constexpr int kRowHalves = kDecodeWarps / 8;   // the second product splits columns eight ways and rows this many ways
+constexpr int kQkTiles = (kDecodeMaxResident + kDecodeWarps - 1) / kDecodeWarps;   // tiles of a round a warp may get in the first product
 constexpr uint32_t kWaitLimit = 1u << 22;      // polls of a copy barrier before giving up (each poll already blocks for a while)
 
 struct DecShared {
   unsigned long long bar[4];                                   // K landed [buffer 0, 1], V landed [buffer 0, 1]
-  unsigned long long inbox_bar;                                // completes when every CTA's share for this CTA's columns has landed
+  unsigned long long inbox_bar;                                // every CTA's share for this CTA's columns has landed
   int last;
   int pad_;
   float warp_m[kDecodeWarps][kMaxGroup];                       // per round: maxima of the warps' rows
-  float2 inbox_ml[kDecodeMaxCluster][kMaxGroup];               // [source CTA][head] (max, sum)
-  uint16_t P[kMaxGroup][kPStride];                             // softmax weights of the round, [head][row]
-  float inbox_o[(kHeadDim + 4 * kDecodeMaxCluster) * kMaxGroup];   // [source CTA][my column][head]; cluster size x columns <= 192
+  float2 inbox_ml[kRowHalves * kDecodeMaxCluster][kMaxGroup];  // [source CTA, row half][head] (max, sum)
+  uint32_t P[kDecodeMaxResident * kPTileWords];                // softmax weights of the round: [tile][head][row pair g: rows 2g, 2g + 1]
+  float inbox_o[kRowHalves * (kHeadDim + 4 * kDecodeMaxCluster) * kMaxGroup];   // [source CTA, row half][my column][head]
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -86,7 +91,6 @@ __device__ __forceinline__ void tensor_copy_4d(uint32_t dst, const CUtensorMap *
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar), "l"(policy)
       : "memory");
 }
-
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -95,6 +99,14 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, u
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
+// D(16x8, fp32) = A(16x16, bf16, row) * B(16x8, bf16, col): the first link of an accumulator chain
+__device__ __forceinline__ void mma_first(float &d0, float &d1, float &d2, float &d3, uint32_t a0, uint32_t a1, uint32_t a2,
+                                          uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
 
 // Byte offset, inside a staged K or V tile (two 2 KB boxes: columns 0..63 and 64..127), of the 16-byte piece
 // `piece` (0..15) of row `row` (0..15): the 128-byte swizzle of the tensor copy XORs the piece index within a
@@ -102,6 +114,10 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, u
 __device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
   return (uint32_t)((piece >> 3) * kHalfBytes + row * 128 + (((piece & 7) ^ (row & 7)) << 4));
 }
+
+// keeps a value that was worked out early in a register, so that the work is not redone (later) where it is used
+__device__ __forceinline__ void pin(uint32_t &x) { asm volatile("" : "+r"(x)); }
+__device__ __forceinline__ void pin(int &x) { asm volatile("" : "+r"(x)); }
 
 // kMulti: the CTA's range is longer than the staging area and goes through it in rounds
 template <bool kMulti>
@@ -120,6 +136,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;
   const int h0 = 2 * c, h1 = 2 * c + 1;                           // the two heads a lane's accumulators belong to
+  const int cg8 = warp & 7, half = warp >> 3;                     // second product: column group and row half of this warp
   const bool append = p.k_new != nullptr;
 
   // tiles of this CTA: an even deal of the head's n_tiles over the gridDim.x CTAs, contiguous ranges
@@ -131,25 +148,26 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
 
   // columns each CTA of the cluster finishes: a multiple of 4, the last CTA may get fewer
   const int cols = ((kHeadDim + cs - 1) / cs + 3) & ~3;
-  const int my_cols = max(0, min(cols, kHeadDim - rank * cols));   // (cluster sizes that do not divide 128 leave the last CTAs fewer, or none)
+  const int my_cols = max(0, min(cols, kHeadDim - rank * cols));
   const int n_pairs = (p.G + 1) >> 1;                             // head pairs in use
 
-  const uint32_t bar0 = smem_u32(&sh.bar[0]);
+  const uint32_t bar0 = smem_u32(&sh.bar[0]), inbox_bar = smem_u32(&sh.inbox_bar);
   if (tid == 0) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) mbar_init(bar0 + 8 * i, 1);
-    mbar_init(smem_u32(&sh.inbox_bar), 1);
+    mbar_init(inbox_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
-    // from every CTA of the cluster: 8 bytes per (own column, head pair in use) and 64 bytes of (max, sum) pairs
-    mbar_expect_tx(smem_u32(&sh.inbox_bar), (uint32_t)(cs * (my_cols * n_pairs * 8 + 64)));
+    // from both row halves of every CTA of the cluster: 8 bytes per (own column, head pair in use) and 64 bytes
+    // of (max, sum) pairs
+    mbar_expect_tx(inbox_bar, (uint32_t)(kRowHalves * cs * (my_cols * n_pairs * 8 + 64)));
   }
   __syncthreads();
   cluster.barrier_arrive();                              // waited for just before the first store into a peer: its barrier is set up
 
-  // the copies of one round, K boxes first: lane i of warp 0 issues requests i, i + 32, ...
+  // the copies of one round, K boxes first: lane i of the issuing warp takes requests i, i + 32, ...
   uint64_t stream_policy;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
   auto issue_round = [&](int r) {
@@ -165,9 +183,9 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     for (int op = lane; op < nt * 4; op += 32) {
       const bool is_v = op >= nt * 2;
       const int o2 = is_v ? op - nt * 2 : op;
-      const int t = o2 >> 1, half = o2 & 1;
-      const uint32_t dst = stage + (uint32_t)((buf * kDecodeRoundTiles + t) * kTileBytes + (is_v ? 2 : 0) * kHalfBytes + half * kHalfBytes);
-      tensor_copy_4d(dst, is_v ? &map_v : &map_k, half * 64, (first_tile + t0 + t) << 4, kvh, b, is_v ? vbar : kbar, stream_policy);
+      const int t = o2 >> 1, hf = o2 & 1;
+      const uint32_t dst = stage + (uint32_t)((buf * kDecodeRoundTiles + t) * kTileBytes + (is_v ? 2 : 0) * kHalfBytes + hf * kHalfBytes);
+      tensor_copy_4d(dst, is_v ? &map_v : &map_k, hf * 64, (first_tile + t0 + t) << 4, kvh, b, is_v ? vbar : kbar, stream_policy);
     }
   };
 
@@ -180,21 +198,24 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
-  if (warp == 0 && my_tiles > 0) {
+  if (warp == kIssueWarp && my_tiles > 0) {
     issue_round(0);
     if (kMulti && n_rounds > 1) issue_round(1);
   }
 
-  // Everything that does not depend on the predecessor's results is worked out before the wait: which of this
-  // lane's score elements are visible to their heads (sink, own segment, window; bit 4i + e for tile i, element
-  // e), and where the finishing stage finds its operands.
+  // ---- everything that does not depend on the predecessor's results is worked out before the wait ----
+  // The instructions after the wait form one long dependent chain per warp, so every address, mask and index
+  // that can be known now is computed now and kept in a register.
+  // (1) which of this lane's score elements are visible to their heads (sink, own segment, window): bit 4i + e
+  //     for the warp's i-th tile of the round, element e of the accumulator
   const int win_lo = p.S + p.n_sel;
   const int seg0_lo = p.S + h0 * p.k_q, seg0_hi = seg0_lo + p.k_q, seg1_lo = seg0_hi, seg1_hi = seg1_lo + p.k_q;
   auto visibility = [&](int t0) {
     uint32_t bits = 0;
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {
-      const int ra = ((first_tile + t0 + warp + kDecodeWarps * i) << 4) + g, rb = ra + 8;
+    for (int i = 0; i < kQkTiles; ++i) {
+      const int r0 = ((first_tile + t0 + warp + kDecodeWarps * i) << 4) + 2 * g;
+      const int ra = r0 + (g >= 4 ? 1 : 0), rb = r0 + (g >= 4 ? 0 : 1);   // tokens of accumulator elements 0, 1 and 2, 3
       const bool va = ra < p.L, vb = rb < p.L;
       const bool sa = ra < p.S || ra >= win_lo, sb = rb < p.S || rb >= win_lo;
       bits |= (va && h0 < p.G && (sa || (ra >= seg0_lo && ra < seg0_hi)) ? 1u : 0u) << (4 * i);
@@ -205,14 +226,48 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     return bits;
   };
   uint32_t vis = visibility(0);
-  // finishing stage: four lanes per output value (own column lc, head fh), lane q of them holds the shares of
-  // source CTAs q and q + 4
-  const int fin_items = my_cols * p.G, fin_q = tid & 3;
+  // (2) fragment addresses: K rows for the first product (ldmatrix), the query rows (ldmatrix), V for the second
+  //     (transposing ldmatrix), the weight words this lane writes and reads
+  // Row order of the K fragments: A row m of the mma (m < 8) holds token 2m (m < 4) or 2m + 1, A row m + 8 the
+  // other token of the pair (2m, 2m + 1).  So a lane's accumulators belong to two neighbouring tokens, whose
+  // weights make one 32-bit word of the second product's B fragment, and the eight rows one ldmatrix phase
+  // reads still fall into eight different bank groups of the swizzled tile.
   const int mi = lane >> 3, l8 = lane & 7;
-  const int arow = (mi & 1) * 8 + l8;                     // ldmatrix row of this lane for K fragments
-  const int vrow = (mi >> 1) * 8 + l8, vpiece = 2 * warp + (mi & 1);
-  const uint32_t v_lane_off = 2 * kHalfBytes + tile_offset(vrow, vpiece);
-  const uint16_t *prow = &sh.P[g][2 * c];
+  const int arow = 2 * l8 + (((mi & 1) != 0) != (l8 >= 4) ? 1 : 0);
+  uint32_t k_off[8];                                     // k-step ks of a tile: tile base + k_off[ks]
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) k_off[ks] = tile_offset(arow, 2 * ks + (mi >> 1));
+  const uint16_t *q_lane = p.q + ((int64_t)b * p.H_q + kvh * p.G + min(g, p.G - 1)) * kHeadDim + 2 * c;   // this lane's first query element
+  uint32_t v_off = 2 * kHalfBytes + tile_offset((mi >> 1) * 8 + l8, 2 * cg8 + (mi & 1));
+  uint32_t pw_addr = smem_u32(sh.P) + (uint32_t)((h0 * kPHeadWords + g) * 4);   // + tile * kPTileWords * 4; head h1: + kPHeadWords * 4
+  uint32_t pr_addr = smem_u32(sh.P) + (uint32_t)((g * kPHeadWords + c) * 4);    // + tile * kPTileWords * 4; rows 2c+8, 2c+9: + 16
+  // (3) where this lane's results go: the owners of its two columns, as addresses in their shared memory
+  const int col_a = 16 * cg8 + g, col_b = col_a + 8;
+  const int own_a = col_a / cols, own_b = col_b / cols;
+  const int src_me = kRowHalves * rank + half;                    // this warp's place among the sources of an inbox
+  uint32_t dst_a, dst_b, bar_a, bar_b, dst_ml = 0, bar_ml = 0;
+  {
+    const uint32_t inbox = smem_u32(sh.inbox_o);
+    const uint32_t la = inbox + (uint32_t)(((src_me * cols + (col_a - own_a * cols)) * kMaxGroup + h0) * 4);
+    const uint32_t lb = inbox + (uint32_t)(((src_me * cols + (col_b - own_b * cols)) * kMaxGroup + h0) * 4);
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst_a) : "r"(la), "r"(own_a));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst_b) : "r"(lb), "r"(own_b));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_a) : "r"(inbox_bar), "r"(own_a));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_b) : "r"(inbox_bar), "r"(own_b));
+    if (cg8 == 0 && g < cs) {                            // lane (g, c) of a half's first warp tells CTA g the (max, sum) of heads 2c, 2c+1
+      const uint32_t lm = smem_u32(&sh.inbox_ml[src_me][h0]);
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst_ml) : "r"(lm), "r"(g));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_ml) : "r"(inbox_bar), "r"(g));
+    }
+  }
+  // (4) the finishing stage: one thread per output value (own column lc, head fh)
+  const int fin_items = my_cols * p.G, n_src = kRowHalves * cs;
+  int fin_lc = tid / p.G, fin_h = tid - fin_lc * p.G;
+  uint16_t *fin_out = p.out + ((int64_t)b * p.H_q + kvh * p.G + fin_h) * kHeadDim + rank * cols + fin_lc;
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) pin(k_off[ks]);
+  asm volatile("" : "+l"(q_lane)); pin(v_off); pin(pw_addr); pin(pr_addr); pin(dst_a); pin(dst_b); pin(bar_a); pin(bar_b); pin(dst_ml); pin(bar_ml);
+  pin(vis); pin(fin_lc); pin(fin_h); asm volatile("" : "+l"(fin_out));
 
   if (p.pdl_mode >= 2) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -222,16 +277,14 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   // What the predecessor may have written is read now, all requests issued back to back (query first: the first
   // product needs it; the step counter last: only the patch of the replaced row needs it), so the round trips to
   // L2 overlap instead of queueing behind one another.
-  // B fragments of Q^T for the first product: lane (g, c) holds head g's dims 16ks + 2c, +1 and 16ks + 8 + 2c, +1
-  uint32_t qb[8][2];
+  uint32_t qb[8][2];                      // B fragments of Q^T: lane (g, c) holds head g's dims 16ks + 2c, +1 and 16ks + 8 + 2c, +1
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) qb[ks][0] = qb[ks][1] = 0u;
   if (g < p.G) {
-    const uint16_t *qrow = p.q + ((int64_t)b * p.H_q + kvh * p.G + g) * kHeadDim;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
-      asm volatile("ld.global.b32 %0, [%1];" : "=r"(qb[ks][0]) : "l"(qrow + 16 * ks + 2 * c));
-      asm volatile("ld.global.b32 %0, [%1];" : "=r"(qb[ks][1]) : "l"(qrow + 16 * ks + 8 + 2 * c));
+      asm volatile("ld.global.b32 %0, [%1];" : "=r"(qb[ks][0]) : "l"(q_lane + 16 * ks));
+      asm volatile("ld.global.b32 %0, [%1];" : "=r"(qb[ks][1]) : "l"(q_lane + 16 * ks + 8));
     }
   }
   const uint16_t *kn = append ? p.k_new + ((int64_t)b * p.H_kv + kvh) * kHeadDim : nullptr;
@@ -249,9 +302,9 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   }
 
   float M0 = -INFINITY, M1 = -INFINITY;   // running maxima of heads 2c, 2c+1 over the CTA's rows (log2 units)
-  float L0 = 0.f, L1 = 0.f;               // running sums of the (bf16-rounded) weights over the CTA's rows
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};    // O^T: (col 16w+g, h0) (col 16w+g, h1) (col 16w+g+8, h0) (col 16w+g+8, h1)
-  bool dead = false;                      // a copy never arrived: the CTA contributes nothing
+  float L0 = 0.f, L1 = 0.f;               // sums of the (bf16-rounded) weights over this warp's rows of the second product
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};    // O^T: (col_a, h0) (col_a, h1) (col_b, h0) (col_b, h1) over this warp's rows
+  bool timed_out = false;                 // a copy never arrived: reported through the status word; the CTA runs on (its output is then meaningless)
   int slot = -1, slot_tile = -1;          // the replaced window row and its CTA-local tile, worked out at first use
 
   for (int r = 0; r < n_rounds; ++r) {
@@ -262,7 +315,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     const uint32_t kbar = bar0 + 8 * buf, vbar = bar0 + 16 + 8 * buf;
     const uint32_t buf_base = stage + (uint32_t)(buf * kDecodeRoundTiles * kTileBytes);
     if (kMulti && r > 0) vis = visibility(t0);
-    if (nt > 0 && !dead && !mbar_wait(kbar, par)) dead = true;
+    if (nt > 0 && !mbar_wait(kbar, par)) timed_out = true;
 
     // the staged copy of the replaced row is stale: the warp that works on its tile patches K and V
     if (append && r == 0) {
@@ -270,9 +323,9 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       slot_tile = (slot >> 4) - first_tile;
     }
     const int st = slot_tile - t0;                       // tile of this round holding the replaced row, if in [0, nt)
-    if (append && st >= 0 && st < nt && (st & (kDecodeWarps - 1)) == warp && !dead) {
-      if (!mbar_wait(vbar, par)) dead = true;
-      if (!dead) {
+    if (append && st >= 0 && st < nt && (st & (kDecodeWarps - 1)) == warp) {
+      if (!mbar_wait(vbar, par)) timed_out = true;
+      {
         const int row = slot & 15, piece = lane & 15;
         const uint32_t dst = buf_base + (uint32_t)(st * kTileBytes + (lane < 16 ? 0 : 2 * kHalfBytes)) + tile_offset(row, piece);
         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(new_row.x), "r"(new_row.y), "r"(new_row.z), "r"(new_row.w) : "memory");
@@ -284,70 +337,73 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       }
       __syncwarp();
     }
-    dead = __any_sync(0xffffffffu, dead);
 
-    // ---- S = K Q^T: this warp's tiles of the round are warp, warp + 8, warp + 16 ----
-    // An mma takes far longer than its issue slot, so the work is laid out as many short independent chains:
-    // per tile four accumulators (k-steps j and j + 4), the fragments of all tiles requested ahead of the mmas.
-    float sv[3][4];
+    // ---- S = K Q^T: this warp's tiles of the round are warp, warp + kDecodeWarps, ... ----
+    // An mma takes far longer than its issue slot, so the work is laid out as short independent chains: per
+    // tile four accumulators (k-steps j and j + 4), the fragments requested ahead of the mmas.
+    float sv[kQkTiles][4];
     float wm0 = -INFINITY, wm1 = -INFINITY;
     {
-      float ch[3][4][4];
+      float ch[kQkTiles][4][4];
+      uint32_t fa[kQkTiles][4][4];
 #pragma unroll
-      for (int i = 0; i < 3; ++i)
+      for (int hf = 0; hf < 2; ++hf) {                   // k-steps 0..3, then 4..7
 #pragma unroll
-        for (int j = 0; j < 4; ++j) ch[i][j][0] = ch[i][j][1] = ch[i][j][2] = ch[i][j][3] = 0.f;
+        for (int i = 0; i < kQkTiles; ++i) {
+          if (warp + kDecodeWarps * i < nt) {
+            const uint32_t tb = buf_base + (uint32_t)((warp + kDecodeWarps * i) * kTileBytes);
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {             // k-steps 0..3, then 4..7: twelve independent mmas each time
-        uint32_t fa[3][4][4];
-#pragma unroll
-        for (int i = 0; i < 3; ++i) {
-          const int t = warp + kDecodeWarps * i;
-          if (t < nt && !dead) {
-            const uint32_t tb = buf_base + (uint32_t)(t * kTileBytes);
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              ldmatrix_x4(tb + tile_offset(arow, 2 * (4 * half + j) + (mi >> 1)), fa[i][j][0], fa[i][j][1], fa[i][j][2], fa[i][j][3]);
+            for (int j = 0; j < 4; ++j) ldmatrix_x4(tb + k_off[4 * hf + j], fa[i][j][0], fa[i][j][1], fa[i][j][2], fa[i][j][3]);
           }
         }
 #pragma unroll
-        for (int i = 0; i < 3; ++i) {
-          const int t = warp + kDecodeWarps * i;
-          if (t < nt && !dead) {
+        for (int i = 0; i < kQkTiles; ++i) {
+          if (warp + kDecodeWarps * i < nt) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              mma_bf16_16816(ch[i][j][0], ch[i][j][1], ch[i][j][2], ch[i][j][3], fa[i][j][0], fa[i][j][1], fa[i][j][2], fa[i][j][3],
-                             qb[4 * half + j][0], qb[4 * half + j][1]);
+            for (int j = 0; j < 4; ++j) {
+              if (hf == 0)
+                mma_first(ch[i][j][0], ch[i][j][1], ch[i][j][2], ch[i][j][3], fa[i][j][0], fa[i][j][1], fa[i][j][2], fa[i][j][3],
+                          qb[j][0], qb[j][1]);
+              else
+                mma_bf16_16816(ch[i][j][0], ch[i][j][1], ch[i][j][2], ch[i][j][3], fa[i][j][0], fa[i][j][1], fa[i][j][2], fa[i][j][3],
+                               qb[4 + j][0], qb[4 + j][1]);
+            }
           }
         }
       }
 #pragma unroll
-      for (int i = 0; i < 3; ++i) {
-        const int t = warp + kDecodeWarps * i;
-        const uint32_t vb4 = (t < nt && !dead) ? (vis >> (4 * i)) & 15u : 0u;
+      for (int i = 0; i < kQkTiles; ++i) {
+        const bool have = warp + kDecodeWarps * i < nt;
+        const uint32_t vb4 = have ? (vis >> (4 * i)) & 15u : 0u;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float x = (ch[i][0][e] + ch[i][1][e]) + (ch[i][2][e] + ch[i][3][e]);
+          const float x = have ? (ch[i][0][e] + ch[i][1][e]) + (ch[i][2][e] + ch[i][3][e]) : 0.f;
           sv[i][e] = ((vb4 >> e) & 1u) ? x * p.scale_log2 : -INFINITY;
         }
         wm0 = fmaxf(wm0, fmaxf(sv[i][0], sv[i][2]));
         wm1 = fmaxf(wm1, fmaxf(sv[i][1], sv[i][3]));
       }
     }
-#pragma unroll
-    for (int off = 4; off < 32; off <<= 1) {
-      wm0 = fmaxf(wm0, __shfl_xor_sync(0xffffffffu, wm0, off));
-      wm1 = fmaxf(wm1, __shfl_xor_sync(0xffffffffu, wm1, off));
-    }
+    // over the eight lanes that hold the same heads (equal c): one warp-wide reduction per head
+    asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(wm0) : "f"(wm0), "r"(0x11111111u << c));
+    asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(wm1) : "f"(wm1), "r"(0x11111111u << c));
     if (g == 0) { sh.warp_m[warp][h0] = wm0; sh.warp_m[warp][h1] = wm1; }
     if (kMulti) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads and patches of the other buffer precede its refill
     __syncthreads();   // A: the round's maxima are complete; every warp is past the round before
 
-    if (kMulti && warp == 0 && r >= 1 && r + 1 < n_rounds) issue_round(r + 1);   // into the buffer of round r - 1
+    if (kMulti && warp == kIssueWarp && r >= 1 && r + 1 < n_rounds) issue_round(r + 1);   // into the buffer of round r - 1
 
-    float R0 = -INFINITY, R1 = -INFINITY;
+    float R0, R1;
+    {
+      float a0[kDecodeWarps], a1[kDecodeWarps];
 #pragma unroll
-    for (int w = 0; w < kDecodeWarps; ++w) { R0 = fmaxf(R0, sh.warp_m[w][h0]); R1 = fmaxf(R1, sh.warp_m[w][h1]); }
+      for (int w = 0; w < kDecodeWarps; ++w) { a0[w] = sh.warp_m[w][h0]; a1[w] = sh.warp_m[w][h1]; }
+#pragma unroll
+      for (int s2 = kDecodeWarps / 2; s2 > 0; s2 >>= 1)   // a tree, not a chain
+#pragma unroll
+        for (int w = 0; w < s2; ++w) { a0[w] = fmaxf(a0[w], a0[w + s2]); a1[w] = fmaxf(a1[w], a1[w + s2]); }
+      R0 = a0[0]; R1 = a1[0];
+    }
     const float N0 = fmaxf(M0, R0), N1 = fmaxf(M1, R1);
     const float s0 = N0 == -INFINITY ? 0.f : N0, s1 = N1 == -INFINITY ? 0.f : N1;
     if (kMulti && r > 0) {                                 // bring sums and accumulators to the new maxima
@@ -356,46 +412,50 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       acc[0] *= f0; acc[2] *= f0; acc[1] *= f1; acc[3] *= f1;
     }
     M0 = N0; M1 = N1;
-    // the weights enter the second product as bf16
+    // the weights enter the second product as bf16: one word per (tile, head, row pair g: rows 2g and 2g + 1)
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < kQkTiles; ++i) {
       const int t = warp + kDecodeWarps * i;
       if (t < nt) {
-        const uint32_t p0 = pack_bf16x2(fast_exp2(sv[i][0] - s0), fast_exp2(sv[i][2] - s0));   // head h0: rows g, g + 8
-        const uint32_t p1 = pack_bf16x2(fast_exp2(sv[i][1] - s1), fast_exp2(sv[i][3] - s1));   // head h1
-        uint16_t *w0 = &sh.P[h0][t * 16 + g], *w1 = &sh.P[h1][t * 16 + g];
-        w0[0] = (uint16_t)(p0 & 0xffffu); w0[8] = (uint16_t)(p0 >> 16);
-        w1[0] = (uint16_t)(p1 & 0xffffu); w1[8] = (uint16_t)(p1 >> 16);
+        const float x0 = fast_exp2(sv[i][0] - s0), x2 = fast_exp2(sv[i][2] - s0);              // head h0: elements 0 and 2
+        const float x1 = fast_exp2(sv[i][1] - s1), x3 = fast_exp2(sv[i][3] - s1);              // head h1: elements 1 and 3
+        const uint32_t p0 = g < 4 ? pack_bf16x2(x0, x2) : pack_bf16x2(x2, x0);                 // (row 2g in the low half)
+        const uint32_t p1 = g < 4 ? pack_bf16x2(x1, x3) : pack_bf16x2(x3, x1);
+        const uint32_t wa = pw_addr + (uint32_t)(t * kPTileWords * 4);
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(wa), "r"(p0) : "memory");
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(wa + kPHeadWords * 4), "r"(p1) : "memory");
       }
     }
-    if (nt > 0 && !dead && !mbar_wait(vbar, par)) dead = true;
-    dead = __any_sync(0xffffffffu, dead);
     __syncthreads();   // B: the weights of the round are in shared memory (and a patched V row is visible)
+    if (nt > 0 && !mbar_wait(vbar, par)) timed_out = true;
 
-    // ---- O^T += V^T P over all rows of the round, columns 16*warp .. 16*warp + 15 ----
-    // Eight tiles per step, each on an accumulator chain of its own; their V fragments and weights are all
-    // requested before the mmas.  The same weights times a fragment of ones give the sums of the rounded
-    // weights per head, in every lane, in the accumulator layout (so numerator and denominator agree, and no
-    // shuffle or shared-memory exchange is needed for them).
-    if (!dead) {
-      float xc[7][4], lc0[4] = {0.f, 0.f, 0.f, 0.f}, lc1[4] = {0.f, 0.f, 0.f, 0.f};
+    // ---- O^T += V^T P: columns 16*cg8 .. +15 over this warp's half of the round's rows ----
+    // A B fragment is two of the weight words (rows 2c, 2c+1 and 2c+8, 2c+9 of head g).  Six tiles per step, each on an
+    // accumulator chain of its own, all fragments requested before the mmas.  The same weights times a fragment
+    // of ones give the sums of the rounded weights per head, in every lane, in the accumulator layout (numerator
+    // and denominator agree; no shuffle or shared-memory exchange is needed for them).
+    {
+      const int nh = kRowHalves == 2 ? (nt + 1) >> 1 : nt;
+      const int t_lo = half ? nh : 0, t_hi = half ? nt : nh;
+      float xc[5][4], lc0[4] = {0.f, 0.f, 0.f, 0.f}, lc1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int u = 0; u < 7; ++u) xc[u][0] = xc[u][1] = xc[u][2] = xc[u][3] = 0.f;
-      const uint32_t vbase = buf_base + v_lane_off;
+      for (int u = 0; u < 5; ++u) xc[u][0] = xc[u][1] = xc[u][2] = xc[u][3] = 0.f;
+      const uint32_t vbase = buf_base + v_off;
       const uint32_t ones = 0x3f803f80u;
-      for (int t8 = 0; t8 < nt; t8 += 8) {
-        uint32_t va[8][4], pb[8][2];
+      for (int t6 = t_lo; t6 < t_hi; t6 += 6) {
+        uint32_t va[6][4], pb[6][2];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (t8 + u < nt) {
-            ldmatrix_x4_trans(vbase + (uint32_t)((t8 + u) * kTileBytes), va[u][0], va[u][1], va[u][2], va[u][3]);
-            pb[u][0] = *reinterpret_cast<const uint32_t *>(prow + (t8 + u) * 16);
-            pb[u][1] = *reinterpret_cast<const uint32_t *>(prow + (t8 + u) * 16 + 8);
+        for (int u = 0; u < 6; ++u) {
+          if (t6 + u < t_hi) {
+            ldmatrix_x4_trans(vbase + (uint32_t)((t6 + u) * kTileBytes), va[u][0], va[u][1], va[u][2], va[u][3]);
+            const uint32_t ra = pr_addr + (uint32_t)((t6 + u) * kPTileWords * 4);
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(pb[u][0]) : "r"(ra));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(pb[u][1]) : "r"(ra + 16));
           }
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (t8 + u < nt) {
+        for (int u = 0; u < 6; ++u) {
+          if (t6 + u < t_hi) {
             if (u == 0) mma_bf16_16816(acc[0], acc[1], acc[2], acc[3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
             else mma_bf16_16816(xc[u - 1][0], xc[u - 1][1], xc[u - 1][2], xc[u - 1][3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
             if (u & 1) mma_bf16_16816(lc1[0], lc1[1], lc1[2], lc1[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
@@ -404,13 +464,12 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
         }
       }
 #pragma unroll
-      for (int e = 0; e < 4; ++e)
-        acc[e] += ((xc[0][e] + xc[1][e]) + (xc[2][e] + xc[3][e])) + ((xc[4][e] + xc[5][e]) + xc[6][e]);
+      for (int e = 0; e < 4; ++e) acc[e] += ((xc[0][e] + xc[1][e]) + (xc[2][e] + xc[3][e])) + xc[4][e];
       L0 += lc0[0] + lc1[0];
       L1 += lc0[1] + lc1[1];
     }
   }
-  if (dead && tid == 0) atomicOr(p.status, kStatusWaitTimeout);
+  if (timed_out) atomicOr(p.status, kStatusWaitTimeout);
 
   // ---- merge the CTAs of the cluster: the owner of a column slice receives it from every CTA ----
   // Every warp sends its 16 columns straight from registers into the owners' inboxes with asynchronous stores
@@ -418,62 +477,62 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   // acknowledgement or for a cluster-wide barrier; a CTA only waits for its own inbox to fill.
   cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs, its barrier is set up
   {
-    auto send2 = [&](uint32_t local_addr, int dst_rank, float x, float y) {
-      uint32_t addr, rbar;
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(addr) : "r"(local_addr), "r"(dst_rank));
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_u32(&sh.inbox_bar)), "r"(dst_rank));
+    auto send2 = [&](uint32_t addr, uint32_t rbar, float x, float y) {
       asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
                    ::"r"(addr), "f"(x), "f"(y), "r"(rbar) : "memory");
     };
-    const uint32_t inbox = smem_u32(sh.inbox_o);
     if (h0 < p.G) {
-      const int col_a = 16 * warp + g, col_b = col_a + 8;
-      const int own_a = col_a / cols, own_b = col_b / cols;
-      send2(inbox + (uint32_t)(((rank * cols + (col_a - own_a * cols)) * kMaxGroup + h0) * 4), own_a, acc[0], acc[1]);
-      send2(inbox + (uint32_t)(((rank * cols + (col_b - own_b * cols)) * kMaxGroup + h0) * 4), own_b, acc[2], acc[3]);
+      send2(dst_a, bar_a, acc[0], acc[1]);
+      send2(dst_b, bar_b, acc[2], acc[3]);
     }
-    if (warp < 2 && 8 * warp + g < cs) {                 // lane (g, c) of warps 0, 1 tells CTA 8*warp + g the (max, sum) of heads 2c and 2c+1
-      const uint32_t mlbox = smem_u32(&sh.inbox_ml[rank][0]);
-      send2(mlbox + (uint32_t)h0 * 8u, 8 * warp + g, M0, L0);
-      send2(mlbox + (uint32_t)h1 * 8u, 8 * warp + g, M1, L1);
+    if (cg8 == 0 && g < cs) {
+      send2(dst_ml, bar_ml, M0, L0);
+      send2(dst_ml + 8u, bar_ml, M1, L1);
     }
   }
-  if (!mbar_wait(smem_u32(&sh.inbox_bar), 0u) && tid == 0) atomicOr(p.status, kStatusWaitTimeout);
+  if (!mbar_wait(inbox_bar, 0u) && tid == 0) atomicOr(p.status, kStatusWaitTimeout);
 
   // ---- finish columns [rank*cols, rank*cols + my_cols) of every head from the inbox ----
   const int bk = b * p.H_kv + kvh;
   const int n_clusters = (int)gridDim.x / cs, cl = ci / cs;
   float *part = p.partials + ((int64_t)bk * n_clusters + cl) * kPartialStride;
-  for (int base = 0; base < fin_items; base += kDecodeThreads / 4) {   // the same trip count in every lane: shuffles inside
-    const int item = min(base + (tid >> 2), fin_items - 1);
-    const bool real = base + (tid >> 2) < fin_items;
-    const int lc = item / p.G, h = item - lc * p.G, col = rank * cols + lc;
-    float2 ml[4];
-    float ov[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {                        // this lane's source CTAs: fin_q, fin_q + 4, ...
-      const int src = fin_q + 4 * j;
-      ml[j] = src < cs ? sh.inbox_ml[src][h] : make_float2(-INFINITY, 0.f);
-      ov[j] = src < cs ? sh.inbox_o[(src * cols + lc) * kMaxGroup + h] : 0.f;
+  for (int item = tid; item < fin_items; item += kDecodeThreads) {
+    if (item != tid) {
+      fin_lc = item / p.G;
+      fin_h = item - fin_lc * p.G;
+      fin_out = p.out + ((int64_t)b * p.H_q + kvh * p.G + fin_h) * kHeadDim + rank * cols + fin_lc;
     }
-    float M = fmaxf(fmaxf(ml[0].x, ml[1].x), fmaxf(ml[2].x, ml[3].x));
-    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));
-    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
-    float o = 0.f, l = 0.f;
+    const int lc = fin_lc, h = fin_h, col = rank * cols + lc;
+    float mx[kRowHalves * kDecodeMaxCluster], ls[kRowHalves * kDecodeMaxCluster], ov[kRowHalves * kDecodeMaxCluster];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float wgt = M == -INFINITY ? 0.f : fast_exp2(ml[j].x - M);
-      o += ov[j] * wgt;
-      l += ml[j].y * wgt;
+    for (int sI = 0; sI < kRowHalves * kDecodeMaxCluster; ++sI) {   // the loads of all sources are in flight together
+      const float2 ml = sI < n_src ? sh.inbox_ml[sI][h] : make_float2(-INFINITY, 0.f);
+      mx[sI] = ml.x; ls[sI] = ml.y;
+      ov[sI] = sI < n_src ? sh.inbox_o[(sI * cols + lc) * kMaxGroup + h] : 0.f;
     }
-    o += __shfl_xor_sync(0xffffffffu, o, 1); l += __shfl_xor_sync(0xffffffffu, l, 1);
-    o += __shfl_xor_sync(0xffffffffu, o, 2); l += __shfl_xor_sync(0xffffffffu, l, 2);
-    if (fin_q != 0 || !real) continue;
+    float tm[kRowHalves * kDecodeMaxCluster];
+#pragma unroll
+    for (int sI = 0; sI < kRowHalves * kDecodeMaxCluster; ++sI) tm[sI] = mx[sI];
+#pragma unroll
+    for (int w2 = kRowHalves * kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
+#pragma unroll
+      for (int sI = 0; sI < w2; ++sI) tm[sI] = fmaxf(tm[sI], tm[sI + w2]);
+    const float M = tm[0];
+#pragma unroll
+    for (int sI = 0; sI < kRowHalves * kDecodeMaxCluster; ++sI) {
+      const float wgt = M == -INFINITY ? 0.f : fast_exp2(mx[sI] - M);
+      ov[sI] *= wgt; ls[sI] *= wgt;
+    }
+#pragma unroll
+    for (int w2 = kRowHalves * kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
+#pragma unroll
+      for (int sI = 0; sI < w2; ++sI) { ov[sI] += ov[sI + w2]; ls[sI] += ls[sI + w2]; }
+    const float o = ov[0], l = ls[0];
     if (n_clusters == 1) {
       float inv;                                           // the output is rounded to bf16: an approximate reciprocal is ample
       asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(l));
       const float outv = l > 0.f ? o * inv : 0.f;
-      p.out[((int64_t)b * p.H_q + kvh * p.G + h) * kHeadDim + col] = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
+      *fin_out = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
       if (p.lse != nullptr && col == 0)
         p.lse[(int64_t)b * p.H_q + kvh * p.G + h] = l > 0.f ? (M + log2f(l)) * kLn2 : -INFINITY;
     } else {
@@ -520,30 +579,26 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   }
 }
 
+
 static size_t decode_smem_bytes(int resident_tiles) {
   return 1024 + (size_t)resident_tiles * kTileBytes + sizeof(DecShared);
 }
 
-// How many clusters of each size can be resident at once when a CTA takes a whole SM (a cluster must fit into
-// one GPC, so this is not n_sm / size: on this part 15 clusters of 8 but 22 of 6).
-// Clusters of 8 CTAs are the portable limit.  (16-CTA clusters were tried: too few of them are co-resident on
-// this part, so the grid ran in two waves.)
-cudaError_t decode_setup(DeviceInfo *dev) {
-  const int max_smem = (int)decode_smem_bytes(kDecodeMaxResident);
-  cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-  if (e != cudaSuccess) return e;
-  for (int c = 0; c <= kDecodeMaxCluster; ++c) dev->cluster_cap[c] = 0;
-  for (int c = 4; c <= kDecodeMaxCluster; ++c) {
+// How many clusters of `c` CTAs with `tiles` resident tiles each can be on the device at once (a cluster must fit
+// into one GPC, so this is not n_sm / c: on this part 15 clusters of 8 whole-SM CTAs but 22 of 6).  Asked of the
+// runtime once per (device, size, tiles) and remembered.  0: unknown.
+static int g_cluster_cap[64][kDecodeMaxCluster + 1][kDecodeMaxResident + 1];   // answer + 1; 0 = not asked yet
+static std::mutex g_cap_mutex;
+
+static int cluster_capacity(int device, int c, int tiles) {
+  if (device < 0 || device >= 64 || c < 1 || c > kDecodeMaxCluster || tiles < 0 || tiles > kDecodeMaxResident) return 0;
+  std::lock_guard<std::mutex> lock(g_cap_mutex);
+  int &slot = g_cluster_cap[device][c][tiles];
+  if (slot == 0) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(c * 64), 1, 1);
     cfg.blockDim = dim3(kDecodeThreads, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)max_smem;
+    cfg.dynamicSmemBytes = decode_smem_bytes(tiles);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = c;
@@ -554,36 +609,50 @@ cudaError_t decode_setup(DeviceInfo *dev) {
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, decode_attn_kernel<false>, &cfg) != cudaSuccess) {
       (void)cudaGetLastError();
-      n = 0;                                             // unknown: this size is then not considered
+      n = 0;
     }
-    dev->cluster_cap[c] = n;
+    slot = n + 1;
   }
-  return cudaSuccess;
+  return slot - 1;
+}
+
+cudaError_t decode_setup(DeviceInfo *dev) {
+  const int max_smem = (int)decode_smem_bytes(kDecodeMaxResident);
+  cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+  (void)dev;
+  return e;
 }
 
 // Launch geometry for a reduced cache of L rows: one cluster per KV head whose CTAs hold their whole range at
 // once when it fits and go through it in rounds otherwise; more clusters per head only beyond kDecodeMaxRounds.
-// heads = batch x KV heads of the launch (0: not known).  When a CTA needs a whole SM and the heads do not fit
-// at once as clusters of 8, smaller clusters are weighed: more of them are resident, each takes longer
-// (about 4.5 us + 0.1 us per tile of a CTA + 1 us per extra round on this part).
+// heads = batch x KV heads of the launch (0, or dev null: not known).  Clusters of 8 (the portable limit) unless a
+// smaller size lets more of the work be resident: back-to-back launches overlap (the next one fetches its rows
+// while this one computes), which only works if the clusters of two launches fit on the device together, so the
+// sizes are compared by  waves of (two launches' clusters) x time of one cluster, the latter about 4 us + 0.07 us
+// per tile of a CTA + 1 us per extra round on this part.  Smaller sizes are considered only where a CTA still
+// holds its whole range at once.
 void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, int *cs, int *resident_tiles, int *smem_bytes) {
   const int n_tiles = (L + 15) / 16;
   int c = 1;
-  while (c < kDecodeBaseCluster && c * 2 <= n_tiles) c <<= 1;                     // cluster size 1, 2, 4 or 8
+  while (c < kDecodeBaseCluster && c * 2 <= n_tiles) c <<= 1;                   // cluster size 1, 2, 4 or 8
   const int per_cluster_cta = kDecodeRoundTiles * kDecodeMaxRounds;              // most tiles a CTA goes through
   const int nc = (n_tiles + c * per_cluster_cta - 1) / (c * per_cluster_cta);
   int per_cta = (n_tiles + c * nc - 1) / (c * nc);                               // most tiles a CTA gets
-  if (dev != nullptr && c == kDecodeBaseCluster && nc == 1 && per_cta > 12 && heads > dev->cluster_cap[c] &&
-      dev->cluster_cap[c] > 0) {
+  if (dev != nullptr && heads > 0 && c == kDecodeBaseCluster && nc == 1) {
     float best = 0.f;
     int best_c = c;
     for (int cand = kDecodeBaseCluster; cand >= 4; --cand) {
-      const int cap = dev->cluster_cap[cand];
-      if (cap <= 0 || n_tiles > cand * per_cluster_cta) continue;
+      if (cand == 7) continue;                                                   // (no more of them fit than of 8)
       const int per = (n_tiles + cand - 1) / cand;
+      if (cand != kDecodeBaseCluster && per > kDecodeMaxResident) continue;
+      const int resident = per <= kDecodeMaxResident ? per : 2 * kDecodeRoundTiles;
       const int rounds = per <= kDecodeMaxResident ? 1 : (per + kDecodeRoundTiles - 1) / kDecodeRoundTiles;
-      const float cost = (float)((heads + cap - 1) / cap) * (4.5f + 0.1f * (float)per + (float)(rounds - 1));
-      if (cand == kDecodeBaseCluster || cost < best) { best = cost; best_c = cand; }
+      const int cap = cluster_capacity(dev->device, cand, resident);
+      if (cap <= 0) continue;
+      const float cost = 0.5f * (float)((2 * heads + cap - 1) / cap) * (4.0f + 0.07f * (float)per + (float)(rounds - 1));
+      if (best == 0.f || cost < best) { best = cost; best_c = cand; }
     }
     c = best_c;
     per_cta = (n_tiles + c - 1) / c;
