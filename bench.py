@@ -187,6 +187,134 @@ def run_reference(args, w):
 
 # ------------------------------------------------------------------------------------------- CUDA arm
 
+class Stack:
+    """The layers of one workload resident on the device, and CUDA graphs of the three phases over them."""
+
+    def __init__(self, B, synth, torch, w, n_layers, graph_steps, dev, hint):
+        self.B, self.torch, self.w, self.dev = B, torch, w, dev
+        self.n_layers, self.graph_steps = n_layers, graph_steps
+        self.sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L, device=dev)
+        strides = []
+        for mode in (0, 1, 2):                      # one score buffer serves every hint mode: the widest stride
+            self.sk.set_select_hint(mode, w.n_sel)
+            strides.append(self.sk.score_stride(w.n_ctx, w.n_init, w.n_recent))
+        self.stride = max(strides)
+        self.set_hint(hint)
+        self.layers = []
+        for l in range(n_layers):
+            lay = synth.make_layer(w, l, dev)
+            lay.pop("heavy")
+            lay["scores"] = torch.empty(w.batch * w.n_q_heads, self.stride, dtype=torch.float32, device=dev)
+            lay["cache"] = self.sk.new_layer(w.n_init, w.n_recent, w.n_sel)
+            lay["out"] = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+            lay["dec"] = [synth.make_decode_inputs(w, l, t, dev) for t in range(graph_steps)]
+            self.layers.append(lay)
+        torch.cuda.synchronize()
+
+    def set_hint(self, mode):
+        self.hint = mode
+        self.sk.set_select_hint(mode, self.w.n_sel)
+
+    def phase_a(self):
+        w = self.w
+        for lay in self.layers:
+            self.B.sagekv_score(self.sk.ctx, lay["q_last"], lay["K"], w.n_ctx, w.n_init, w.n_recent, lay["scores"], self.stride)
+
+    def phase_b(self):
+        w = self.w
+        for lay in self.layers:
+            c = lay["cache"]
+            self.B.sagekv_select_compact(self.sk.ctx, lay["scores"], self.stride, lay["K"], lay["V"], w.n_ctx, w.n_init,
+                                         w.n_recent, w.n_sel, c.idx, c.Kc, c.Vc, c.state)
+
+    def phase_c(self):
+        for t in range(self.graph_steps):
+            for lay in self.layers:
+                d = lay["dec"][t]
+                self.sk.decode_attn(d["q"], d["k_new"], d["v_new"], lay["cache"], lay["out"])
+
+    def graph(self, fn):
+        fn()                                         # eager once: loads modules, sets function attributes
+        self.torch.cuda.synchronize()
+        g = self.torch.cuda.CUDAGraph()
+        with self.torch.cuda.graph(g):
+            fn()
+        return g
+
+    def time_graph(self, g, replays, reps):
+        """Mean milliseconds of `replays` back-to-back replays, over `reps` measurements after one warm-up."""
+        torch = self.torch
+        for _ in range(replays):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        tot = 0.0
+        for _ in range(reps):
+            e0.record()
+            for _ in range(replays):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            tot += e0.elapsed_time(e1)
+        return tot / reps
+
+    def check(self, O):
+        """Layer 0 of what was timed against the oracle: scores, indices, reduced cache, one decode step."""
+        import numpy as np
+        torch, w, lay = self.torch, self.w, self.layers[0]
+        bits = lambda t: t.detach().cpu().contiguous().view(torch.uint16).numpy()
+        self.phase_a(); self.phase_b()
+        torch.cuda.synchronize()
+        cache = lay["cache"]
+        ok = True
+        refs = []
+        for b in range(w.batch):
+            got = lay["scores"].view(w.batch, w.n_q_heads, -1)[b, :, : w.E].cpu().numpy()
+            ref = O.score(bits(lay["q_last"][b]), bits(lay["K"][b]), w.n_init, w.n_recent)
+            ok &= bool(np.all(np.abs(got - ref) <= 1e-3 * np.abs(ref) + 1e-30))
+            idx = cache.indices()[b].cpu().numpy()
+            ok &= bool(np.array_equal(idx, O.select(got, w.k_q, w.n_init)))
+            Kc_ref, Vc_ref = O.compact(bits(lay["K"][b]), bits(lay["V"][b]), idx, w.n_init, w.n_recent)
+            Kc, Vc = cache.cache()
+            ok &= bool(np.array_equal(bits(Kc[b]), Kc_ref) and np.array_equal(bits(Vc[b]), Vc_ref))
+            refs.append((Kc_ref, Vc_ref))
+        d = lay["dec"][0]
+        out = self.sk.decode_attn(d["q"], d["k_new"], d["v_new"], cache)      # one step with append, step counter 0
+        torch.cuda.synchronize()
+        for b in range(w.batch):
+            o_ref, _, _ = O.decode_step(bits(d["q"][b]), bits(d["k_new"][b]), bits(d["v_new"][b]), refs[b][0], refs[b][1], 0,
+                                        w.n_init, w.k_q, w.n_recent)
+            ok &= bool(np.all(np.abs(out[b].float().cpu().numpy() - o_ref) <= 1e-2 + 1e-2 * np.abs(o_ref)))
+        return ok
+
+    def close(self):
+        self.sk.close()
+        self.layers = []
+
+
+def side_workload(B, synth, torch, name, n_layers, dev, hint, check, O):
+    """select+compact, score and decode per layer on a few layers of another workload (not part of the timed step)."""
+    w = synth.workload(name)
+    st = Stack(B, synth, torch, w, n_layers, 4, dev, hint)
+    st.sk.set_overlap(2)
+    ga, gb, gc = st.graph(st.phase_a), st.graph(st.phase_b), st.graph(st.phase_c)
+    a = st.time_graph(ga, 2, 3) * 1e3 / (2 * n_layers)
+    b = st.time_graph(gb, 2, 3) * 1e3 / (2 * n_layers)
+    c = st.time_graph(gc, 8, 3) * 1e3 / (8 * 4 * n_layers)
+    ab = algorithmic_bytes(w)
+    peak, _ = measured_peak()
+    rec = {"workload": name, "layers_timed": n_layers, "of_layers": w.n_layers, "batch": w.batch, "select_hint_mode": hint,
+           "score_us_per_layer": a, "select_compact_us_per_layer": b, "decode_attn_us_per_layer_step": c,
+           "frac_of_peak": {"score": ab["score"] / (a * 1e-6) / 1e9 / peak,
+                            "select_compact": ab["select_compact"] / (b * 1e-6) / 1e9 / peak,
+                            "decode_attn": ab["decode_attn"] / (c * 1e-6) / 1e9 / peak}}
+    if check:
+        rec["parity"] = st.check(O)
+    st.close()
+    del st
+    torch.cuda.empty_cache()
+    return rec
+
+
 def run_cuda(args, w):
     import torch
     from paper_2503_08879_b200 import build as _build, replicas, synth
@@ -202,52 +330,23 @@ def run_cuda(args, w):
     replicas.init("nccl", dev)
     replicas.barrier()
     from paper_2503_08879_b200 import binding as B
+    O = None
+    if args.check:
+        from oracle import sagekv_oracle as O
 
     n_layers = args.layers or w.n_layers
     decode_steps = args.decode_steps if args.decode_steps is not None else w.decode_steps
     graph_steps = min(8, max(1, decode_steps))
     decode_steps = (decode_steps // graph_steps) * graph_steps
-    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L, device=dev)
-
-    # ---- inputs, resident in HBM before anything is timed ----
-    layers = []
-    for l in range(n_layers):
-        lay = synth.make_layer(w, l, dev)
-        lay.pop("heavy")
-        lay["scores"] = sk.new_scores(w.n_ctx, w.n_init, w.n_recent)
-        lay["cache"] = sk.new_layer(w.n_init, w.n_recent, w.n_sel)
-        lay["out"] = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
-        lay["dec"] = [synth.make_decode_inputs(w, l, t, dev) for t in range(graph_steps)]
-        layers.append(lay)
-    torch.cuda.synchronize()
-
-    def phase_a():
-        for lay in layers:
-            sk.score(lay["q_last"], lay["K"], w.n_init, w.n_recent, lay["scores"])
-
-    def phase_b():
-        for lay in layers:
-            sk.select_compact(lay["scores"], lay["K"], lay["V"], w.n_init, w.n_recent, w.n_sel, lay["cache"])
-
-    def phase_c():
-        for t in range(graph_steps):
-            for lay in layers:
-                d = lay["dec"][t]
-                sk.decode_attn(d["q"], d["k_new"], d["v_new"], lay["cache"], lay["out"])
+    hint = args.hint
+    st = Stack(B, synth, torch, w, n_layers, graph_steps, dev, hint)
+    sk, layers = st.sk, st.layers
 
     # decode launches overlap with their predecessor; with several layers the kernel before a decode call
-    # belongs to another layer, so the reduced cache may be prefetched before the dependency wait
+    # belongs to another layer, so the reduced cache may be fetched before the dependency wait
     overlap = args.overlap if args.overlap is not None else (2 if n_layers > 1 else 1)
     sk.set_overlap(overlap)
-    phase_a(); phase_b(); phase_c()          # eager once: loads modules, sets function attributes
-    torch.cuda.synchronize()
-    graphs = []
-    for fn in (phase_a, phase_b, phase_c):
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            fn()
-        graphs.append(g)
-    ga, gb, gc = graphs
+    ga, gb, gc = st.graph(st.phase_a), st.graph(st.phase_b), st.graph(st.phase_c)
     c_replays = decode_steps // graph_steps
 
     def step(ev=None):
@@ -270,8 +369,8 @@ def run_cuda(args, w):
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     torch.cuda.synchronize()
     t_wall0 = time.perf_counter()
-    for s in range(args.steps):
-        step(evs[s])
+    for s_ in range(args.steps):
+        step(evs[s_])
     torch.cuda.synchronize()
     t_wall = time.perf_counter() - t_wall0
     replicas.barrier()
@@ -286,9 +385,34 @@ def run_cuda(args, w):
     tot_ms = replicas.max_over_ranks(tot_ms, dev)
     a_us, b_us, c_us = (replicas.max_over_ranks(x, dev) for x in (a_us, b_us, c_us))
 
+    # ---- beside the timed step (rank 0, one GPU): the other settings of the same calls, and the Qwen shape ----
+    by_hint, by_overlap, other, parity = {}, {}, [], None
+    if rank == 0 and args.gpus == 1 and not args.quick:
+        for mode in (0, 1, 2):
+            st.set_hint(mode)
+            g_a, g_b = (ga, gb) if mode == hint else (st.graph(st.phase_a), st.graph(st.phase_b))
+            by_hint[str(mode)] = {"score_us_per_layer": st.time_graph(g_a, 1, 3) * 1e3 / n_layers,
+                                  "select_compact_us_per_layer": st.time_graph(g_b, 1, 3) * 1e3 / n_layers}
+        st.set_hint(hint)
+        st.phase_a(); st.phase_b()                   # leave the caches as the timed step left them
+        for mode in (0, 1, 2):
+            sk.set_overlap(mode)
+            g_c = gc if mode == overlap else st.graph(st.phase_c)
+            by_overlap[str(mode)] = st.time_graph(g_c, 8, 3) * 1e3 / (8 * graph_steps * n_layers)
+        sk.set_overlap(overlap)
+    if args.check and rank == 0:
+        parity = st.check(O)
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = measure_e2e(args, w, sk, layers, dev, torch)
     e2e["value"] = replicas.max_over_ranks(e2e["value"], dev)
+    cpu = cpu_baseline(w, layers[0], torch) if (rank == 0 and args.gpus == 1 and not args.no_cpu_baseline) else None
+    st.close()
+    del st, layers, ga, gb, gc
+    torch.cuda.empty_cache()
+    if rank == 0 and args.gpus == 1 and not args.quick:
+        for name in ("C4-b1", "C4-b4"):
+            other.append(side_workload(B, synth, torch, name, 4, dev, hint, args.check, O))
 
     peak, peak_kind = measured_peak()
     ab = algorithmic_bytes(w)
@@ -297,11 +421,21 @@ def run_cuda(args, w):
         return {"kernel": kernel, "us_per_launch": us, "bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
                 "frac": gbs / peak, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
                 "algorithmic_bytes": ab[name], "traffic": ncu_traffic(kernel, files)}
+    score_kernel = ("score_logits_kernel+score_finalize_candidates_kernel" if hint == 2
+                    else "score_logits_kernel+score_finalize_kernel")
     kernels = {
-        "score": roof("score", a_us, "score_logits_kernel+score_finalize_kernel", ["score.cu", "common.cuh"]),
+        "score": roof("score", a_us, score_kernel, ["score.cu", "select_compact.cu", "common.cuh"]),
         "select_compact": roof("select_compact", b_us, "select_compact_kernel", ["select_compact.cu", "common.cuh"]),
         "decode_attn": roof("decode_attn", c_us, "decode_attn_kernel", ["decode_attn.cu", "common.cuh"]),
     }
+    if by_hint:
+        kernels["select_compact"]["by_hint_mode"] = by_hint
+        kernels["select_compact"]["note"] = ("hint mode 2: sagekv_score leaves a candidate list behind each row and "
+                                             "sagekv_select_compact ranks it instead of reading the row, so its DRAM "
+                                             "traffic is below the algorithmic bytes (which count the scores); the work "
+                                             "moved shows in score_us_per_layer of the same mode")
+    if by_overlap:
+        kernels["decode_attn"]["by_overlap_mode"] = by_overlap
     share = {"score": a_us * n_layers, "select_compact": b_us * n_layers, "decode_attn": c_us * c_launches}
     dominant = max(share, key=share.get)
 
@@ -314,10 +448,12 @@ def run_cuda(args, w):
                            w.n_q_heads, w.n_kv_heads, w.head_dim),
                        "layers": n_layers, "batch": w.batch, "n_ctx": w.n_ctx, "budget": w.budget, "n_init": w.n_init,
                        "n_recent": w.n_recent, "k_per_kv_head": w.n_sel, "k_q": w.k_q,
-                       "decode_steps_per_step": decode_steps, "decode_overlap_mode": overlap, "parallelism": "replicas x%d" % args.gpus,
+                       "decode_steps_per_step": decode_steps, "decode_overlap_mode": overlap, "select_hint_mode": hint,
+                       "parallelism": "replicas x%d" % args.gpus,
                        "l2": "inputs larger than L2: layers visited round-robin, %.0f MB of K per layer, %.0f MB of "
                              "reduced caches per decode step" % (ab["score"] / 1e6, ab["decode_attn"] * n_layers / 1e6)},
             "score_us_per_layer": a_us, "select_compact_us_per_layer": b_us, "decode_attn_us_per_layer_step": c_us,
+            "score_plus_select_compact_us_per_layer": a_us + b_us,
             "decode_attn_hbm_gbs": kernels["decode_attn"]["achieved"],
             "decode_attn_frac_of_peak": kernels["decode_attn"]["frac"],
             "roofline": {k: kernels[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")},
@@ -328,10 +464,16 @@ def run_cuda(args, w):
             "wall_ms_per_step": t_wall * 1e3 / args.steps,
             "e2e": e2e, "clocks": clocks,
         }
-        if args.gpus == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w, layers[0], torch)
+        for rec in other:
+            tag = rec["workload"].lower().replace("-", "_")
+            line["select_compact_us_per_layer_" + tag] = rec["select_compact_us_per_layer"]
+        if other:
+            line["other_workloads"] = other
+        if parity is not None:
+            line["parity"] = bool(parity and all(r.get("parity", True) for r in other))
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
         print(json.dumps(line), flush=True)
-    sk.close()
     replicas.shutdown()
 
 
@@ -339,6 +481,7 @@ def measure_e2e(args, w, sk, layers, dev, torch):
     """select+compact per layer with HOST inputs and outputs: pinned scores, K, V in; idx, Kc, Vc out."""
     n_host = min(2, len(layers))
     host = []
+    sk.set_select_hint(0)                                # host scores come from anywhere: the plain select path
     for lay in layers[:n_host]:
         host.append({k: lay[k].cpu().pin_memory() for k in ("scores", "K", "V")})
     stage = {"scores": torch.empty_like(layers[0]["scores"]), "K": torch.empty_like(layers[0]["K"]),
@@ -426,6 +569,9 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--overlap", type=int, default=None, help="sagekv_set_overlap mode for the decode phase")
+    ap.add_argument("--hint", type=int, default=2, help="sagekv_set_select_hint mode for the score and select phases")
+    ap.add_argument("--check", action="store_true", help="compare layer 0 of every timed workload with the CPU oracle")
+    ap.add_argument("--quick", action="store_true", help="only the timed step: no other modes, no other workloads")
     args = ap.parse_args()
     from paper_2503_08879_b200 import synth
     w = synth.workload(args.workload)

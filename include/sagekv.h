@@ -201,9 +201,25 @@ int sagekv_set_overlap(sagekv_ctx *ctx, int mode);
  *           sagekv_scores_row_stride() and a buffer that spans
  *           batch*H_q * stride floats; both calls use the words only when the
  *           stride leaves room for them.
- * `k` is reserved for hints that depend on the later call's k (pass the k that
- * sagekv_select_compact will get, or 0).  The setting applies to later calls on
- * the context.  Errors: INVALID (null context, unknown mode, k < 0). */
+ *   mode 2  the caller also passes the `k` that the coming
+ *           sagekv_select_compact calls will be given.  While it normalises a
+ *           row of at least 14337 scores, sagekv_score then runs the first half
+ *           of the selection on it (a bound not above the k/G-th largest score of
+ *           the row, and every score at or above the bound as a candidate) and
+ *           writes, behind the E scores of every row, eight tag words and the
+ *           candidates in position order as 64-bit words, at most
+ *           1.5*(k/G) + 256 of them; sagekv_scores_row_stride() gives the stride
+ *           that leaves room.  sagekv_select_compact, called with the same k,
+ *           buffer and stride, ranks that list instead of reading the row.
+ *           It BELIEVES the list: the caller vouches that the scores, and the
+ *           words behind them, are exactly what sagekv_score wrote.  Scores
+ *           edited in between are not noticed (use mode 0 or 1 for scores from
+ *           anywhere else).  With another k, a stride without the room, or
+ *           shorter rows, both calls behave as in mode 0.  Same results as
+ *           mode 0 on the scores sagekv_score wrote.
+ * In modes 0 and 1 `k` is ignored.  The setting applies to later calls on the
+ * context.  Errors: INVALID (null context, unknown mode, k < 0, k not a multiple
+ * of G, mode 2 with k = 0). */
 int sagekv_set_select_hint(sagekv_ctx *ctx, int mode, int32_t k);
 
 /* Smallest scores_row_stride (in floats, a multiple of 4) that holds a row of

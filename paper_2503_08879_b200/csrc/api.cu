@@ -23,7 +23,7 @@ struct sagekv_ctx {
   int32_t *status;          // one int32: kStatus* bits raised by the kernels
   int last_cuda_error;
   int overlap;              // 0, 1 or 2: see sagekv_set_overlap
-  int hint;                 // 0, 1: see sagekv_set_select_hint
+  int hint;                 // 0, 1, 2: see sagekv_set_select_hint
   int32_t hint_k;
 };
 
@@ -164,6 +164,10 @@ int sagekv_score(sagekv_ctx *ctx, const void *q_last, const void *K, sagekv_stri
   p.row_stride = scores_row_stride;
   p.partials = ctx->score_partials;
   p.sketch = ctx->hint == 1;
+  if (ctx->hint == 2 && ctx->hint_k > 0) {
+    const int64_t kq = ctx->hint_k / ctx->G;
+    p.list_k_q = (int)(kq < E ? kq : E);
+  }
   p.status = ctx->status;
   p.n_chunks = (int)((E + kScoreChunk - 1) / kScoreChunk);
   p.E = (int)E;
@@ -221,6 +225,7 @@ int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_r
   p.B = ctx->shape.batch;
   p.status = ctx->status;
   p.sketch = ctx->hint == 1;
+  p.list = ctx->hint == 2 && k == ctx->hint_k;
   const cudaError_t e = launch_select_compact(p, ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   state->n_init = n_init;
@@ -282,7 +287,7 @@ int sagekv_set_overlap(sagekv_ctx *ctx, int mode) {
 }
 
 int sagekv_set_select_hint(sagekv_ctx *ctx, int mode, int32_t k) {
-  if (ctx == nullptr || mode < 0 || mode > 1 || k < 0) return SAGEKV_ERR_INVALID;
+  if (ctx == nullptr || mode < 0 || mode > 2 || k < 0 || k % ctx->G != 0 || (mode == 2 && k == 0)) return SAGEKV_ERR_INVALID;
   ctx->hint = mode;
   ctx->hint_k = k;
   return SAGEKV_OK;
@@ -295,6 +300,12 @@ int64_t sagekv_scores_row_stride(const sagekv_ctx *ctx, int64_t n_ctx, int32_t n
   int64_t stride = (E + 3) & ~(int64_t)3;
   if (stride < 4) stride = 4;
   if (ctx->hint == 1 && E >= kSketchMinE) stride += kSketchRoom;
+  if (ctx->hint == 2) {
+    const int64_t kq = ctx->hint_k / ctx->G;
+    const int k_q = (int)(kq < E ? kq : E);
+    const int64_t with_list = stride + ((list_room(k_q) + 3) & ~(int64_t)3);
+    if (list_applies(E, k_q, with_list)) stride = with_list;
+  }
   return stride;
 }
 

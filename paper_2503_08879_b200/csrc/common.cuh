@@ -30,6 +30,7 @@ struct ScoreParams {
   float scale_log2;        // softmax scale * log2(e)
   bool sketch = false;     // leave the histogram of the group maxima behind each row that has room for it
   int64_t sketch_off = -1; // set by launch_score: where in a row it goes, or -1
+  int list_k_q = 0;        // > 0: leave the candidate list for a select step with this k_q behind each row that has room
   int32_t *status = nullptr;   // status word of the context, or null (see kStatus*)
 };
 cudaError_t launch_score(const ScoreParams &p, int n_sm, cudaStream_t stream);
@@ -57,6 +58,25 @@ inline __host__ __device__ bool sketch_fits(int64_t E, int64_t row_stride) {
   return E >= kSketchMinE && row_stride >= sketch_offset(E) + kSketchRoom;
 }
 
+// ---- the candidate list the score step can leave behind each row for the select step ------------------------
+// (hint mode 2, which the caller asks for together with the k of the coming select call.)  While it normalises a
+// row the score step runs the first half of the select step's prefilter: a bound T0 not above the k_q-th largest
+// score, and every score >= T0 as a candidate.  Behind the E scores (from float round_up(E,4) on): eight tag
+// words, a constant, E, k_q, the number of candidates M, the key of T0, the key of the row maximum and two spare
+// words, then the M candidates in position order as 64-bit words, (key << 32) | (2^32 - 1 - offset in the
+// eviction region).  M = 0: no list (the prefilter did not apply to the row).  The select step ranks the list
+// instead of scanning the row, and believes it: the caller vouches that the scores were not touched in between.
+constexpr uint32_t kListMagic = 0x53414732u;
+constexpr int kListTagWords = 8;
+inline __host__ __device__ int list_cand_cap(int k_q) { return (k_q + k_q / 2 + 256) & ~1; }
+inline __host__ __device__ int64_t list_room(int k_q) { return kListTagWords + 2 * (int64_t)list_cand_cap(k_q); }   // 32-bit words
+// the prefilter runs on clusters of 8 CTAs of 512 threads: k_q small against the 4096 thread maxima, slices short
+// enough for its tables
+inline __host__ __device__ bool list_applies(int64_t E, int k_q, int64_t row_stride) {
+  return E >= kSketchMinE && k_q >= 1 && 2 * (int64_t)k_q <= 8 * 512 && E <= (int64_t)8 * 16 * 8 * 512 * 4 &&
+         row_stride >= sketch_offset(E) + list_room(k_q);
+}
+
 // ---- select + compact ------------------------------------------------------
 struct SelectParams {
   const float *scores;
@@ -70,9 +90,12 @@ struct SelectParams {
   int E, S, R, N, k_q, G, H_q, H_kv, B;
   int32_t *status = nullptr;   // status word of the context, or null
   bool sketch = false;         // the caller asked for the histograms behind the rows to be used (sagekv_set_select_hint)
+  bool list = false;           // the caller vouches for the candidate lists behind the rows (hint mode 2)
 };
 cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t stream);
 cudaError_t select_compact_setup();   // one-time function attributes
+// second pass of the score step in hint mode 2: normalise the rows and leave the candidate lists behind them
+cudaError_t launch_score_finalize_candidates(const ScoreParams &p, cudaStream_t stream);
 
 // ---- decode attention ------------------------------------------------------
 #if !defined(SAGEKV_DECODE_WARPS)

@@ -243,11 +243,13 @@ __global__ void __launch_bounds__(kSketchThreads) score_finalize_sketch_kernel(c
 cudaError_t launch_score(const ScoreParams &p_in, int n_sm, cudaStream_t stream) {
   if (p_in.E <= 0) return cudaSuccess;
   ScoreParams p = p_in;
-  p.sketch_off = p.sketch && sketch_fits(p.E, p.row_stride) ? sketch_offset(p.E) : (int64_t)-1;
+  const bool list = p.list_k_q > 0 && list_applies(p.E, p.list_k_q, p.row_stride);
+  p.sketch_off = !list && p.sketch && sketch_fits(p.E, p.row_stride) ? sketch_offset(p.E) : (int64_t)-1;
   dim3 grid(p.n_chunks, p.H_kv, p.B);
   score_logits_kernel<<<grid, kScoreWarps * 32, 0, stream>>>(p);
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
+  if (list) return launch_score_finalize_candidates(p, stream);
   const int rows = p.B * p.H_q;
   if (p.sketch_off >= 0) {
     score_finalize_sketch_kernel<<<dim3(kSketchSlices, rows), kSketchThreads, 0, stream>>>(p, sketch_chunk(p.E));

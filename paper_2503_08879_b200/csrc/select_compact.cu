@@ -154,7 +154,8 @@ __device__ __forceinline__ int n_iterations(int n_vec) { return (n_vec + 8 * kSe
 
 // The eight vectors of iteration `it` of this thread, all loads issued before any use.  Missing ones read as
 // -inf, which is below every threshold and never a maximum.
-template <bool kStaged>
+// kCoherent: the slice was written earlier in this kernel (by this thread), so the read-only path must not be used.
+template <bool kStaged, bool kCoherent = false>
 __device__ __forceinline__ void load8(const float *data, int n_vec, int it, float4 (&x)[8]) {
   const float ninf = -INFINITY;
 #pragma unroll
@@ -165,6 +166,9 @@ __device__ __forceinline__ void load8(const float *data, int n_vec, int it, floa
       if (kStaged) {
         const uint32_t a = (uint32_t)__cvta_generic_to_shared(data + 4 * v);
         asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x[u].x), "=f"(x[u].y), "=f"(x[u].z), "=f"(x[u].w) : "r"(a));
+      } else if (kCoherent) {
+        asm volatile("ld.global.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(x[u].x), "=f"(x[u].y), "=f"(x[u].z), "=f"(x[u].w) : "l"(data + 4 * v) : "memory");
       } else {
         asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];"
                      : "=f"(x[u].x), "=f"(x[u].y), "=f"(x[u].z), "=f"(x[u].w) : "l"(data + 4 * v));
@@ -198,9 +202,14 @@ struct SketchHint {
   uint32_t kmax;   // key of the row maximum
 };
 
-template <bool kStaged, bool kSketch>
-__device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c,
-                           const SketchHint &hint, bool entered) {
+// The path is cut in two: fast_candidates (steps 1 to 3: every CTA ends with the same position-sorted candidate
+// list, the bound T0 and the row maximum) and fast_decide (steps 4 and 5).  The score step can run the first
+// half itself while it normalises a row (kOwnMax: the caller hands in the maximum of the thread's own elements,
+// which it has just written to `c.data`) and leave the list behind the row for the select step to start from.
+template <bool kStaged, bool kSketch, bool kOwnMax = false>
+__device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c,
+                               const SketchHint &hint, bool entered, float own_max, uint32_t &T0_out, uint32_t &kmax_out,
+                               int &M_out) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned long long *cand_local = reinterpret_cast<unsigned long long *>(c.scratch);
   unsigned long long *cand_all = cand_local + c.cand_cap;            // 16-byte aligned: cand_cap is even
@@ -243,7 +252,9 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
   uint32_t tmax = 0;   // 0 is below the key of every number: "no element"
   {
     float fm = -INFINITY;
-    if (kStaged) {
+    if (kOwnMax) {
+      fm = own_max;
+    } else if (kStaged) {
       const int q = n_it * 2;                            // items (it, u) per copy group
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
@@ -267,7 +278,7 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
         for (int u = 0; u < 8; ++u) fm = fmaxf(fmaxf(fm, x[u].x), fmaxf(x[u].y, fmaxf(x[u].z, x[u].w)));
       }
     }
-    if (has_tail) fm = fmaxf(fm, c.data[tail_i]);
+    if (has_tail && !kOwnMax) fm = fmaxf(fm, c.data[tail_i]);
     if (tid < n_vec || has_tail) tmax = score_key(fm);
   }
   sh.gmax[tid] = tmax;
@@ -327,7 +338,7 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
   if (kSketch && kStaged) cp_async_wait<0>();            // no pass over the slice so far: this thread's copies must have landed
   auto hit_mask = [&](int it) {
     float4 x[8];
-    load8<kStaged>(c.data, n_vec, it, x);
+    load8<kStaged, kOwnMax>(c.data, n_vec, it, x);
     uint32_t m = 0;
 #pragma unroll
     for (int u = 0; u < 8; ++u)
@@ -443,6 +454,18 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
   // This CTA is done with its peers' shared memory (the values it read are stored and past a barrier); the
   // arrival is waited for before the kernel ends.  It orders no data, so it need not be a release.
   asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+  T0_out = T0; kmax_out = kmax; M_out = M;
+  return kFastDone;
+}
+
+// Steps 4 and 5 on a position-sorted candidate list that every CTA of the cluster holds in `cand_all` (at least
+// k_q entries, each >= T0; sh.hist_fast zero, sh.n_border zero).  arrived: the CTA has a cluster arrival pending
+// (from fast_candidates) that has to be waited for before another path may run.
+__device__ int fast_decide(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c, uint32_t T0,
+                           uint32_t kmax, int M, bool arrived) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  unsigned long long *cand_all = reinterpret_cast<unsigned long long *>(c.scratch) + c.cand_cap;
+  unsigned char *flag = reinterpret_cast<unsigned char *>(cand_all + c.cand_cap + 2);
 
   // 4. which candidates are kept (every CTA decides for all of them).  A 512-bin histogram of the candidate
   //    keys over [T0, row maximum] locates the bin b1 holding the k_q-th largest: higher bins are kept, lower
@@ -470,7 +493,7 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
   __syncthreads();
   const int nb = sh.n_border;
   if (nb > kSelThreads) {                                // a large group of near-equal scores at the cut
-    cluster.barrier_wait();
+    if (arrived) cluster.barrier_wait();
     return kFastGeneral;
   }
   for (int j = warp; j < nb; j += kSelWarps) {           // one warp per candidate of the border bin
@@ -509,6 +532,16 @@ __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const Sele
   }
   __syncthreads();
   return kFastDone;
+}
+
+template <bool kStaged, bool kSketch>
+__device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c,
+                           const SketchHint &hint, bool entered) {
+  uint32_t T0 = 0u, kmax = 0u;
+  int M = 0;
+  const int code = fast_candidates<kStaged, kSketch>(cluster, sh, p, c, hint, entered, 0.f, T0, kmax, M);
+  if (code != kFastDone) return code;
+  return fast_decide(cluster, sh, p, c, T0, kmax, M, true);
 }
 
 // ---- general path -------------------------------------------------------------------------------
@@ -625,7 +658,7 @@ __device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const 
 
 __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const SelectParams p, int n_rows, int chunk,
                                                                       int resident, int list_cap, int cand_cap,
-                                                                      int try_fast, int64_t sketch_off) {
+                                                                      int try_fast, int64_t sketch_off, int64_t list_off) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   cg::cluster_group cluster = cg::this_cluster();
   const int cs = cluster.num_blocks();
@@ -669,6 +702,20 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(hint.bin0) : "l"(sk + kSketchBins + 2));
     asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(hint.kmax) : "l"(sk + kSketchBins + 3));
   }
+  // the candidate list of the score step, if the caller vouches for it: its tag words and this thread's share of
+  // the entries (as many as the list can have; which of them count is known once the tag is here)
+  constexpr int kListRegs = 7;                            // 7 x 512 entries: the longest list there can be (k_q = 2048)
+  uint32_t lt[6] = {0u, 0u, 0u, 0u, 0u, 0u};
+  unsigned long long le[kListRegs] = {0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull};
+  if (list_off >= 0) {
+    const uint32_t *tg = reinterpret_cast<const uint32_t *>(p.scores + (int64_t)c.row * p.row_stride + list_off);
+#pragma unroll
+    for (int i = 0; i < 6; ++i) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(lt[i]) : "l"(tg + i));
+    const unsigned long long *le_src = reinterpret_cast<const unsigned long long *>(tg + kListTagWords);
+#pragma unroll
+    for (int i = 0; i < kListRegs; ++i)
+      if (tid + i * kSelThreads < cand_cap) asm volatile("ld.global.nc.u64 %0, [%1];" : "=l"(le[i]) : "l"(le_src + tid + i * kSelThreads));
+  }
   if (!resident && sketch_off >= 0 && tid == 0 && c.n_local >= 4) {
     // not staged: ask for the slice to be brought into L2 while the threshold bound is worked out from the hint
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(grow), "r"((uint32_t)(c.n_local >> 2) * 16u) : "memory");
@@ -693,17 +740,39 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   }
 
   // The gather list follows the buffers of the path that runs (see select_smem_bytes).
-  bool done = false;
+  bool done = false, exit_wait = false;   // exit_wait: a cluster arrival of the prefilter is still to be waited for
   if (try_fast) {
     c.list = reinterpret_cast<int2 *>(c.scratch + (size_t)cand_cap * 16 + 16 + (((size_t)cand_cap + 15) & ~(size_t)15));
     int code = kFastRetry;
-    if (sketch_off >= 0 && tag0 == kSketchMagic && tag1 == (uint32_t)p.E)   // the same words in every CTA of the row
+    if (list_off >= 0 && lt[0] == kListMagic && lt[1] == (uint32_t)p.E && lt[2] == (uint32_t)p.k_q && (int)lt[3] >= p.k_q &&
+        (int)lt[3] <= cand_cap && cand_cap <= kListRegs * kSelThreads) {   // the same words in every CTA of the row
+      // start from the score step's list: no pass over the row, no exchange between the CTAs
+      const int M = (int)lt[3];
+      unsigned long long *cand_all = reinterpret_cast<unsigned long long *>(c.scratch) + cand_cap;
+#pragma unroll
+      for (int i = 0; i < kListRegs; ++i)
+        if (tid + i * kSelThreads < M) cand_all[tid + i * kSelThreads] = le[i];
+      if (tid == 0) sh.n_border = 0;
+      cluster.barrier_wait();                              // the arrive at kernel entry; no peer's memory is touched on this path
+      __syncthreads();
+      code = fast_decide(cluster, sh, p, c, lt[4], lt[5], M, false);
+      if (code == kFastGeneral) {                          // (a large group of equal scores at the cut)
+        c.list = reinterpret_cast<int2 *>(c.scratch + kGeneralScratch);
+        general_select(cluster, sh, p, c);
+        code = kFastDone;
+      }
+      done = true;
+    }
+    if (!done && sketch_off >= 0 && tag0 == kSketchMagic && tag1 == (uint32_t)p.E)   // the same words in every CTA of the row
       code = resident ? fast_select<true, true>(cluster, sh, p, c, hint, false)
                       : fast_select<false, true>(cluster, sh, p, c, hint, false);
-    if (code == kFastRetry || code == kFastRetryEntered)
-      code = resident ? fast_select<true, false>(cluster, sh, p, c, hint, code == kFastRetryEntered)
-                      : fast_select<false, false>(cluster, sh, p, c, hint, code == kFastRetryEntered);
-    done = code == kFastDone;
+    if (!done) {
+      if (code == kFastRetry || code == kFastRetryEntered)
+        code = resident ? fast_select<true, false>(cluster, sh, p, c, hint, code == kFastRetryEntered)
+                        : fast_select<false, false>(cluster, sh, p, c, hint, code == kFastRetryEntered);
+      done = code == kFastDone;
+      exit_wait = done;
+    }
   } else {
     cluster.barrier_wait();
   }
@@ -753,7 +822,108 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     }
   }
   if (cid == 0 && rank == 0 && tid == 0) *p.d_step = 0;
-  if (done) cluster.barrier_wait();   // fast path: a peer may still have been copying this CTA's candidates
+  if (exit_wait) cluster.barrier_wait();   // prefilter path: a peer may still have been copying this CTA's candidates
+}
+
+// ---- second pass of the score step in hint mode 2 -----------------------------------------------------------
+// One cluster of 8 CTAs per score row.  Each CTA normalises its slice of the row in place (logits in log2 units
+// -> probabilities, exactly as score_finalize_kernel does), keeps the slice in shared memory when it fits, and
+// then the cluster runs the first half of the select step's prefilter on it (fast_candidates, the thread maxima
+// coming from the normalisation loop).  CTA 0 leaves the position-sorted candidate list and its tag behind the
+// row (layout: common.cuh); M = 0 when the prefilter did not apply.
+__global__ void __launch_bounds__(kSelThreads, 2) score_finalize_candidates_kernel(const ScoreParams sp, const SelectParams p,
+                                                                                 int chunk, int resident, int cand_cap,
+                                                                                 int64_t list_off) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int cs = cluster.num_blocks();
+  const int rank = cluster.block_rank();
+  const int row = blockIdx.x / cs;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  cluster.barrier_arrive();   // completed in fast_candidates: every CTA of the cluster runs before anyone writes into a peer
+  SelShared &sh = *reinterpret_cast<SelShared *>(smem_raw);
+  float *staged = reinterpret_cast<float *>(smem_raw + sizeof(SelShared));
+  SelCtx c;
+  c.cs = cs; c.rank = rank; c.row = row; c.chunk = chunk;
+  c.lo = rank * chunk;
+  c.n_local = max(0, min(p.E - c.lo, chunk));
+  c.list = nullptr;
+  c.list_cap = 0;
+  c.scratch = smem_raw + sizeof(SelShared) + (resident ? (size_t)chunk * sizeof(float) : 0);
+  c.cand_cap = cand_cap;
+  sh.hist_fast[tid] = 0;
+
+  // (max, sum) of the row from the first pass's partials
+  float *sm_m = reinterpret_cast<float *>(&sh.red[0][0]), *sm_l = reinterpret_cast<float *>(&sh.red[1][0]);   // free until the prefilter
+  float m = -INFINITY, l = 0.f;
+  const float2 *part = sp.partials + (int64_t)row * sp.n_chunks;
+  for (int i = tid; i < sp.n_chunks; i += kSelThreads) {
+    const float2 v = part[i];
+    merge_ml(m, l, v.x, v.y);
+  }
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1)
+    merge_ml(m, l, __shfl_xor_sync(0xffffffffu, m, off), __shfl_xor_sync(0xffffffffu, l, off));
+  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+  __syncthreads();
+  m = sm_m[0]; l = sm_l[0];
+#pragma unroll
+  for (int w = 1; w < kSelWarps; ++w) merge_ml(m, l, sm_m[w], sm_l[w]);
+  const float inv = 1.f / l;
+  __syncthreads();   // the prefilter reuses the words the pairs were exchanged in
+
+  // normalise this thread's vectors (the ones it works on in the prefilter: see n_iterations)
+  float *grow = sp.scores + (int64_t)row * sp.row_stride + c.lo;
+  const int n_vec = c.n_local >> 2, n_it = n_iterations(n_vec);
+  float fm = -INFINITY;
+  for (int it = 0; it < n_it; ++it) {
+    float4 x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int v = (it * 8 + u) * kSelThreads + tid;
+      if (v < n_vec) x[u] = *reinterpret_cast<const float4 *>(grow + 4 * v);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int v = (it * 8 + u) * kSelThreads + tid;
+      if (v < n_vec) {
+        x[u].x = fast_exp2(x[u].x - m) * inv; x[u].y = fast_exp2(x[u].y - m) * inv;
+        x[u].z = fast_exp2(x[u].z - m) * inv; x[u].w = fast_exp2(x[u].w - m) * inv;
+        *reinterpret_cast<float4 *>(grow + 4 * v) = x[u];
+        if (resident) *reinterpret_cast<float4 *>(staged + 4 * v) = x[u];
+        fm = fmaxf(fmaxf(fm, x[u].x), fmaxf(x[u].y, fmaxf(x[u].z, x[u].w)));
+      }
+    }
+  }
+  const int tail_i = (n_vec << 2) + tid;
+  if (tail_i < c.n_local) {
+    const float y = fast_exp2(grow[tail_i] - m) * inv;
+    grow[tail_i] = y;
+    if (resident) staged[tail_i] = y;
+    fm = fmaxf(fm, y);
+  }
+  c.data = resident ? staged : grow;
+
+  SketchHint none = {0u, 0u, 0u};
+  uint32_t T0 = 0u, kmax = 0u;
+  int M = 0;
+  const int code = resident ? fast_candidates<true, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M)
+                            : fast_candidates<false, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M);
+  uint32_t *tag = reinterpret_cast<uint32_t *>(sp.scores + (int64_t)row * sp.row_stride + list_off);
+  if (code == kFastDone) {
+    if (rank == 0) {
+      const unsigned long long *cand_all = reinterpret_cast<const unsigned long long *>(c.scratch) + cand_cap;
+      unsigned long long *dst = reinterpret_cast<unsigned long long *>(tag + kListTagWords);
+      for (int i = tid; i < M; i += kSelThreads) dst[i] = cand_all[i];
+    }
+    cluster.barrier_wait();   // a peer may still have been copying this CTA's candidates
+  } else {
+    M = 0;
+  }
+  if (rank == 0 && tid == 0) {
+    tag[0] = kListMagic; tag[1] = (uint32_t)p.E; tag[2] = (uint32_t)p.k_q; tag[3] = (uint32_t)M;
+    tag[4] = T0; tag[5] = kmax; tag[6] = 0u; tag[7] = 0u;
+  }
 }
 
 static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, int share, bool resident) {
@@ -767,7 +937,36 @@ static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, int share
 }
 
 cudaError_t select_compact_setup() {
-  return cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSmemLimit);
+  cudaError_t e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSmemLimit);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(score_finalize_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSmemLimit);
+}
+
+cudaError_t launch_score_finalize_candidates(const ScoreParams &sp, cudaStream_t stream) {
+  const int rows = sp.B * sp.H_q, cs = kMaxCluster;
+  int chunk = (sp.E + cs - 1) / cs;
+  chunk = (chunk + 3) & ~3;
+  const int cand_cap = list_cand_cap(sp.list_k_q);
+  // two CTAs per SM keep every row's cluster resident at once: stage the slice only while two such CTAs fit
+  const bool resident = select_smem_bytes(chunk, 1, cand_cap, 0, true) <= (size_t)kSelSmemLimit / 2;
+  const size_t smem = select_smem_bytes(chunk, 1, cand_cap, 0, resident);
+  SelectParams p = {};
+  p.E = sp.E;
+  p.k_q = sp.list_k_q;
+  p.status = sp.status;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(rows * cs), 1, 1);
+  cfg.blockDim = dim3(kSelThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, score_finalize_candidates_kernel, sp, p, chunk, (int)resident, cand_cap, sketch_offset(sp.E));
 }
 
 cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t stream) {
@@ -776,7 +975,8 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   // The rows may carry the group maxima of the score step (see common.cuh): then the threshold bound costs no
   // pass over the data, the slice is read straight from global memory (no staging: it is needed once), and with
   // many rows smaller clusters pay, because two CTAs per SM times the SM count is all that runs at once.
-  const bool sketch = select && p.sketch && sketch_fits(p.E, p.row_stride);
+  const bool list = select && p.list && list_applies(p.E, p.k_q, p.row_stride);
+  const bool sketch = list || (select && p.sketch && sketch_fits(p.E, p.row_stride));   // both read the row unstaged, if at all
   // cluster size: slices of at least 2048 scores, at most 8 CTAs (the portable limit)
   int cs = 1;
   while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E && (!sketch || (int64_t)n_rows * cs * 2 <= 2 * (int64_t)n_sm)) cs <<= 1;
@@ -816,9 +1016,10 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const int64_t sketch_off = try_fast && sketch ? sketch_offset(p.E) : (int64_t)-1;
+  const int64_t sketch_off = try_fast && sketch && !list ? sketch_offset(p.E) : (int64_t)-1;
+  const int64_t list_off = try_fast && list ? sketch_offset(p.E) : (int64_t)-1;
   return cudaLaunchKernelEx(&cfg, select_compact_kernel, p, n_rows, chunk, (int)resident, list_cap, cand_cap,
-                            try_fast, sketch_off);
+                            try_fast, sketch_off, list_off);
 }
 
 }  // namespace sagekv

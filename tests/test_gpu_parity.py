@@ -93,7 +93,7 @@ def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0, hint=0
         K, V = Kp[:, :, : w.n_ctx, :128], Vp[:, :, : w.n_ctx, :128]
     sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L, softmax_scale=scale)
     sk.set_overlap(overlap)
-    sk.set_select_hint(hint, w.n_sel)
+    sk.set_select_hint(hint if (hint < 2 or w.n_sel > 0) else 0, w.n_sel)
     stride = sk.score_stride(w.n_ctx, w.n_init, w.n_recent)
     n_rows = w.batch * w.n_q_heads
     buf = torch.full((n_rows, stride + 8), 7.5, dtype=torch.float32, device=device)
@@ -199,7 +199,7 @@ def test_c1_full_config(B):
     # and 56 rows: clusters of 4
     ("C4-b1", dict(n_ctx=20000, batch=2), 1),
 ])
-@pytest.mark.parametrize("hint", [0, 1])
+@pytest.mark.parametrize("hint", [0, 1, 2])
 def test_scaled_configs(B, name, kw, n_decode, hint):
     w = synth.workload(name).with_(n_layers=1, **kw)
     run_pipeline(B, w, n_decode, hint=hint)
@@ -245,12 +245,43 @@ def test_full_size_128k_one_layer(B):
     ("C5-4096", 0),     # 512K: the select step reads its unstaged slice in four rounds, the score grid has 2047 chunks
     ("C5-4096", 1),
     ("C5-8192", 1),
+    ("C3-2048", 2),     # and starting from the candidate lists the score step leaves behind the rows
+    ("C4-b1", 2),
+    ("C5-4096", 2),
+    ("C5-8192", 2),
 ])
 def test_every_workload_at_full_size_one_layer(B, name, hint):
     """Each workload at its full context and budget, one layer, with and without the hint behind the score
     rows: scores, indices, reduced cache, two decode steps, all against the oracle."""
     w = synth.workload(name).with_(n_layers=1)
     run_pipeline(B, w, 2, hint=hint)
+
+
+def test_candidate_lists_with_a_large_group_of_equal_scores_at_the_cut(B):
+    """Hint mode 2 on rows in which several hundred tokens share one key, placed so that the k-th score falls
+    inside that group: the select step starts from the score step's list, finds too many equal scores at the cut
+    for its exact ranking and hands the row to the radix path.  The lowest positions of the group must be kept."""
+    w = synth.workload("C2").with_(n_ctx=30001, n_layers=1, budget=4 + 128 + 4 * 300, structure="count", heavy=(100,))
+    dev = "cuda"
+    lay = synth.make_layer(w, 0, dev)
+    g = torch.Generator(device=dev).manual_seed(77)
+    for kvh in range(w.n_kv_heads):                      # 800 copies of one strong key per KV head
+        pos = torch.randperm(w.E, generator=g, device=dev)[:800] + w.n_init
+        q_hat = lay["q_last"][0, kvh * w.G].float()
+        q_hat = q_hat / q_hat.norm()
+        lay["K"][0, kvh, pos] = (3.0 * q_hat).to(torch.bfloat16)
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, 1, max_ctx=w.n_ctx, max_len=w.L)
+    for hint in (2, 0):
+        sk.set_select_hint(hint, w.n_sel)
+        scores = sk.score(lay["q_last"], lay["K"], w.n_init, w.n_recent)
+        layer = sk.select_compact(scores, lay["K"], lay["V"], w.n_init, w.n_recent, w.n_sel)
+        torch.cuda.synchronize()
+        got = scores[:, : w.E].cpu().numpy()
+        idx = layer.indices()[0].cpu().numpy()
+        assert np.array_equal(idx, O.select(got, w.k_q, w.n_init)), hint
+        check_compact(layer, lay, idx, w, 0)
+    assert sk.status() == 0
+    sk.close()
 
 
 @pytest.mark.parametrize("scale", [0.05, 0.2])
