@@ -209,7 +209,7 @@ struct SketchHint {
 template <bool kStaged, bool kSketch, bool kOwnMax = false>
 __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c,
                                const SketchHint &hint, bool entered, float own_max, uint32_t &T0_out, uint32_t &kmax_out,
-                               int &M_out) {
+                               int &M_out, int &my_start) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned long long *cand_local = reinterpret_cast<unsigned long long *>(c.scratch);
   unsigned long long *cand_all = cand_local + c.cand_cap;            // 16-byte aligned: cand_cap is even
@@ -443,6 +443,13 @@ __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const 
   // same counts in every CTA: the whole cluster takes the same way out
   if (overflow || M > c.cand_cap) return kSketch ? kFastRetryEntered : kFastGeneral;
   if (kSketch && M < p.k_q) return kFastRetryEntered;    // the sketch did not describe these scores
+  my_start = start[0];
+#pragma unroll
+  for (int r = 1; r < kMaxCluster; ++r) my_start = r == c.rank ? start[r] : my_start;
+  if (kOwnMax) {   // the score step: each CTA writes its own part of the row's list to global memory; no peer's memory is read
+    T0_out = T0; kmax_out = kmax; M_out = M;
+    return kFastDone;
+  }
   // every CTA takes a copy of all candidates, in CTA order: the list is sorted by position
   for (int i = tid; i < M; i += kSelThreads) {
     int r = 0;
@@ -538,8 +545,8 @@ template <bool kStaged, bool kSketch>
 __device__ int fast_select(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c,
                            const SketchHint &hint, bool entered) {
   uint32_t T0 = 0u, kmax = 0u;
-  int M = 0;
-  const int code = fast_candidates<kStaged, kSketch>(cluster, sh, p, c, hint, entered, 0.f, T0, kmax, M);
+  int M = 0, my_start = 0;
+  const int code = fast_candidates<kStaged, kSketch>(cluster, sh, p, c, hint, entered, 0.f, T0, kmax, M, my_start);
   if (code != kFastDone) return code;
   return fast_decide(cluster, sh, p, c, T0, kmax, M, true);
 }
@@ -829,8 +836,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
 // One cluster of 8 CTAs per score row.  Each CTA normalises its slice of the row in place (logits in log2 units
 // -> probabilities, exactly as score_finalize_kernel does), keeps the slice in shared memory when it fits, and
 // then the cluster runs the first half of the select step's prefilter on it (fast_candidates, the thread maxima
-// coming from the normalisation loop).  CTA 0 leaves the position-sorted candidate list and its tag behind the
-// row (layout: common.cuh); M = 0 when the prefilter did not apply.
+// coming from the normalisation loop).  Every CTA writes its part of the position-sorted candidate list behind
+// the row, CTA 0 the tag (layout: common.cuh); M = 0 when the prefilter did not apply.
 __global__ void __launch_bounds__(kSelThreads, 2) score_finalize_candidates_kernel(const ScoreParams sp, const SelectParams p,
                                                                                  int chunk, int resident, int cand_cap,
                                                                                  int64_t list_off) {
@@ -906,17 +913,15 @@ __global__ void __launch_bounds__(kSelThreads, 2) score_finalize_candidates_kern
 
   SketchHint none = {0u, 0u, 0u};
   uint32_t T0 = 0u, kmax = 0u;
-  int M = 0;
-  const int code = resident ? fast_candidates<true, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M)
-                            : fast_candidates<false, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M);
+  int M = 0, my_start = 0;
+  const int code = resident ? fast_candidates<true, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M, my_start)
+                            : fast_candidates<false, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M, my_start);
   uint32_t *tag = reinterpret_cast<uint32_t *>(sp.scores + (int64_t)row * sp.row_stride + list_off);
-  if (code == kFastDone) {
-    if (rank == 0) {
-      const unsigned long long *cand_all = reinterpret_cast<const unsigned long long *>(c.scratch) + cand_cap;
-      unsigned long long *dst = reinterpret_cast<unsigned long long *>(tag + kListTagWords);
-      for (int i = tid; i < M; i += kSelThreads) dst[i] = cand_all[i];
-    }
-    cluster.barrier_wait();   // a peer may still have been copying this CTA's candidates
+  if (code == kFastDone) {   // the CTAs' lists, one behind the other, are the row's list in position order
+    const unsigned long long *cand_local = reinterpret_cast<const unsigned long long *>(c.scratch);
+    unsigned long long *dst = reinterpret_cast<unsigned long long *>(tag + kListTagWords) + my_start;
+    const int n_mine = sh.cand_cnt[rank];
+    for (int i = tid; i < n_mine; i += kSelThreads) dst[i] = cand_local[i];
   } else {
     M = 0;
   }
