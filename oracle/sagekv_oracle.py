@@ -22,6 +22,10 @@ Notation (Section 2, Step 1, and Appendix A.2):
 Positions are 0-based here: sink [0,S), eviction region [S,S+E), recent window
 [S+E, N-1), last token N-1  (the paper's P_{1:S}, P_{S+1:S+E}, P_{S+E+1:N-1}, P_N).
 
+Section 3.1's baselines that are restated here for the comparison paths: StreamLLM_R
+(rope_rotate, compact_window_rope: Appendix A.1) and the pooled reading of
+Step 2 (select_pooled, compact_pooled, decode_step_pooled).
+
 Pins (tests/test_oracle_pins.py): budget_split <- the numbers Appendix A.2
 prints; score <- closed forms (uniform keys, one planted key), row sums, a
 library softmax; select <- exhaustive subset search on tiny rows, library
@@ -47,6 +51,11 @@ __all__ = [
     "compact",
     "decode_step",
     "full_attention",
+    "rope_rotate",
+    "compact_window_rope",
+    "select_pooled",
+    "compact_pooled",
+    "decode_step_pooled",
 ]
 
 
@@ -280,4 +289,100 @@ def decode_step(q_bits: np.ndarray, k_new_bits, v_new_bits,
         keep[h, S + G * k: L] = True
     o, lse = full_attention(bf16_bits_to_f64(q_bits), bf16_bits_to_f64(Kc),
                             bf16_bits_to_f64(Vc), keep=keep, scale=scale)
+    return o, lse, step
+
+
+# --------------------------------------------------------------------------
+# StreamLLM_R (Section 3.1 "Baselines", Appendix A.1): pre-RoPE cache, positions
+# counted inside the window
+# --------------------------------------------------------------------------
+
+def rope_rotate(x: np.ndarray, pos, theta: float = 10000.0) -> np.ndarray:
+    """Rotary position embedding of rows x [..., d] (float64) at positions pos.
+
+    Dimension i < d/2 is paired with dimension i + d/2 (the layout of the
+    Llama and Qwen models the paper runs); the pair is turned by the angle
+    pos * theta**(-2i/d):
+        y[i]       = x[i] cos(a_i) - x[i + d/2] sin(a_i)
+        y[i + d/2] = x[i + d/2] cos(a_i) + x[i] sin(a_i),   a_i = pos * theta**(-2i/d)
+    pos is a scalar or an array broadcastable to x's leading dimensions.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[-1]
+    half = d // 2
+    inv_freq = float(theta) ** (-(np.arange(half, dtype=np.float64) * 2.0) / d)
+    ang = np.asarray(pos, dtype=np.float64)[..., None] * inv_freq
+    c, s_ = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s_, x2 * c + x1 * s_], axis=-1)
+
+
+def compact_window_rope(K_pre_bits: np.ndarray, V_bits: np.ndarray, S: int, R: int,
+                        theta: float = 10000.0) -> tuple[np.ndarray, np.ndarray]:
+    """StreamLLM_R's cache: sink + recent + last token of a PRE-RoPE key cache,
+    every kept key rotated by its index inside the kept window (Appendix A.1:
+    relative positions are assigned within the sliding window), values copied.
+
+    K_pre_bits, V_bits uint16 [H_kv, N, d].  Returns (Kc, Vc) uint16
+    [H_kv, S + R + 1, d]; row r of Kc is rope_rotate(K_pre[token(r)], r) rounded
+    to bf16, with token(r) = r for r < S and N - 1 - (S + R) + r otherwise.
+    """
+    H_kv, N, d = K_pre_bits.shape
+    E = partition(N, S, R)["E"]
+    L = S + R + 1
+    rows = list(range(0, S)) + list(range(S + E, N))
+    assert len(rows) == L
+    Kc = np.zeros((H_kv, L, d), dtype=np.uint16)
+    Vc = np.zeros((H_kv, L, d), dtype=np.uint16)
+    for g in range(H_kv):
+        for r, t in enumerate(rows):
+            Kc[g, r] = f64_to_bf16_bits(rope_rotate(bf16_bits_to_f64(K_pre_bits[g, t]), float(r), theta))
+            Vc[g, r] = V_bits[g, t]
+    return Kc, Vc
+
+
+# --------------------------------------------------------------------------
+# The pooled reading of Step 2 (one selection per KV head from the summed
+# scores of its G query heads); the per-head reading above is the one the
+# paper's budget rule fixes, this one is kept as the alternative
+# --------------------------------------------------------------------------
+
+def select_pooled(p: np.ndarray, K_sel: int, S: int, G: int) -> np.ndarray:
+    """One top-K_sel per KV head from the sum of its G query heads' score rows.
+
+    p [H_q, E]; rows g*G .. g*G+G-1 are added in float64, in head order, and
+    rounded to p's dtype before they are compared (so a float32 caller compares
+    float32 sums); then `select` on the H_kv summed rows.  Returns int32
+    [H_kv, min(K_sel, E)].
+    """
+    H_q, E = p.shape
+    H_kv = H_q // G
+    pooled = np.zeros((H_kv, E), dtype=np.float64)
+    for g in range(H_kv):
+        for j in range(G):
+            pooled[g] += p[g * G + j].astype(np.float64)
+    return select(pooled.astype(p.dtype), K_sel, S)
+
+
+def compact_pooled(K_bits: np.ndarray, V_bits: np.ndarray, idx: np.ndarray,
+                   S: int, R: int) -> tuple[np.ndarray, np.ndarray]:
+    """Reduced cache for the pooled reading: rows(g) = sink ++ idx[g] ++ recent ++ last."""
+    H_kv = K_bits.shape[0]
+    assert idx.shape[0] == H_kv
+    return compact(K_bits, V_bits, idx, S, R)      # with H_q = H_kv the segment layout is one list per KV head
+
+
+def decode_step_pooled(q_bits: np.ndarray, k_new_bits, v_new_bits, Kc: np.ndarray, Vc: np.ndarray,
+                       step: int, S: int, K_sel: int, R: int,
+                       scale: float | None = None) -> tuple[np.ndarray, np.ndarray, int]:
+    """Step 4 for the pooled reading: every query head attends to ALL rows of its KV head's reduced cache."""
+    H_kv, L, d = Kc.shape
+    assert L == S + K_sel + R + 1
+    if k_new_bits is not None:
+        slot = S + K_sel + (step % (R + 1))
+        for g in range(H_kv):
+            Kc[g, slot] = k_new_bits[g]
+            Vc[g, slot] = v_new_bits[g]
+        step = step + 1
+    o, lse = full_attention(bf16_bits_to_f64(q_bits), bf16_bits_to_f64(Kc), bf16_bits_to_f64(Vc), keep=None, scale=scale)
     return o, lse, step

@@ -107,6 +107,11 @@ def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0, hint=0
     sk.select_compact(scores, K, V, w.n_init, w.n_recent, w.n_sel, layer)
     torch.cuda.synchronize()
     assert torch.equal(first, scores[:, : w.E])                       # the score step repeats bit for bit
+    if hint == 2 and w.E >= 14337 and 0 < w.k_q <= 2048:                # the lists are there and were usable
+        E4 = (w.E + 3) // 4 * 4
+        tags = scores[:, E4:E4 + 8].cpu().numpy().view(np.uint32)
+        assert (tags[:, 0] == 0x53414732).all() and (tags[:, 1] == w.E).all() and (tags[:, 2] == min(w.k_q, w.E)).all()
+        assert (tags[:, 3] >= min(w.k_q, w.E)).mean() >= 0.9, tags[:, 3]   # M = 0 only where the prefilter did not apply
     assert (buf[:, stride:] == 7.5).all()                             # nothing written behind the rows' stride
     if hint == 0:
         assert (buf[:, w.E:] == 7.5).all()

@@ -60,6 +60,24 @@ def test_select_random_rows_bit_exact(B, E, k_q):
     assert np.array_equal(idx, O.select(rows, k_q, 3))
 
 
+@pytest.mark.parametrize("E", [200000, 524027])
+@pytest.mark.parametrize("k_q", [959, 1983])
+def test_select_long_rows_several_load_rounds(B, E, k_q):
+    """Rows long enough that a thread of the prefilter goes through its slice in several rounds of eight vectors:
+    staged slices at E = 200000 (two rounds), unstaged ones at E = 524027 (four), each with a run of large scores
+    across a slice border and a group of equal scores at the cut."""
+    rng = np.random.default_rng(E + k_q)
+    rows = (rng.random((2, E), dtype=np.float32) ** 10).astype(np.float32)
+    slice_len = ((E + 7) // 8 + 3) // 4 * 4
+    for h in range(2):
+        rows[h, slice_len * 2 - 100: slice_len * 2 + 140] = 0.97 + 0.02 * rng.random(240, dtype=np.float32)   # a run over a border
+        kth = np.sort(rows[h])[::-1][k_q - 1]
+        tie = rng.choice(E, 60, replace=False)
+        rows[h, tie] = kth                                                                                  # equal scores at the cut
+    idx = run_select(B, rows, k_q, H_kv=1)
+    assert np.array_equal(idx, O.select(rows, k_q, 3))
+
+
 def test_select_ties_lowest_position_wins(B):
     E = 9000
     rng = np.random.default_rng(5)

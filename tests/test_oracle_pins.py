@@ -306,3 +306,93 @@ def test_decode_recent_window_rolls():
             for g in range(H_kv):
                 got = {Kc[g, r].tobytes() for r in range(S + G * k, L)}
                 assert got == {kv[0].tobytes() for kv in win[g]}
+
+
+# ---------------------------------------------------------------- StreamLLM_R: rotary positions inside the window
+
+def test_rope_rotation_group_properties():
+    """Rotation by 0 is the identity, rotations add up, norms are kept, and the product of a rotated query and
+    a rotated key depends only on the difference of their positions (what makes positions 'relative')."""
+    rng = np.random.default_rng(41)
+    x, y = rng.standard_normal((5, 128)), rng.standard_normal((5, 128))
+    assert np.array_equal(O.rope_rotate(x, 0.0), x)
+    np.testing.assert_allclose(O.rope_rotate(O.rope_rotate(x, 3.0), 11.0), O.rope_rotate(x, 14.0), atol=1e-12)
+    np.testing.assert_allclose(np.linalg.norm(O.rope_rotate(x, 977.0), axis=-1), np.linalg.norm(x, axis=-1), rtol=1e-12)
+    for p, q in ((7, 2), (1007, 1002), (40000, 39995)):
+        a = np.sum(O.rope_rotate(x, float(p)) * O.rope_rotate(y, float(q)), axis=-1)
+        b = np.sum(O.rope_rotate(x, 5.0) * y, axis=-1)
+        np.testing.assert_allclose(a, b, rtol=0, atol=1e-9)
+    np.testing.assert_allclose(O.rope_rotate(x, np.arange(5.0))[3], O.rope_rotate(x[3], 3.0), atol=1e-14)
+
+
+def test_rope_is_a_complex_multiplication():
+    """The textbook form: (x_i + i x_{i+d/2}) * exp(i * pos * theta^(-2i/d)); a swapped sign, a wrong pairing
+    (neighbouring dimensions) or a wrong exponent fails this."""
+    rng = np.random.default_rng(42)
+    d, theta, pos = 64, 500000.0, 1234.0
+    x = rng.standard_normal(d)
+    z = (x[: d // 2] + 1j * x[d // 2:]) * np.exp(1j * pos * theta ** (-np.arange(d // 2) * 2.0 / d))
+    np.testing.assert_allclose(O.rope_rotate(x, pos, theta), np.concatenate([z.real, z.imag]), atol=1e-12)
+
+
+def test_rope_matches_the_llama_implementation_of_a_library():
+    tr = pytest.importorskip("transformers")
+    from transformers.models.llama.modeling_llama import LlamaRotaryEmbedding, apply_rotary_pos_emb
+    cfg = tr.LlamaConfig(hidden_size=4 * 32, num_attention_heads=4, head_dim=32, rope_theta=10000.0,
+                         max_position_embeddings=256)
+    rot = LlamaRotaryEmbedding(cfg)
+    rng = np.random.default_rng(43)
+    x = rng.standard_normal((1, 1, 9, 32)).astype(np.float32)          # [batch, heads, positions, head_dim]
+    pos = torch.arange(20, 29)[None]
+    cos, sin = rot(torch.from_numpy(x), pos)
+    got, _ = apply_rotary_pos_emb(torch.from_numpy(x), torch.from_numpy(x), cos, sin)
+    want = O.rope_rotate(x[0, 0].astype(np.float64), np.arange(20.0, 29.0), 10000.0)
+    np.testing.assert_allclose(got[0, 0].double().numpy(), want, atol=2e-5)
+
+
+def test_compact_window_rope_rows_and_positions():
+    """Which token lands in which row, rotated by the row's own index; values untouched."""
+    rng = np.random.default_rng(44)
+    H, N, d, S, R = 2, 40, 16, 3, 5
+    K, V = rand_bits(rng, H, N, d), rand_bits(rng, H, N, d)
+    Kc, Vc = O.compact_window_rope(K, V, S, R, theta=100.0)
+    tokens = [0, 1, 2, 34, 35, 36, 37, 38, 39]
+    assert Kc.shape == (H, 9, d)
+    for r, t in enumerate(tokens):
+        assert np.array_equal(Vc[:, r], V[:, t])
+        x = bf16_val(K[:, t])
+        z = (x[:, : d // 2] + 1j * x[:, d // 2:]) * np.exp(1j * r * 100.0 ** (-np.arange(d // 2) * 2.0 / d))
+        assert np.array_equal(Kc[:, r], bf16(np.concatenate([z.real, z.imag], axis=-1)))
+    assert np.array_equal(Kc[:, 0], K[:, 0])                              # position 0: no rotation
+
+
+# ---------------------------------------------------------------- the pooled reading of Step 2
+
+def test_select_pooled_is_select_on_the_summed_rows():
+    rng = np.random.default_rng(45)
+    p = rng.random((6, 50)).astype(np.float32)
+    idx = O.select_pooled(p, 7, 4, G=3)
+    assert idx.shape == (2, 7)
+    for g in range(2):
+        summed = (p[3 * g].astype(np.float64) + p[3 * g + 1] + p[3 * g + 2]).astype(np.float32)
+        best = sorted(sorted(range(50), key=lambda i: (-summed[i], i))[:7])
+        assert idx[g].tolist() == [4 + i for i in best]
+    assert np.array_equal(O.select_pooled(p, 7, 4, G=1), O.select(p, 7, 4))   # G = 1: nothing to pool
+
+
+def test_decode_pooled_equals_full_attention_over_the_kept_rows():
+    rng = np.random.default_rng(46)
+    Hq, Hkv, N, d, S, R, Ksel = 4, 2, 60, 16, 2, 6, 9
+    K, V, q = rand_bits(rng, Hkv, N, d), rand_bits(rng, Hkv, N, d), rand_bits(rng, Hq, d)
+    p = O.score(q, K, S, R).astype(np.float32)
+    idx = O.select_pooled(p, Ksel, S, G=2)
+    Kc, Vc = O.compact_pooled(K, V, idx, S, R)
+    o, lse, step = O.decode_step_pooled(q, None, None, Kc, Vc, 0, S, Ksel, R)
+    for h in range(Hq):
+        g = h // 2
+        rows = list(range(S)) + idx[g].tolist() + list(range(N - 1 - R, N))
+        want = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(bf16_val(q[h]))[None, None], torch.from_numpy(bf16_val(K[g, rows]))[None],
+            torch.from_numpy(bf16_val(V[g, rows]))[None])[0, 0]
+        np.testing.assert_allclose(o[h], want.numpy(), atol=1e-10)
+    assert step == 0
