@@ -185,6 +185,47 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
  * Errors: INVALID for a null context or a mode outside 0..2. */
 int sagekv_set_overlap(sagekv_ctx *ctx, int mode);
 
+/* How the G query heads of a KV head share its selected slots.
+ *   0  (default, the paper's reading: Step 2 selects per query head and the
+ *      budget of Appendix A.2 counts G*k slots) every query head keeps its own
+ *      k/G tokens and attends to the sink, its own segment and the window.
+ *   1  pooled: sagekv_select_compact expects ONE score row per KV head
+ *      (batch*H_kv rows, e.g. from sagekv_pool_scores), keeps the k best tokens
+ *      of it (idx is [batch, H_kv, min(k,E)], k need not divide by G), and in
+ *      sagekv_decode_attn every query head attends to all L rows of its KV
+ *      head's cache.  The hints of sagekv_set_select_hint do not apply.
+ * A reduced cache must be decoded in the mode it was built in.
+ * Errors: INVALID (null context, unknown mode). */
+int sagekv_set_group_mode(sagekv_ctx *ctx, int mode);
+
+/* For group mode 1: pooled[b*H_kv + g][i] = sum over the G query heads h of KV
+ * head g of scores[b*H_q + h][i], i in [0,E), added in head order in fp32.
+ *   scores  fp32, batch*H_q rows of stride scores_row_stride, as sagekv_score
+ *           writes them;  pooled  fp32, batch*H_kv rows of stride
+ *           pooled_row_stride (>= E, a multiple of 4; base 16-byte aligned).
+ * Errors: INVALID, ALIGN, UNSUPPORTED (n_ctx above max_ctx), DEVICE, CUDA. */
+int sagekv_pool_scores(sagekv_ctx *ctx, const float *scores, int64_t scores_row_stride, int64_t n_ctx,
+                       int32_t n_init, int32_t n_recent, float *pooled, int64_t pooled_row_stride, void *stream);
+
+/* Section 3.1 "Baselines", StreamLLM_R, and Appendix A.1: the cache of a
+ * sliding-window method that stores keys BEFORE rotary position embedding and
+ * counts positions inside the kept window.  Builds the reduced cache of
+ * sink + recent + last token (no selection: L = S + R + 1 rows per KV head)
+ * from a pre-RoPE key cache, rotating the key that lands in row r by position r:
+ *     a_i = r * rope_theta^(-2i/128),   i in [0,64)
+ *     Kc[r][i]      = K[t][i] cos(a_i) - K[t][i+64] sin(a_i)
+ *     Kc[r][i + 64] = K[t][i+64] cos(a_i) + K[t][i] sin(a_i)
+ * (dimension i paired with i + 64), t = r for r < S, else n_ctx - L + r;
+ * computed in double precision, rounded once to bf16.  V rows are copied
+ * verbatim.  `state` is filled as by sagekv_select_compact with k = 0 and
+ * *d_step is set to 0, so sagekv_decode_attn can run on the result; rows
+ * appended later are stored as given (the caller rotates new keys).
+ * Errors: INVALID (null, bad partition, rope_theta <= 1), ALIGN, UNSUPPORTED
+ * (n_ctx above max_ctx, L above max_len), DEVICE, CUDA. */
+int sagekv_compact_window_rope(sagekv_ctx *ctx, const void *K_pre, const void *V, sagekv_strides ks,
+                               int64_t n_ctx, int32_t n_init, int32_t n_recent, float rope_theta,
+                               void *Kc, void *Vc, sagekv_strides cs, sagekv_cache_state *state, void *stream);
+
 /* Optional hint from the score step to the select step (no counterpart in the
  * paper; it changes no result).  Off by default: sagekv_score then writes, and
  * sagekv_select_compact reads, nothing but the E scores of each row, whatever

@@ -57,6 +57,13 @@ lib.sagekv_set_select_hint.argtypes = [_vp, C.c_int, _i32]
 lib.sagekv_set_select_hint.restype = C.c_int
 lib.sagekv_scores_row_stride.argtypes = [_vp, _i64, _i32, _i32]
 lib.sagekv_scores_row_stride.restype = _i64
+lib.sagekv_set_group_mode.argtypes = [_vp, C.c_int]
+lib.sagekv_set_group_mode.restype = C.c_int
+lib.sagekv_pool_scores.argtypes = [_vp, _vp, _i64, _i64, _i32, _i32, _vp, _i64, _vp]
+lib.sagekv_pool_scores.restype = C.c_int
+lib.sagekv_compact_window_rope.argtypes = [_vp, _vp, _vp, Strides, _i64, _i32, _i32, C.c_float, _vp, _vp, Strides,
+                                           C.POINTER(CacheState), _vp]
+lib.sagekv_compact_window_rope.restype = C.c_int
 lib.sagekv_status.argtypes = [_vp, C.POINTER(_i32)]
 lib.sagekv_status.restype = C.c_int
 lib.sagekv_status_code.argtypes = [_i32]
@@ -136,6 +143,23 @@ def sagekv_scores_row_stride(ctx, n_ctx: int, n_init: int, n_recent: int) -> int
     if r < 0:
         _check(int(r), "sagekv_scores_row_stride", ctx)
     return int(r)
+
+
+def sagekv_set_group_mode(ctx, mode: int):
+    _check(lib.sagekv_set_group_mode(ctx, mode), "sagekv_set_group_mode", ctx)
+
+
+def sagekv_pool_scores(ctx, scores, scores_row_stride: int, n_ctx: int, n_init: int, n_recent: int, pooled,
+                       pooled_row_stride: int):
+    _check(lib.sagekv_pool_scores(ctx, _ptr(scores), scores_row_stride, n_ctx, n_init, n_recent, _ptr(pooled),
+                                  pooled_row_stride, _stream()), "sagekv_pool_scores", ctx)
+
+
+def sagekv_compact_window_rope(ctx, K_pre, V, n_ctx: int, n_init: int, n_recent: int, rope_theta: float, Kc, Vc,
+                               state: CacheState):
+    _check(lib.sagekv_compact_window_rope(ctx, _ptr(K_pre), _ptr(V), _kv_strides(K_pre), n_ctx, n_init, n_recent,
+                                          rope_theta, _ptr(Kc), _ptr(Vc), _kv_strides(Kc), C.byref(state), _stream()),
+           "sagekv_compact_window_rope", ctx)
 
 
 def sagekv_status(ctx) -> int:

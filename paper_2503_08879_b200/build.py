@@ -12,7 +12,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsagekv.so")
 LIB_CHECKED = os.path.join(HERE, "libsagekv_checked.so")   # the same interface built with -DSAGEKV_CHECKS
-SOURCES = ["api.cu", "score.cu", "score_static.cu", "select_compact.cu", "decode_attn.cu"]
+SOURCES = ["api.cu", "score.cu", "score_static.cu", "select_compact.cu", "decode_attn.cu", "variants.cu"]
 
 
 def nvcc_path() -> str:

@@ -25,6 +25,7 @@ struct sagekv_ctx {
   int overlap;              // 0, 1 or 2: see sagekv_set_overlap
   int hint;                 // 0, 1, 2: see sagekv_set_select_hint
   int32_t hint_k;
+  int group_mode;           // 0: a selection per query head (the paper's), 1: one per KV head from pooled scores
 };
 
 namespace {
@@ -89,6 +90,7 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   ctx->overlap = 0;
   ctx->hint = 0;
   ctx->hint_k = 0;
+  ctx->group_mode = 0;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || device_setup(dev, &ctx->dev) != cudaSuccess) {
     delete ctx;
@@ -188,17 +190,18 @@ int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_r
   if (ctx == nullptr || K == nullptr || V == nullptr || Kc == nullptr || Vc == nullptr || state == nullptr ||
       state->d_step == nullptr)
     return SAGEKV_ERR_INVALID;
-  if (n_init < 0 || n_recent < 0 || k < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx ||
-      k % ctx->G != 0)
+  const bool pooled = ctx->group_mode == 1;
+  const int G = pooled ? 1 : ctx->G;                    // pooled: one score row and one list per KV head
+  if (n_init < 0 || n_recent < 0 || k < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx || k % G != 0)
     return SAGEKV_ERR_INVALID;
   if (n_ctx > ctx->max_ctx) return SAGEKV_ERR_UNSUPPORTED;
   if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
   const int64_t E = n_ctx - 1 - n_init - n_recent;
-  int64_t k_q = k / ctx->G;
+  int64_t k_q = k / G;
   if (k_q > E) k_q = E;
   if (k_q > 0 && (scores == nullptr || idx == nullptr || scores_row_stride < E)) return SAGEKV_ERR_INVALID;
   if (ks.token_stride < kHeadDim || cs.token_stride < kHeadDim) return SAGEKV_ERR_INVALID;
-  const int64_t L = (int64_t)n_init + ctx->G * k_q + n_recent + 1;
+  const int64_t L = (int64_t)n_init + G * k_q + n_recent + 1;
   if (L > ctx->max_len) return SAGEKV_ERR_UNSUPPORTED;
   if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !strides_ok(ks) || !strides_ok(cs) ||
       (k_q > 0 && (!aligned16(scores) || scores_row_stride % 4 != 0)))
@@ -219,18 +222,18 @@ int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_r
   p.R = n_recent;
   p.N = (int)n_ctx;
   p.k_q = (int)k_q;
-  p.G = ctx->G;
-  p.H_q = ctx->shape.n_q_heads;
+  p.G = G;
+  p.H_q = pooled ? ctx->shape.n_kv_heads : ctx->shape.n_q_heads;
   p.H_kv = ctx->shape.n_kv_heads;
   p.B = ctx->shape.batch;
   p.status = ctx->status;
-  p.sketch = ctx->hint == 1;
-  p.list = ctx->hint == 2 && k == ctx->hint_k;
+  p.sketch = !pooled && ctx->hint == 1;
+  p.list = !pooled && ctx->hint == 2 && k == ctx->hint_k;
   const cudaError_t e = launch_select_compact(p, ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   state->n_init = n_init;
   state->k_q = (int32_t)k_q;
-  state->n_sel = (int32_t)(ctx->G * k_q);
+  state->n_sel = (int32_t)(G * k_q);
   state->n_recent = n_recent;
   state->ring_len = n_recent + 1;
   state->len = (int32_t)L;
@@ -243,7 +246,8 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
     return SAGEKV_ERR_INVALID;
   if ((k_new == nullptr) != (v_new == nullptr)) return SAGEKV_ERR_INVALID;
   if (k_new != nullptr && state->d_step == nullptr) return SAGEKV_ERR_INVALID;
-  if (state->n_init < 0 || state->k_q < 0 || state->n_recent < 0 || state->n_sel != ctx->G * state->k_q ||
+  const bool pooled = ctx->group_mode == 1;
+  if (state->n_init < 0 || state->k_q < 0 || state->n_recent < 0 || state->n_sel != (pooled ? 1 : ctx->G) * state->k_q ||
       state->ring_len != state->n_recent + 1 || state->len != state->n_init + state->n_sel + state->ring_len ||
       cs.token_stride < kHeadDim)
     return SAGEKV_ERR_INVALID;
@@ -276,6 +280,7 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
   p.B = ctx->shape.batch;
   p.scale_log2 = ctx->scale * kLog2e;
   p.pdl_mode = ctx->overlap;
+  p.pooled = pooled ? 1 : 0;
   const cudaError_t e = launch_decode(p, *ctx->dev, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
 }
@@ -283,6 +288,66 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
 int sagekv_set_overlap(sagekv_ctx *ctx, int mode) {
   if (ctx == nullptr || mode < 0 || mode > 2) return SAGEKV_ERR_INVALID;
   ctx->overlap = mode;
+  return SAGEKV_OK;
+}
+
+int sagekv_set_group_mode(sagekv_ctx *ctx, int mode) {
+  if (ctx == nullptr || mode < 0 || mode > 1) return SAGEKV_ERR_INVALID;
+  ctx->group_mode = mode;
+  return SAGEKV_OK;
+}
+
+int sagekv_pool_scores(sagekv_ctx *ctx, const float *scores, int64_t scores_row_stride, int64_t n_ctx, int32_t n_init,
+                       int32_t n_recent, float *pooled, int64_t pooled_row_stride, void *stream) {
+  if (ctx == nullptr || scores == nullptr || pooled == nullptr) return SAGEKV_ERR_INVALID;
+  if (n_init < 0 || n_recent < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx) return SAGEKV_ERR_INVALID;
+  if (n_ctx > ctx->max_ctx) return SAGEKV_ERR_UNSUPPORTED;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
+  const int64_t E = n_ctx - 1 - n_init - n_recent;
+  if (scores_row_stride < E || pooled_row_stride < E) return SAGEKV_ERR_INVALID;
+  if (!aligned16(scores) || !aligned16(pooled) || scores_row_stride % 4 != 0 || pooled_row_stride % 4 != 0) return SAGEKV_ERR_ALIGN;
+  const cudaError_t e = launch_pool_scores(scores, scores_row_stride, pooled, pooled_row_stride, (int)E, ctx->G,
+                                           ctx->shape.batch * ctx->shape.n_kv_heads, ctx->dev->n_sm,
+                                           static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
+}
+
+int sagekv_compact_window_rope(sagekv_ctx *ctx, const void *K_pre, const void *V, sagekv_strides ks, int64_t n_ctx,
+                               int32_t n_init, int32_t n_recent, float rope_theta, void *Kc, void *Vc, sagekv_strides cs,
+                               sagekv_cache_state *state, void *stream) {
+  if (ctx == nullptr || K_pre == nullptr || V == nullptr || Kc == nullptr || Vc == nullptr || state == nullptr ||
+      state->d_step == nullptr)
+    return SAGEKV_ERR_INVALID;
+  if (n_init < 0 || n_recent < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx || !(rope_theta > 1.f) ||
+      ks.token_stride < kHeadDim || cs.token_stride < kHeadDim)
+    return SAGEKV_ERR_INVALID;
+  if (n_ctx > ctx->max_ctx || (int64_t)n_init + n_recent + 1 > ctx->max_len) return SAGEKV_ERR_UNSUPPORTED;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
+  if (!aligned16(K_pre) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !strides_ok(ks) || !strides_ok(cs))
+    return SAGEKV_ERR_ALIGN;
+  WindowRopeParams p;
+  p.K = static_cast<const uint16_t *>(K_pre);
+  p.V = static_cast<const uint16_t *>(V);
+  p.ks = ks;
+  p.Kc = static_cast<uint16_t *>(Kc);
+  p.Vc = static_cast<uint16_t *>(Vc);
+  p.cs = cs;
+  p.d_step = state->d_step;
+  p.status = ctx->status;
+  p.S = n_init;
+  p.R = n_recent;
+  p.N = (int)n_ctx;
+  p.H_kv = ctx->shape.n_kv_heads;
+  p.B = ctx->shape.batch;
+  p.theta = rope_theta;
+  const cudaError_t e = launch_compact_window_rope(p, ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  state->n_init = n_init;
+  state->k_q = 0;
+  state->n_sel = 0;
+  state->n_recent = n_recent;
+  state->ring_len = n_recent + 1;
+  state->len = n_init + n_recent + 1;
   return SAGEKV_OK;
 }
 

@@ -97,6 +97,21 @@ cudaError_t select_compact_setup();   // one-time function attributes
 // second pass of the score step in hint mode 2: normalise the rows and leave the candidate lists behind them
 cudaError_t launch_score_finalize_candidates(const ScoreParams &p, cudaStream_t stream);
 
+// ---- comparison paths (variants.cu) -----------------------------------------
+struct WindowRopeParams {
+  const uint16_t *K, *V;   // K before rotary embedding
+  sagekv_strides ks;
+  uint16_t *Kc, *Vc;
+  sagekv_strides cs;
+  int32_t *d_step;
+  int32_t *status;
+  int S, R, N, H_kv, B;
+  float theta;
+};
+cudaError_t launch_compact_window_rope(const WindowRopeParams &p, int n_sm, cudaStream_t stream);
+cudaError_t launch_pool_scores(const float *scores, int64_t row_stride, float *pooled, int64_t pooled_stride, int E, int G,
+                               int n_groups, int n_sm, cudaStream_t stream);
+
 // ---- decode attention ------------------------------------------------------
 #if !defined(SAGEKV_DECODE_WARPS)
 #define SAGEKV_DECODE_WARPS 8
@@ -123,6 +138,7 @@ struct DecodeParams {
   int S, k_q, n_sel, ring_len, L, G, H_q, H_kv, B;
   float scale_log2;
   int pdl_mode;            // 0 plain launch, 1 programmatic dependent launch, 2 also fetch the cache before the wait
+  int pooled;              // 1: every query head sees all selected rows of its KV head (k_q = n_sel), 0: its own segment
 };
 
 // What the one-time set-up of a device leaves behind (function attributes are set as a side effect).

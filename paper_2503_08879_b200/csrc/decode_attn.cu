@@ -209,7 +209,8 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   // (1) which of this lane's score elements are visible to their heads (sink, own segment, window): bit 4i + e
   //     for the warp's i-th tile of the round, element e of the accumulator
   const int win_lo = p.S + p.n_sel;
-  const int seg0_lo = p.S + h0 * p.k_q, seg0_hi = seg0_lo + p.k_q, seg1_lo = seg0_hi, seg1_hi = seg1_lo + p.k_q;
+  const int seg0_lo = p.S + (p.pooled ? 0 : h0 * p.k_q), seg0_hi = seg0_lo + p.k_q;
+  const int seg1_lo = p.S + (p.pooled ? 0 : h1 * p.k_q), seg1_hi = seg1_lo + p.k_q;
   auto visibility = [&](int t0) {
     uint32_t bits = 0;
 #pragma unroll
