@@ -24,7 +24,8 @@ Positions are 0-based here: sink [0,S), eviction region [S,S+E), recent window
 
 Section 3.1's baselines that are restated here for the comparison paths: StreamLLM_R
 (rope_rotate, compact_window_rope: Appendix A.1) and the pooled reading of
-Step 2 (select_pooled, compact_pooled, decode_step_pooled).
+Step 2 (select_pooled, compact_pooled, decode_step_pooled), and a Quest-style block-wise
+per-step selection (quest_*), the comparison system of Section 3.1.
 
 Pins (tests/test_oracle_pins.py): budget_split <- the numbers Appendix A.2
 prints; score <- closed forms (uniform keys, one planted key), row sums, a
@@ -56,6 +57,10 @@ __all__ = [
     "select_pooled",
     "compact_pooled",
     "decode_step_pooled",
+    "quest_summaries",
+    "quest_bounds",
+    "quest_select",
+    "quest_attention",
 ]
 
 
@@ -386,3 +391,71 @@ def decode_step_pooled(q_bits: np.ndarray, k_new_bits, v_new_bits, Kc: np.ndarra
         step = step + 1
     o, lse = full_attention(bf16_bits_to_f64(q_bits), bf16_bits_to_f64(Kc), bf16_bits_to_f64(Vc), keep=None, scale=scale)
     return o, lse, step
+
+
+# --------------------------------------------------------------------------
+# Quest-style comparator (Section 3.1 "Baselines": a block-wise top-k selection
+# method, run at every decode step on the FULL cache)
+# --------------------------------------------------------------------------
+
+def quest_summaries(K_bits: np.ndarray, S: int, R: int, block: int = 16) -> tuple[np.ndarray, np.ndarray]:
+    """Element-wise minimum and maximum of the keys of every block of `block`
+    consecutive tokens of the eviction region [S, S+E) (the last block may be
+    shorter).  K_bits uint16 [H_kv, N, d].  Returns (kmin, kmax) as bf16 bit
+    patterns [H_kv, n_blocks, d], n_blocks = ceil(E / block); minima and maxima
+    of bf16 values are bf16 values, so nothing is rounded.
+    """
+    H_kv, N, d = K_bits.shape
+    part = partition(N, S, R)
+    E = part["E"]
+    n_blocks = (E + block - 1) // block
+    kmin = np.zeros((H_kv, n_blocks, d), dtype=np.uint16)
+    kmax = np.zeros((H_kv, n_blocks, d), dtype=np.uint16)
+    for g in range(H_kv):
+        for j in range(n_blocks):
+            lo, hi = S + j * block, min(S + E, S + (j + 1) * block)
+            x = bf16_bits_to_f64(K_bits[g, lo:hi])
+            kmin[g, j] = f64_to_bf16_bits(x.min(axis=0))
+            kmax[g, j] = f64_to_bf16_bits(x.max(axis=0))
+    return kmin, kmax
+
+
+def quest_bounds(q_bits: np.ndarray, kmin_bits: np.ndarray, kmax_bits: np.ndarray,
+                 scale: float | None = None) -> np.ndarray:
+    """Upper bound of the attention logit of any token of a block:
+        u[h, j] = scale * sum_c max(q[h, c] * kmin[h // G, j, c], q[h, c] * kmax[h // G, j, c])
+    float64 [H_q, n_blocks]."""
+    q = bf16_bits_to_f64(q_bits)
+    H_q, d = q.shape
+    H_kv, n_blocks, _ = kmin_bits.shape
+    G = H_q // H_kv
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    lo, hi = bf16_bits_to_f64(kmin_bits), bf16_bits_to_f64(kmax_bits)
+    u = np.zeros((H_q, n_blocks), dtype=np.float64)
+    for h in range(H_q):
+        g = h // G
+        u[h] = np.sum(np.maximum(q[h] * lo[g], q[h] * hi[g]), axis=-1) * scale
+    return u
+
+
+def quest_select(u: np.ndarray, n_keep: int) -> np.ndarray:
+    """The n_keep blocks of largest bound per query head (ties: lower block), ascending.  int32 [H_q, min(n_keep, n_blocks)]."""
+    return select(u, n_keep, 0)
+
+
+def quest_attention(q_bits: np.ndarray, K_bits: np.ndarray, V_bits: np.ndarray, blocks: np.ndarray,
+                    S: int, R: int, block: int = 16, scale: float | None = None) -> np.ndarray:
+    """Attention of every query head over sink + the tokens of its selected blocks + recent window + last token of
+    the full cache.  float64 [H_q, d]."""
+    H_kv, N, d = K_bits.shape
+    H_q = q_bits.shape[0]
+    E = partition(N, S, R)["E"]
+    keep = np.zeros((H_q, N), dtype=bool)
+    keep[:, :S] = True
+    keep[:, S + E:] = True
+    for h in range(H_q):
+        for j in blocks[h]:
+            keep[h, S + int(j) * block: min(S + E, S + (int(j) + 1) * block)] = True
+    o, _ = full_attention(bf16_bits_to_f64(q_bits), bf16_bits_to_f64(K_bits), bf16_bits_to_f64(V_bits), keep=keep, scale=scale)
+    return o

@@ -396,3 +396,45 @@ def test_decode_pooled_equals_full_attention_over_the_kept_rows():
             torch.from_numpy(bf16_val(V[g, rows]))[None])[0, 0]
         np.testing.assert_allclose(o[h], want.numpy(), atol=1e-10)
     assert step == 0
+
+
+# ---------------------------------------------------------------- Quest-style block selection
+
+def test_quest_bound_dominates_every_token_and_is_tight_for_single_token_blocks():
+    rng = np.random.default_rng(51)
+    Hq, Hkv, N, d, S, R = 4, 2, 133, 16, 3, 6
+    K, q = rand_bits(rng, Hkv, N, d), rand_bits(rng, Hq, d)
+    E = N - 1 - S - R
+    kmin, kmax = O.quest_summaries(K, S, R, block=16)
+    assert kmin.shape == (Hkv, (E + 15) // 16, d)
+    u = O.quest_bounds(q, kmin, kmax)
+    logits = np.einsum("hc,htc->ht", bf16_val(q), bf16_val(K)[np.repeat(np.arange(Hkv), 2)]) / math.sqrt(d)
+    for h in range(Hq):
+        for j in range(u.shape[1]):
+            blk = logits[h, S + 16 * j: min(S + E, S + 16 * (j + 1))]
+            assert np.all(blk <= u[h, j] + 1e-12)
+    # the summaries themselves, block by block, from torch's own bf16 arithmetic
+    kv = torch.from_numpy(bf16_val(K))
+    assert np.array_equal(bf16_val(kmin[1, 2]), kv[1, S + 32: S + 48].min(dim=0).values.numpy())
+    assert np.array_equal(bf16_val(kmax[0, -1]), kv[0, S + 16 * (u.shape[1] - 1): S + E].max(dim=0).values.numpy())
+    # blocks of one token: the bound is the logit itself
+    kmin1, kmax1 = O.quest_summaries(K, S, R, block=1)
+    np.testing.assert_allclose(O.quest_bounds(q, kmin1, kmax1), logits[:, S:S + E], atol=1e-12)
+
+
+def test_quest_attention_is_masked_full_attention():
+    rng = np.random.default_rng(52)
+    Hq, Hkv, N, d, S, R = 4, 2, 90, 16, 2, 5
+    K, V, q = rand_bits(rng, Hkv, N, d), rand_bits(rng, Hkv, N, d), rand_bits(rng, Hq, d)
+    kmin, kmax = O.quest_summaries(K, S, R)
+    blocks = O.quest_select(O.quest_bounds(q, kmin, kmax), 2)
+    assert blocks.shape == (Hq, 2) and np.all(np.diff(blocks, axis=1) > 0)
+    o = O.quest_attention(q, K, V, blocks, S, R)
+    E = N - 1 - S - R
+    for h in range(Hq):
+        g = h // 2
+        rows = list(range(S)) + [t for j in blocks[h] for t in range(S + 16 * j, min(S + E, S + 16 * (j + 1)))] + list(range(S + E, N))
+        want = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(bf16_val(q[h]))[None, None], torch.from_numpy(bf16_val(K[g, rows]))[None],
+            torch.from_numpy(bf16_val(V[g, rows]))[None])[0, 0]
+        np.testing.assert_allclose(o[h], want.numpy(), atol=1e-10)
