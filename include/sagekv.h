@@ -226,6 +226,36 @@ int sagekv_compact_window_rope(sagekv_ctx *ctx, const void *K_pre, const void *V
                                int64_t n_ctx, int32_t n_init, int32_t n_recent, float rope_theta,
                                void *Kc, void *Vc, sagekv_strides cs, sagekv_cache_state *state, void *stream);
 
+/* ---- A Quest-style comparator (Section 3.1 "Baselines": a block-wise top-k
+ * selection method; Section 3.2 compares memory efficiency with it).  It keeps
+ * the FULL cache and selects blocks anew at every decode step; these three calls
+ * are its selection half, on the same data layout as the method's own calls.
+ *
+ * sagekv_quest_build: per block of SAGEKV_QUEST_BLOCK = 16 consecutive tokens of
+ * the eviction region (the last block may be shorter), the element-wise minimum
+ * and maximum of the keys.  kmin, kmax  bf16 [batch, H_kv, n_blocks, 128]
+ * contiguous, n_blocks = ceil(E / 16); exact (no rounding).  Built once.
+ * Errors: INVALID, ALIGN, UNSUPPORTED (n_ctx above max_ctx), DEVICE, CUDA. */
+#define SAGEKV_QUEST_BLOCK 16
+int sagekv_quest_build(sagekv_ctx *ctx, const void *K, sagekv_strides ks, int64_t n_ctx, int32_t n_init,
+                       int32_t n_recent, void *kmin, void *kmax, void *stream);
+
+/* Per decode step: bounds[b*H_q + h][j] = scale * sum_c max(q[b,h,c]*kmin[b,h/G,j,c],
+ * q[b,h,c]*kmax[b,h/G,j,c]), an upper bound of the attention logit of every token of
+ * block j (fp32 products and sums).  bounds: batch*H_q rows of stride
+ * bounds_row_stride >= n_blocks.  Errors: INVALID, ALIGN, DEVICE, CUDA. */
+int sagekv_quest_bounds(sagekv_ctx *ctx, const void *q, const void *kmin, const void *kmax, int64_t n_blocks,
+                        float *bounds, int64_t bounds_row_stride, void *stream);
+
+/* The selection of sagekv_select_compact without the gather: per row of `scores`
+ * (batch*H_q rows of n values, stride scores_row_stride, a multiple of 4; base
+ * 16-byte aligned) the min(k_q, n) largest, lower index winning ties, written
+ * ascending as 0-based indices to idx [batch*H_q, min(k_q, n)].  n may not exceed
+ * the context's max_ctx.  Used for the comparator's block selection.
+ * Errors: INVALID, ALIGN, UNSUPPORTED, DEVICE, CUDA. */
+int sagekv_select_topk(sagekv_ctx *ctx, const float *scores, int64_t scores_row_stride, int64_t n,
+                       int32_t k_q, int32_t *idx, void *stream);
+
 /* Optional hint from the score step to the select step (no counterpart in the
  * paper; it changes no result).  Off by default: sagekv_score then writes, and
  * sagekv_select_compact reads, nothing but the E scores of each row, whatever

@@ -64,6 +64,12 @@ lib.sagekv_pool_scores.restype = C.c_int
 lib.sagekv_compact_window_rope.argtypes = [_vp, _vp, _vp, Strides, _i64, _i32, _i32, C.c_float, _vp, _vp, Strides,
                                            C.POINTER(CacheState), _vp]
 lib.sagekv_compact_window_rope.restype = C.c_int
+lib.sagekv_quest_build.argtypes = [_vp, _vp, Strides, _i64, _i32, _i32, _vp, _vp, _vp]
+lib.sagekv_quest_build.restype = C.c_int
+lib.sagekv_quest_bounds.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]
+lib.sagekv_quest_bounds.restype = C.c_int
+lib.sagekv_select_topk.argtypes = [_vp, _vp, _i64, _i64, _i32, _vp, _vp]
+lib.sagekv_select_topk.restype = C.c_int
 lib.sagekv_status.argtypes = [_vp, C.POINTER(_i32)]
 lib.sagekv_status.restype = C.c_int
 lib.sagekv_status_code.argtypes = [_i32]
@@ -160,6 +166,21 @@ def sagekv_compact_window_rope(ctx, K_pre, V, n_ctx: int, n_init: int, n_recent:
     _check(lib.sagekv_compact_window_rope(ctx, _ptr(K_pre), _ptr(V), _kv_strides(K_pre), n_ctx, n_init, n_recent,
                                           rope_theta, _ptr(Kc), _ptr(Vc), _kv_strides(Kc), C.byref(state), _stream()),
            "sagekv_compact_window_rope", ctx)
+
+
+def sagekv_quest_build(ctx, K, n_ctx: int, n_init: int, n_recent: int, kmin, kmax):
+    _check(lib.sagekv_quest_build(ctx, _ptr(K), _kv_strides(K), n_ctx, n_init, n_recent, _ptr(kmin), _ptr(kmax), _stream()),
+           "sagekv_quest_build", ctx)
+
+
+def sagekv_quest_bounds(ctx, q, kmin, kmax, n_blocks: int, bounds, bounds_row_stride: int):
+    _check(lib.sagekv_quest_bounds(ctx, _ptr(q), _ptr(kmin), _ptr(kmax), n_blocks, _ptr(bounds), bounds_row_stride,
+                                   _stream()), "sagekv_quest_bounds", ctx)
+
+
+def sagekv_select_topk(ctx, scores, scores_row_stride: int, n: int, k_q: int, idx):
+    _check(lib.sagekv_select_topk(ctx, _ptr(scores), scores_row_stride, n, k_q, _ptr(idx), _stream()),
+           "sagekv_select_topk", ctx)
 
 
 def sagekv_status(ctx) -> int:

@@ -351,6 +351,57 @@ int sagekv_compact_window_rope(sagekv_ctx *ctx, const void *K_pre, const void *V
   return SAGEKV_OK;
 }
 
+int sagekv_quest_build(sagekv_ctx *ctx, const void *K, sagekv_strides ks, int64_t n_ctx, int32_t n_init, int32_t n_recent,
+                       void *kmin, void *kmax, void *stream) {
+  if (ctx == nullptr || K == nullptr || kmin == nullptr || kmax == nullptr) return SAGEKV_ERR_INVALID;
+  if (n_init < 0 || n_recent < 0 || n_ctx < 1 || (int64_t)n_init + n_recent + 1 > n_ctx || ks.token_stride < kHeadDim)
+    return SAGEKV_ERR_INVALID;
+  if (n_ctx > ctx->max_ctx) return SAGEKV_ERR_UNSUPPORTED;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
+  if (!aligned16(K) || !aligned16(kmin) || !aligned16(kmax) || !strides_ok(ks)) return SAGEKV_ERR_ALIGN;
+  const int64_t E = n_ctx - 1 - n_init - n_recent;
+  const cudaError_t e = launch_quest_build(static_cast<const uint16_t *>(K), ks, static_cast<uint16_t *>(kmin),
+                                           static_cast<uint16_t *>(kmax), n_init, (int)E, ctx->shape.n_kv_heads,
+                                           ctx->shape.batch, ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
+}
+
+int sagekv_quest_bounds(sagekv_ctx *ctx, const void *q, const void *kmin, const void *kmax, int64_t n_blocks, float *bounds,
+                        int64_t bounds_row_stride, void *stream) {
+  if (ctx == nullptr || q == nullptr || kmin == nullptr || kmax == nullptr || bounds == nullptr || n_blocks < 0 ||
+      bounds_row_stride < n_blocks || n_blocks > (int64_t)1 << 28)
+    return SAGEKV_ERR_INVALID;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
+  if (!aligned16(q) || !aligned16(kmin) || !aligned16(kmax)) return SAGEKV_ERR_ALIGN;
+  const cudaError_t e = launch_quest_bounds(static_cast<const uint16_t *>(q), static_cast<const uint16_t *>(kmin),
+                                            static_cast<const uint16_t *>(kmax), bounds, bounds_row_stride, (int)n_blocks,
+                                            ctx->G, ctx->shape.n_q_heads, ctx->shape.n_kv_heads, ctx->shape.batch, ctx->scale,
+                                            ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
+}
+
+int sagekv_select_topk(sagekv_ctx *ctx, const float *scores, int64_t scores_row_stride, int64_t n, int32_t k_q, int32_t *idx,
+                       void *stream) {
+  if (ctx == nullptr || scores == nullptr || idx == nullptr || n < 1 || k_q < 1 || scores_row_stride < n) return SAGEKV_ERR_INVALID;
+  if (n > ctx->max_ctx) return SAGEKV_ERR_UNSUPPORTED;
+  if (!on_own_device(ctx)) return SAGEKV_ERR_DEVICE;
+  if (!aligned16(scores) || scores_row_stride % 4 != 0) return SAGEKV_ERR_ALIGN;
+  SelectParams p = {};
+  p.scores = scores;
+  p.row_stride = scores_row_stride;
+  p.idx = idx;
+  p.E = (int)n;
+  p.N = (int)n + 1;
+  p.k_q = (int)(k_q < n ? k_q : n);
+  p.G = ctx->G;
+  p.H_q = ctx->shape.n_q_heads;
+  p.H_kv = ctx->shape.n_kv_heads;
+  p.B = ctx->shape.batch;
+  p.status = ctx->status;
+  const cudaError_t e = launch_select_compact(p, ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
+}
+
 int sagekv_set_select_hint(sagekv_ctx *ctx, int mode, int32_t k) {
   if (ctx == nullptr || mode < 0 || mode > 2 || k < 0 || k % ctx->G != 0 || (mode == 2 && k == 0)) return SAGEKV_ERR_INVALID;
   ctx->hint = mode;

@@ -112,6 +112,12 @@ cudaError_t launch_compact_window_rope(const WindowRopeParams &p, int n_sm, cuda
 cudaError_t launch_pool_scores(const float *scores, int64_t row_stride, float *pooled, int64_t pooled_stride, int E, int G,
                                int n_groups, int n_sm, cudaStream_t stream);
 
+constexpr int kQuestBlock = 16;   // tokens per block of the Quest-style summaries (SAGEKV_QUEST_BLOCK)
+cudaError_t launch_quest_build(const uint16_t *K, sagekv_strides ks, uint16_t *kmin, uint16_t *kmax, int S, int E, int H_kv,
+                               int B, int n_sm, cudaStream_t stream);
+cudaError_t launch_quest_bounds(const uint16_t *q, const uint16_t *kmin, const uint16_t *kmax, float *u, int64_t u_stride,
+                                int n_blocks, int G, int H_q, int H_kv, int B, float scale, int n_sm, cudaStream_t stream);
+
 // ---- decode attention ------------------------------------------------------
 #if !defined(SAGEKV_DECODE_WARPS)
 #define SAGEKV_DECODE_WARPS 8

@@ -790,14 +790,15 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
 
   // gather the rows on this CTA's list into head j's segment of the reduced cache: a warp moves four rows at a
   // time (K in lanes 0-15, V in lanes 16-31), all loads issued before the stores
-  const int n_list = min(sh.list_count, list_cap);
+  const bool gather = p.Kc != nullptr;                   // null: the caller wants the indices only
+  const int n_list = gather ? min(sh.list_count, list_cap) : 0;
   const uint16_t *src_base = (lane < 16 ? p.K : p.V) + (int64_t)b * p.ks.batch_stride + (int64_t)kvh * p.ks.head_stride +
                              (lane & 15) * 8;
   uint16_t *dst_base = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
                        ((int64_t)p.S + (int64_t)j * p.k_q) * p.cs.token_stride + (lane & 15) * 8;
   // The sink, recent and last rows of the KV head (positions known without the scores) are shared out over the
   // warps of the head's G clusters, at most one row per warp per round, loaded together with the first batch.
-  const int n_static = p.S + p.R + 1;
+  const int n_static = gather ? p.S + p.R + 1 : 0;
   const int static_stride = p.G * cs * kSelWarps;
   int sr = (j * cs + rank) * kSelWarps + warp;           // this warp's first static row
   for (int e0 = warp * 4; e0 < n_list || sr < n_static; e0 += kSelWarps * 4) {
@@ -828,7 +829,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
       sr += static_stride;
     }
   }
-  if (cid == 0 && rank == 0 && tid == 0) *p.d_step = 0;
+  if (cid == 0 && rank == 0 && tid == 0 && p.d_step != nullptr) *p.d_step = 0;
   if (exit_wait) cluster.barrier_wait();   // prefilter path: a peer may still have been copying this CTA's candidates
 }
 

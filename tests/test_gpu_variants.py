@@ -134,3 +134,53 @@ def test_pooled_group_mode_matches_the_oracle(B, name, kw, K_sel):
         check_out(out[b], ref)
     assert sk.status() == 0
     sk.close()
+
+
+@pytest.mark.parametrize("name,kw", [("C1", dict()), ("C4-b1", dict(n_ctx=20000, batch=2)), ("C2", dict(n_ctx=32768 - 7))])
+def test_quest_style_block_selection_matches_the_oracle(B, name, kw):
+    """Block summaries bit-exact (minima and maxima of bf16 values are not rounded), bounds within 1e-3 of the sum of
+    the absolute terms (fp32 sums of 128 products), block selection bit-exact on the GPU's own bounds and, against
+    the oracle's bounds, different only for blocks whose bound is within that tolerance of the cut."""
+    w = synth.workload(name).with_(n_layers=1, **kw)
+    dev = "cuda"
+    lay = synth.make_layer(w, 0, dev)
+    S, R, E = w.n_init, w.n_recent, w.E
+    nb = (E + 15) // 16
+    keep = max(1, w.k_q // 16)
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, 128, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    kmin = torch.full((w.batch, w.n_kv_heads, nb + 1, 128), 3.0, dtype=torch.bfloat16, device=dev)
+    kmax = torch.full_like(kmin, 3.0)
+    B.sagekv_quest_build(sk.ctx, lay["K"], w.n_ctx, S, R, kmin, kmax)
+    torch.cuda.synchronize()
+    # the kernel writes [batch, H_kv, nb, 128] contiguous: view the buffers that way
+    km = kmin.flatten()[: w.batch * w.n_kv_heads * nb * 128].view(w.batch, w.n_kv_heads, nb, 128)
+    kM = kmax.flatten()[: w.batch * w.n_kv_heads * nb * 128].view(w.batch, w.n_kv_heads, nb, 128)
+    assert (kmin.flatten()[w.batch * w.n_kv_heads * nb * 128:] == 3.0).all()             # nothing written behind
+    stride = (nb + 3) // 4 * 4
+    u = torch.full((w.batch * w.n_q_heads, stride), 7.5, dtype=torch.float32, device=dev)
+    B.sagekv_quest_bounds(sk.ctx, lay["q_last"], km, kM, nb, u, stride)
+    idx = torch.full((w.batch * w.n_q_heads, keep + 1), -7, dtype=torch.int32, device=dev)
+    B.sagekv_select_topk(sk.ctx, u, stride, nb, keep, idx.flatten()[: w.batch * w.n_q_heads * keep].view(-1, keep))
+    torch.cuda.synchronize()
+    assert (u[:, nb:] == 7.5).all()
+    got_idx = idx.flatten()[: w.batch * w.n_q_heads * keep].view(w.batch, w.n_q_heads, keep).cpu().numpy()
+    assert (idx.flatten()[w.batch * w.n_q_heads * keep:] == -7).all()
+    for b in range(w.batch):
+        rmin, rmax = O.quest_summaries(bits(lay["K"][b]), S, R)
+        assert np.array_equal(bits(km[b]), rmin) and np.array_equal(bits(kM[b]), rmax)
+        ref_u = O.quest_bounds(bits(lay["q_last"][b]), rmin, rmax)
+        got_u = u.view(w.batch, w.n_q_heads, stride)[b, :, :nb].cpu().numpy()
+        qf = O.bf16_bits_to_f64(bits(lay["q_last"][b]))
+        G = w.G
+        for h in range(w.n_q_heads):
+            mag = np.sum(np.maximum(np.abs(qf[h] * O.bf16_bits_to_f64(rmin[h // G])), np.abs(qf[h] * O.bf16_bits_to_f64(rmax[h // G]))),
+                         axis=-1) / np.sqrt(128.0)
+            assert np.all(np.abs(got_u[h] - ref_u[h]) <= 1e-3 * mag + 1e-6)
+        assert np.array_equal(got_idx[b], O.quest_select(got_u, keep))
+        ref_idx = O.quest_select(ref_u, keep)
+        for h in range(w.n_q_heads):
+            diff = set(got_idx[b, h].tolist()) ^ set(ref_idx[h].tolist())
+            cut = np.sort(ref_u[h])[::-1][keep - 1]
+            assert all(abs(ref_u[h, j] - cut) <= 2e-3 * max(1.0, abs(cut)) for j in diff)
+    assert sk.status() == 0
+    sk.close()
