@@ -12,6 +12,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsagekv.so")
 LIB_CHECKED = os.path.join(HERE, "libsagekv_checked.so")   # the same interface built with -DSAGEKV_CHECKS
+LIB_TRACE = os.path.join(HERE, "libsagekv_trace.so")       # built with -DSAGEKV_TRACE: timeline stamps in the decode kernel
 SOURCES = ["api.cu", "score.cu", "score_static.cu", "select_compact.cu", "decode_attn.cu", "variants.cu"]
 
 
@@ -30,15 +31,15 @@ def needs_build(lib: str = LIB) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, checks: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, checks: bool = False, trace: bool = False) -> str:
     """checks=True builds libsagekv_checked.so: every global-memory index of the kernels is range-checked and a
     violation is reported through sagekv_status instead of being executed (load it with SAGEKV_LIB=<path>)."""
-    lib = LIB_CHECKED if checks else LIB
+    lib = LIB_TRACE if trace else (LIB_CHECKED if checks else LIB)
     if not force and not needs_build(lib):
         return lib
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", lib] + (["-DSAGEKV_CHECKS"] if checks else []) + [os.path.join(CSRC, s) for s in SOURCES]
+           "-o", lib] + (["-DSAGEKV_TRACE"] if trace else (["-DSAGEKV_CHECKS"] if checks else [])) + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -51,4 +52,4 @@ def build(force: bool = False, verbose: bool = False, checks: bool = False) -> s
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv, checks="--checks" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, checks="--checks" in sys.argv, trace="--trace" in sys.argv))

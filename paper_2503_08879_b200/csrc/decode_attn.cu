@@ -119,6 +119,34 @@ __device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
 __device__ __forceinline__ void pin(uint32_t &x) { asm volatile("" : "+r"(x)); }
 __device__ __forceinline__ void pin(int &x) { asm volatile("" : "+r"(x)); }
 
+// ---- timeline of a launch (only in a build with -DSAGEKV_TRACE; the normal build contains none of it) ----------
+// Thread 0 of every CTA notes the global timer at ten points and leaves the record in a ring in device memory,
+// which sagekv_trace_read copies out.  A stamp that has to follow a computation carries a (never true) dependence on
+// its result, so that it cannot be scheduled ahead of it.
+#if defined(SAGEKV_TRACE)
+constexpr int kTraceSlots = 1 << 15, kTraceStamps = 12;
+__device__ unsigned long long g_trace[kTraceSlots][kTraceStamps];
+__device__ unsigned int g_trace_n;
+__device__ __forceinline__ unsigned long long trace_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define SAGEKV_TRACE_BEGIN unsigned long long trace_t[kTraceStamps] = {0ull};
+#define SAGEKV_STAMP(i) do { if (threadIdx.x == 0) trace_t[i] = trace_now(); } while (0)
+#define SAGEKV_STAMP_AFTER(i, val_) do { if (threadIdx.x == 0) trace_t[i] = trace_now() + (unsigned long long)((val_) == 1.2345e-33f); } while (0)
+#define SAGEKV_TRACE_END do { if (threadIdx.x == 0) { \
+    const unsigned int slot_ = atomicAdd(&g_trace_n, 1u) % kTraceSlots; \
+    trace_t[10] = ((unsigned long long)blockIdx.x << 32) | ((unsigned long long)blockIdx.y << 16) | blockIdx.z; \
+    trace_t[11] = gridDim.x; \
+    for (int i_ = 0; i_ < kTraceStamps; ++i_) g_trace[slot_][i_] = trace_t[i_]; } } while (0)
+#else
+#define SAGEKV_TRACE_BEGIN
+#define SAGEKV_STAMP(i) do { } while (0)
+#define SAGEKV_STAMP_AFTER(i, val_) do { } while (0)
+#define SAGEKV_TRACE_END do { } while (0)
+#endif
+
 // kMulti: the CTA's range is longer than the staging area and goes through it in rounds
 template <bool kMulti>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
@@ -138,6 +166,8 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   const int h0 = 2 * c, h1 = 2 * c + 1;                           // the two heads a lane's accumulators belong to
   const int cg8 = warp & 7, half = warp >> 3;                     // second product: column group and row half of this warp
   const bool append = p.k_new != nullptr;
+  SAGEKV_TRACE_BEGIN
+  SAGEKV_STAMP(0);
 
   // tiles of this CTA: an even deal of the head's n_tiles over the gridDim.x CTAs, contiguous ranges
   const int n_tiles = (p.L + 15) >> 4;
@@ -270,10 +300,12 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   asm volatile("" : "+l"(q_lane)); pin(v_off); pin(pw_addr); pin(pr_addr); pin(dst_a); pin(dst_b); pin(bar_a); pin(bar_b); pin(dst_ml); pin(bar_ml);
   pin(vis); pin(fin_lc); pin(fin_h); asm volatile("" : "+l"(fin_out));
 
+  SAGEKV_STAMP(1);
   if (p.pdl_mode >= 2) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
+  SAGEKV_STAMP(2);
 
   // What the predecessor may have written is read now, all requests issued back to back (query first: the first
   // product needs it; the step counter last: only the patch of the replaced row needs it), so the round trips to
@@ -317,6 +349,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     const uint32_t buf_base = stage + (uint32_t)(buf * kDecodeRoundTiles * kTileBytes);
     if (kMulti && r > 0) vis = visibility(t0);
     if (nt > 0 && !mbar_wait(kbar, par)) timed_out = true;
+    if (r == 0) SAGEKV_STAMP(3);
 
     // the staged copy of the replaced row is stale: the warp that works on its tile patches K and V
     if (append && r == 0) {
@@ -406,6 +439,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       R0 = a0[0]; R1 = a1[0];
     }
     const float N0 = fmaxf(M0, R0), N1 = fmaxf(M1, R1);
+    if (r == 0) SAGEKV_STAMP_AFTER(4, N0 + N1);
     const float s0 = N0 == -INFINITY ? 0.f : N0, s1 = N1 == -INFINITY ? 0.f : N1;
     if (kMulti && r > 0) {                                 // bring sums and accumulators to the new maxima
       const float f0 = fast_exp2(M0 - s0), f1 = fast_exp2(M1 - s1);
@@ -428,6 +462,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       }
     }
     __syncthreads();   // B: the weights of the round are in shared memory (and a patched V row is visible)
+    if (r == 0) SAGEKV_STAMP(5);
     if (nt > 0 && !mbar_wait(vbar, par)) timed_out = true;
 
     // ---- O^T += V^T P: columns 16*cg8 .. +15 over this warp's half of the round's rows ----
@@ -471,6 +506,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     }
   }
   if (timed_out) atomicOr(p.status, kStatusWaitTimeout);
+  SAGEKV_STAMP_AFTER(6, acc[0] + acc[1] + acc[2] + acc[3]);
 
   // ---- merge the CTAs of the cluster: the owner of a column slice receives it from every CTA ----
   // Every warp sends its 16 columns straight from registers into the owners' inboxes with asynchronous stores
@@ -491,7 +527,9 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       send2(dst_ml + 8u, bar_ml, M1, L1);
     }
   }
+  SAGEKV_STAMP(7);
   if (!mbar_wait(inbox_bar, 0u) && tid == 0) atomicOr(p.status, kStatusWaitTimeout);
+  SAGEKV_STAMP(8);
 
   // ---- finish columns [rank*cols, rank*cols + my_cols) of every head from the inbox ----
   const int bk = b * p.H_kv + kvh;
@@ -578,6 +616,8 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     p.tickets[p.B * p.H_kv] = 0;
     *p.d_step = step + 1;
   }
+  SAGEKV_STAMP(9);
+  SAGEKV_TRACE_END;
 }
 
 
@@ -724,3 +764,18 @@ cudaError_t launch_decode(const DecodeParams &p, const DeviceInfo &dev, cudaStre
 }
 
 }  // namespace sagekv
+
+#if defined(SAGEKV_TRACE)
+// Copies the records out (host buffer of 32768 x 12 64-bit words), returns how many launches' CTAs were recorded
+// since the last call, and starts a new recording.  Synchronises the device.
+extern "C" int sagekv_trace_read(unsigned long long *host, unsigned int *n_records) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return SAGEKV_ERR_CUDA;
+  unsigned int n = 0, zero = 0;
+  if (cudaMemcpyFromSymbol(&n, sagekv::g_trace_n, sizeof(n)) != cudaSuccess) return SAGEKV_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(host, sagekv::g_trace, sizeof(unsigned long long) * sagekv::kTraceSlots * sagekv::kTraceStamps) != cudaSuccess)
+    return SAGEKV_ERR_CUDA;
+  if (cudaMemcpyToSymbol(sagekv::g_trace_n, &zero, sizeof(zero)) != cudaSuccess) return SAGEKV_ERR_CUDA;
+  *n_records = n;
+  return SAGEKV_OK;
+}
+#endif
