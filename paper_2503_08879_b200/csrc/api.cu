@@ -101,7 +101,8 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   ctx->max_chunks = (int)((max_ctx + kScoreChunk - 1) / kScoreChunk);
   {
     int cs, resident, smem;
-    decode_geometry(max_len, 0, nullptr, &ctx->max_splits, &cs, &resident, &smem);   // clusters per head at the largest L
+    decode_geometry(max_len, 0, nullptr, &ctx->max_splits, &cs, &resident, &smem);   // clusters per head at the largest L ...
+    if (ctx->max_splits < 4) ctx->max_splits = 4;                                    // ... or the most the launch geometry ever chooses
   }
   const size_t n_rows = (size_t)shape->batch * shape->n_q_heads;
   const size_t n_heads = (size_t)shape->batch * shape->n_kv_heads;

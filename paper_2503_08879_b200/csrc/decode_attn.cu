@@ -666,38 +666,46 @@ cudaError_t decode_setup(DeviceInfo *dev) {
   return e;
 }
 
-// Launch geometry for a reduced cache of L rows: one cluster per KV head whose CTAs hold their whole range at
-// once when it fits and go through it in rounds otherwise; more clusters per head only beyond kDecodeMaxRounds.
-// heads = batch x KV heads of the launch (0, or dev null: not known).  Clusters of 8 (the portable limit) unless a
-// smaller size lets more of the work be resident: back-to-back launches overlap (the next one fetches its rows
-// while this one computes), which only works if the clusters of two launches fit on the device together, so the
-// sizes are compared by  waves of (two launches' clusters) x time of one cluster, the latter about 4 us + 0.07 us
-// per tile of a CTA + 1 us per extra round on this part.  Smaller sizes are considered only where a CTA still
-// holds its whole range at once.
+// Launch geometry for a reduced cache of L rows: nc clusters of c CTAs per KV head.  A CTA holds its whole range at
+// once when it fits (up to kDecodeMaxResident tiles) and goes through it in rounds otherwise; with nc > 1 the
+// clusters' results are merged through scratch by the last CTA to arrive.  heads = batch x KV heads of the launch
+// (0, or dev null: not known; then one cluster of 8 per head, more only beyond kDecodeMaxRounds rounds).
+// Back-to-back launches overlap (the next one fetches its rows while this one computes), which only works if the
+// clusters of two launches fit on the device together, so the candidates are compared by
+//     waves of (two launches' clusters) / 2  x  time of one cluster,
+// the latter, measured on this part, about 4 us + 0.07 us per tile of a round + 3.5 us per further round + 1.5 us
+// for the merge through scratch.  (15 clusters of 8 whole-SM CTAs fit at once, 22 of 6, 26 of 5, 33 of 4.)
+constexpr int kDecodeMaxClustersPerHead = 4;
+
 void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, int *cs, int *resident_tiles, int *smem_bytes) {
   const int n_tiles = (L + 15) / 16;
   int c = 1;
   while (c < kDecodeBaseCluster && c * 2 <= n_tiles) c <<= 1;                   // cluster size 1, 2, 4 or 8
   const int per_cluster_cta = kDecodeRoundTiles * kDecodeMaxRounds;              // most tiles a CTA goes through
-  const int nc = (n_tiles + c * per_cluster_cta - 1) / (c * per_cluster_cta);
-  int per_cta = (n_tiles + c * nc - 1) / (c * nc);                               // most tiles a CTA gets
-  if (dev != nullptr && heads > 0 && c == kDecodeBaseCluster && nc == 1) {
+  int nc = (n_tiles + c * per_cluster_cta - 1) / (c * per_cluster_cta);
+  if (dev != nullptr && heads > 0 && c == kDecodeBaseCluster) {
     float best = 0.f;
-    int best_c = c;
-    for (int cand = kDecodeBaseCluster; cand >= 4; --cand) {
-      if (cand == 7) continue;                                                   // (no more of them fit than of 8)
-      const int per = (n_tiles + cand - 1) / cand;
-      if (cand != kDecodeBaseCluster && per > kDecodeMaxResident) continue;
-      const int resident = per <= kDecodeMaxResident ? per : 2 * kDecodeRoundTiles;
-      const int rounds = per <= kDecodeMaxResident ? 1 : (per + kDecodeRoundTiles - 1) / kDecodeRoundTiles;
-      const int cap = cluster_capacity(dev->device, cand, resident);
-      if (cap <= 0) continue;
-      const float cost = 0.5f * (float)((2 * heads + cap - 1) / cap) * (4.0f + 0.07f * (float)per + (float)(rounds - 1));
-      if (best == 0.f || cost < best) { best = cost; best_c = cand; }
+    int best_c = c, best_nc = nc;
+    for (int cand_nc = nc; cand_nc <= nc; ++cand_nc) {   // (more clusters per head than needed were measured: the merge through scratch and the lost overlap cost more than the rounds saved)
+      for (int cand = kDecodeBaseCluster; cand >= 4; --cand) {
+        if (cand == 7) continue;                                                 // (no more of them fit than of 8)
+        const int per = (n_tiles + cand * cand_nc - 1) / (cand * cand_nc);
+        if (per > per_cluster_cta) continue;
+        if (per < 4 && cand_nc > 1) continue;                                    // too little work per CTA to pay for the merge
+        const int resident = per <= kDecodeMaxResident ? per : 2 * kDecodeRoundTiles;
+        const int rounds = per <= kDecodeMaxResident ? 1 : (per + kDecodeRoundTiles - 1) / kDecodeRoundTiles;
+        const int cap = cluster_capacity(dev->device, cand, resident);
+        if (cap <= 0) continue;
+        const float one = 4.0f + 0.07f * (float)(rounds == 1 ? per : kDecodeRoundTiles) + 3.5f * (float)(rounds - 1) +
+                          (cand_nc > 1 ? 1.5f : 0.f);
+        const float cost = 0.5f * (float)((2 * heads * cand_nc + cap - 1) / cap) * one;
+        if (best == 0.f || cost < best) { best = cost; best_c = cand; best_nc = cand_nc; }
+      }
     }
     c = best_c;
-    per_cta = (n_tiles + c - 1) / c;
+    nc = best_nc;
   }
+  const int per_cta = (n_tiles + c * nc - 1) / (c * nc);                         // most tiles a CTA gets
   *n_clusters = nc;
   *cs = c;
   *resident_tiles = per_cta <= kDecodeMaxResident ? per_cta : 2 * kDecodeRoundTiles;
