@@ -119,14 +119,10 @@ cudaError_t launch_quest_bounds(const uint16_t *q, const uint16_t *kmin, const u
                                 int n_blocks, int G, int H_q, int H_kv, int B, float scale, int n_sm, cudaStream_t stream);
 
 // ---- decode attention ------------------------------------------------------
-#if !defined(SAGEKV_DECODE_WARPS)
-#define SAGEKV_DECODE_WARPS 8
-#endif
-constexpr int kDecodeWarps = SAGEKV_DECODE_WARPS;                      // warps per CTA: 8, or 16 (two row halves in the second product)
+constexpr int kDecodeWarps = 8;                                        // consumer warps per CTA (one more warp issues the copies)
 constexpr int kDecodeMaxCluster = 8;                                   // CTAs per cluster (the portable limit)
-constexpr int kDecodeMaxResident = 24;                                 // 16-row tiles (K and V) a CTA holds at once: 192 KB
-constexpr int kDecodeRoundTiles = 12;                                  // tiles per round when the partition is longer (two buffers)
-constexpr int kDecodeMaxRounds = 8;                                    // rounds before a head gets more clusters
+constexpr int kDecodeSlots = 44;                                       // 4 KB slots of a CTA's staging area, one K or one V tile each: 176 KB
+constexpr int kDecodeMaxTiles = kDecodeSlots;                          // most 16-row tiles a CTA takes: its K tiles must all be resident
 constexpr int kPartialStride = kMaxGroup * kHeadDim + 2 * kMaxGroup;   // floats per cluster result: O[8][128], m[8], l[8]
 
 struct DecodeParams {

@@ -4,21 +4,23 @@
 // Flash-decoding on thread-block clusters.  The L rows of one KV head are cut into 16-row tiles that are
 // dealt evenly, as contiguous ranges, to the CTAs of one cluster.  A CTA brings its K and V tiles into shared
 // memory with tensor copies (one 16-row x 64-column box per request, 128-byte swizzle, completion counted on
-// an mbarrier): a few requests per lane of one warp instead of hundreds of 16-byte copies per warp.  When the
-// range fits (up to 24 tiles) everything is requested at once; longer ranges go through two buffers of 12
-// tiles in rounds, the next round's copies in flight while this one is worked on.  Per round:
-//   S = K Q^T     16 rows x 8 heads per mma, a tile per warp in turn.  A fragments come from the swizzled
-//                 tile with ldmatrix, the query (B fragments) sits in registers.
-//   softmax       one maximum per head over the whole CTA (two block barriers per round), so no partial
-//                 result is ever rescaled inside a round; the weights, rounded to bf16, go to shared memory.
-//   O^T = V^T P   split by COLUMNS: warp w accumulates columns 16w..16w+15 of all heads over all rows of the
-//                 round (transposing ldmatrix for V, the weights as B fragments).  The warps' results are
+// an mbarrier), issued by a ninth warp that does nothing else.  The staging area has 44 slots of one tile
+// (K or V) each.  All K tiles of the range are resident from the start; so are the V tiles while slots last,
+// and the remaining V tiles take over the K slots as soon as the first product is done.  There is one pass:
+//   S = K Q^T     16 rows x 8 heads per mma, a tile per warp in turn (the scores of all its tiles stay in
+//                 registers).  A fragments come from the swizzled tile with ldmatrix, the query (B fragments)
+//                 sits in registers.
+//   softmax       ONE maximum per head over the whole CTA (two block barriers in all), so nothing is ever
+//                 rescaled; the weights, rounded to bf16, go to shared memory for all tiles.
+//   O^T = V^T P   split by COLUMNS: warp w accumulates columns 16w..16w+15 of all heads over all rows
+//                 (transposing ldmatrix for V, the weights as B fragments).  The warps' results are
 //                 disjoint, so nothing is exchanged or summed inside the CTA.
 // Every head masks the rows of the other heads' segments.  The CTAs of a cluster are merged through
-// distributed shared memory: each warp stores its 16 columns straight from registers into the inbox of the
-// CTA that finishes those columns, one cluster barrier, and each CTA writes its slice of the 128 output
-// columns.  With several clusters per head (very long caches) the cluster results go to scratch and the CTA
-// that arrives last (one atomic ticket, no waiting) merges them.
+// distributed shared memory: each warp sends its 16 columns straight from registers into the inbox of the
+// CTA that finishes those columns with asynchronous stores counted on that CTA's barrier (one way, no
+// cluster barrier), and each CTA writes its slice of the 128 output columns.  With several clusters per
+// head (caches beyond 44 tiles per CTA) the cluster results go to scratch and the CTA that arrives last
+// (one atomic ticket, no waiting) merges them.
 // The staged copy of the window row that the new token replaces is overwritten in shared memory from
 // k_new / v_new once it has landed, and the CTA owning that row stores the new token into the cache.
 // Every wait on a copy barrier is bounded: a wait that runs out sets kStatusWaitTimeout in the context's status
@@ -35,26 +37,26 @@ namespace cg = cooperative_groups;
 
 namespace sagekv {
 
-constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kDecodeThreads = (kDecodeWarps + 1) * 32;   // eight consumer warps and the warp that issues the copies
+constexpr int kConsumerThreads = kDecodeWarps * 32;
 constexpr int kDecodeBaseCluster = 8;          // the cluster size tried first (the portable limit)
-constexpr int kTileBytes = 2 * 16 * 256;       // 16 rows of K and of V
+constexpr int kSlotBytes = 16 * 256;           // a slot of the staging area: 16 rows of K or of V
 constexpr int kHalfBytes = 16 * 128;           // 16 rows x 64 columns: one box of the tensor copy
 constexpr int kPHeadWords = 12;                // 32-bit words per (tile, head) of the weight buffer: 8 used, 4 spread the banks
 constexpr int kPTileWords = kMaxGroup * kPHeadWords;
-constexpr int kIssueWarp = kDecodeWarps - 1;   // the warp with the fewest tiles issues the copies
-constexpr int kRowHalves = kDecodeWarps / 8;   // the second product splits columns eight ways and rows this many ways
-constexpr int kQkTiles = (kDecodeMaxResident + kDecodeWarps - 1) / kDecodeWarps;   // tiles of a round a warp may get in the first product
+constexpr int kQkGroup = 3;                    // tiles of the first product a warp works on at once
+constexpr int kQkTiles = (kDecodeMaxTiles + kDecodeWarps - 1) / kDecodeWarps;   // tiles a warp may get in the first product (6)
 constexpr uint32_t kWaitLimit = 1u << 22;      // polls of a copy barrier before giving up (each poll already blocks for a while)
 
 struct DecShared {
-  unsigned long long bar[4];                                   // K landed [buffer 0, 1], V landed [buffer 0, 1]
+  unsigned long long bar[3];                                   // K landed, early V landed, late V landed
   unsigned long long inbox_bar;                                // every CTA's share for this CTA's columns has landed
   int last;
-  int pad_;
-  float warp_m[kDecodeWarps][kMaxGroup];                       // per round: maxima of the warps' rows
-  float2 inbox_ml[kRowHalves * kDecodeMaxCluster][kMaxGroup];  // [source CTA, row half][head] (max, sum)
-  uint32_t P[kDecodeMaxResident * kPTileWords];                // softmax weights of the round: [tile][head][row pair g: rows 2g, 2g + 1]
-  float inbox_o[kRowHalves * (kHeadDim + 4 * kDecodeMaxCluster) * kMaxGroup];   // [source CTA, row half][my column][head]
+  int pad_[3];
+  float warp_m[kDecodeWarps][kMaxGroup];                       // maxima of the warps' rows
+  float2 inbox_ml[kDecodeMaxCluster][kMaxGroup];               // [source CTA][head] (max, sum)
+  uint32_t P[kDecodeMaxTiles * kPTileWords];                   // softmax weights: [tile][head][row pair g: rows 2g, 2g + 1]
+  float inbox_o[(kHeadDim + 4 * kDecodeMaxCluster) * kMaxGroup];   // [source CTA][my column][head]; cluster size x columns <= 160
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -147,15 +149,21 @@ __device__ __forceinline__ unsigned long long trace_now() {
 #define SAGEKV_TRACE_END do { } while (0)
 #endif
 
-// kMulti: the CTA's range is longer than the staging area and goes through it in rounds
-template <bool kMulti>
+__device__ __forceinline__ void bar_sync(int id, int n_threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+
+// n_slots: slots of this launch's staging area (min(2 * most tiles of a CTA, kDecodeSlots)).
+// kLong: a CTA may have more tiles than half the slots (part of V arrives late, a warp may have up to six tiles in
+// the first product); false keeps the common case free of that.
+template <bool kLong>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
 decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                   const int resident_tiles) {
+                   const int n_slots) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t stage = (raw + 1023u) & ~1023u;                 // the tiles: boxes on 1024-byte boundaries
-  DecShared &sh = *reinterpret_cast<DecShared *>(smem_raw + (stage - raw) + (size_t)resident_tiles * kTileBytes);
+  const uint32_t stage = (raw + 1023u) & ~1023u;                 // the slots: boxes on 1024-byte boundaries
+  DecShared &sh = *reinterpret_cast<DecShared *>(smem_raw + (stage - raw) + (size_t)n_slots * kSlotBytes);
 
   cg::cluster_group cluster = cg::this_cluster();
   const int cs = cluster.num_blocks();
@@ -164,7 +172,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;
   const int h0 = 2 * c, h1 = 2 * c + 1;                           // the two heads a lane's accumulators belong to
-  const int cg8 = warp & 7, half = warp >> 3;                     // second product: column group and row half of this warp
+  const bool producer = warp == kDecodeWarps;
   const bool append = p.k_new != nullptr;
   SAGEKV_TRACE_BEGIN
   SAGEKV_STAMP(0);
@@ -173,51 +181,34 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   const int n_tiles = (p.L + 15) >> 4;
   const int base_n = n_tiles / (int)gridDim.x, rem = n_tiles % (int)gridDim.x;
   const int first_tile = ci * base_n + min(ci, rem);
-  const int my_tiles = base_n + (ci < rem ? 1 : 0);
-  const int n_rounds = kMulti ? (my_tiles + kDecodeRoundTiles - 1) / kDecodeRoundTiles : 1;
+  const int n = base_n + (ci < rem ? 1 : 0);                      // my tiles: K tile t in slot t
+  // V tile t sits in slot n + t while slots last (the early ones, requested at once); the others (late) take
+  // slot n + t - n_slots, a K slot, once the first product is done
+  constexpr int kQk = kLong ? kQkTiles : kQkGroup;           // tiles of the first product a warp may have
+  const int n_early = kLong ? min(n, n_slots - n) : n, n_late = n - n_early;
+  auto v_slot = [&](int t) { return (!kLong || t < n_early) ? n + t : n + t - n_slots; };
 
   // columns each CTA of the cluster finishes: a multiple of 4, the last CTA may get fewer
   const int cols = ((kHeadDim + cs - 1) / cs + 3) & ~3;
   const int my_cols = max(0, min(cols, kHeadDim - rank * cols));
   const int n_pairs = (p.G + 1) >> 1;                             // head pairs in use
 
-  const uint32_t bar0 = smem_u32(&sh.bar[0]), inbox_bar = smem_u32(&sh.inbox_bar);
+  const uint32_t kbar = smem_u32(&sh.bar[0]), vbar_e = smem_u32(&sh.bar[1]), vbar_l = smem_u32(&sh.bar[2]);
+  const uint32_t inbox_bar = smem_u32(&sh.inbox_bar);
   if (tid == 0) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) mbar_init(bar0 + 8 * i, 1);
+    mbar_init(kbar, 1);
+    mbar_init(vbar_e, 1);
+    mbar_init(vbar_l, 1);
     mbar_init(inbox_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
-    // from both row halves of every CTA of the cluster: 8 bytes per (own column, head pair in use) and 64 bytes
-    // of (max, sum) pairs
-    mbar_expect_tx(inbox_bar, (uint32_t)(kRowHalves * cs * (my_cols * n_pairs * 8 + 64)));
+    // from every CTA of the cluster: 8 bytes per (own column, head pair in use) and 64 bytes of (max, sum) pairs
+    mbar_expect_tx(inbox_bar, (uint32_t)(cs * (my_cols * n_pairs * 8 + 64)));
   }
   __syncthreads();
   cluster.barrier_arrive();                              // waited for just before the first store into a peer: its barrier is set up
-
-  // the copies of one round, K boxes first: lane i of the issuing warp takes requests i, i + 32, ...
-  uint64_t stream_policy;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
-  auto issue_round = [&](int r) {
-    const int buf = kMulti ? (r & 1) : 0;
-    const int t0 = kMulti ? r * kDecodeRoundTiles : 0;
-    const int nt = kMulti ? min(kDecodeRoundTiles, my_tiles - t0) : my_tiles;
-    const uint32_t kbar = bar0 + 8 * buf, vbar = bar0 + 16 + 8 * buf;
-    if (lane == 0) {
-      mbar_expect_tx(kbar, (uint32_t)nt * (kTileBytes / 2));
-      mbar_expect_tx(vbar, (uint32_t)nt * (kTileBytes / 2));
-    }
-    __syncwarp();
-    for (int op = lane; op < nt * 4; op += 32) {
-      const bool is_v = op >= nt * 2;
-      const int o2 = is_v ? op - nt * 2 : op;
-      const int t = o2 >> 1, hf = o2 & 1;
-      const uint32_t dst = stage + (uint32_t)((buf * kDecodeRoundTiles + t) * kTileBytes + (is_v ? 2 : 0) * kHalfBytes + hf * kHalfBytes);
-      tensor_copy_4d(dst, is_v ? &map_v : &map_k, hf * 64, (first_tile + t0 + t) << 4, kvh, b, is_v ? vbar : kbar, stream_policy);
-    }
-  };
 
   // Programmatic dependent launch: until the wait returns, nothing that an earlier kernel on the stream may
   // still be writing is read (q, k_new, v_new, the step counter) and nothing at all is written to global
@@ -228,71 +219,88 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
-  if (warp == kIssueWarp && my_tiles > 0) {
-    issue_round(0);
-    if (kMulti && n_rounds > 1) issue_round(1);
+
+  // ---- the warp that issues the copies: lane i takes requests i, i + 32, ... (two boxes per tile) ----
+  if (producer) {
+    uint64_t stream_policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
+    auto issue = [&](const CUtensorMap *map, int t_lo, int t_hi, bool is_v, uint32_t bar) {   // tiles [t_lo, t_hi)
+      if (lane == 0 && t_hi > t_lo) mbar_expect_tx(bar, (uint32_t)(t_hi - t_lo) * kSlotBytes);
+      __syncwarp();
+      for (int op = lane; op < (t_hi - t_lo) * 2; op += 32) {
+        const int t = t_lo + (op >> 1), hf = op & 1;
+        const uint32_t dst = stage + (uint32_t)((is_v ? v_slot(t) : t) * kSlotBytes + hf * kHalfBytes);
+        tensor_copy_4d(dst, map, hf * 64, (first_tile + t) << 4, kvh, b, bar, stream_policy);
+      }
+    };
+    // (In prefetch mode this warp never waits for the predecessor: it reads nothing of it, and what it requests
+    // after barrier A comes after the consumers' wait.  It leaves the release of the successor to the consumers,
+    // who give it after their wait: a release from here would let a second launch run ahead.)
+    issue(&map_k, 0, n, false, kbar);
+    issue(&map_v, 0, n_early, true, vbar_e);
+    bar_sync(1, kDecodeThreads);                         // A: every consumer warp is done with the K slots
+    if (kLong && n_late > 0) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // their reads (and a patched row) precede the refill
+      issue(&map_v, n_early, n, true, vbar_l);
+    }
+    return;                                              // (its cluster arrival at entry stands; it takes part in nothing else)
   }
 
   // ---- everything that does not depend on the predecessor's results is worked out before the wait ----
   // The instructions after the wait form one long dependent chain per warp, so every address, mask and index
   // that can be known now is computed now and kept in a register.
   // (1) which of this lane's score elements are visible to their heads (sink, own segment, window): bit 4i + e
-  //     for the warp's i-th tile of the round, element e of the accumulator
-  const int win_lo = p.S + p.n_sel;
-  const int seg0_lo = p.S + (p.pooled ? 0 : h0 * p.k_q), seg0_hi = seg0_lo + p.k_q;
-  const int seg1_lo = p.S + (p.pooled ? 0 : h1 * p.k_q), seg1_hi = seg1_lo + p.k_q;
-  auto visibility = [&](int t0) {
-    uint32_t bits = 0;
-#pragma unroll
-    for (int i = 0; i < kQkTiles; ++i) {
-      const int r0 = ((first_tile + t0 + warp + kDecodeWarps * i) << 4) + 2 * g;
-      const int ra = r0 + (g >= 4 ? 1 : 0), rb = r0 + (g >= 4 ? 0 : 1);   // tokens of accumulator elements 0, 1 and 2, 3
-      const bool va = ra < p.L, vb = rb < p.L;
-      const bool sa = ra < p.S || ra >= win_lo, sb = rb < p.S || rb >= win_lo;
-      bits |= (va && h0 < p.G && (sa || (ra >= seg0_lo && ra < seg0_hi)) ? 1u : 0u) << (4 * i);
-      bits |= (va && h1 < p.G && (sa || (ra >= seg1_lo && ra < seg1_hi)) ? 2u : 0u) << (4 * i);
-      bits |= (vb && h0 < p.G && (sb || (rb >= seg0_lo && rb < seg0_hi)) ? 4u : 0u) << (4 * i);
-      bits |= (vb && h1 < p.G && (sb || (rb >= seg1_lo && rb < seg1_hi)) ? 8u : 0u) << (4 * i);
-    }
-    return bits;
-  };
-  uint32_t vis = visibility(0);
-  // (2) fragment addresses: K rows for the first product (ldmatrix), the query rows (ldmatrix), V for the second
-  //     (transposing ldmatrix), the weight words this lane writes and reads
+  //     for the warp's i-th tile, element e of the accumulator
   // Row order of the K fragments: A row m of the mma (m < 8) holds token 2m (m < 4) or 2m + 1, A row m + 8 the
   // other token of the pair (2m, 2m + 1).  So a lane's accumulators belong to two neighbouring tokens, whose
   // weights make one 32-bit word of the second product's B fragment, and the eight rows one ldmatrix phase
   // reads still fall into eight different bank groups of the swizzled tile.
+  const int win_lo = p.S + p.n_sel;
+  const int seg0_lo = p.S + (p.pooled ? 0 : h0 * p.k_q), seg0_hi = seg0_lo + p.k_q;
+  const int seg1_lo = p.S + (p.pooled ? 0 : h1 * p.k_q), seg1_hi = seg1_lo + p.k_q;
+  uint32_t vis = 0;
+#pragma unroll
+  for (int i = 0; i < kQk; ++i) {
+    const int r0 = ((first_tile + warp + kDecodeWarps * i) << 4) + 2 * g;
+    const int ra = r0 + (g >= 4 ? 1 : 0), rb = r0 + (g >= 4 ? 0 : 1);   // tokens of accumulator elements 0, 1 and 2, 3
+    const bool va = ra < p.L, vb = rb < p.L;
+    const bool sa = ra < p.S || ra >= win_lo, sb = rb < p.S || rb >= win_lo;
+    vis |= (va && h0 < p.G && (sa || (ra >= seg0_lo && ra < seg0_hi)) ? 1u : 0u) << (4 * i);
+    vis |= (va && h1 < p.G && (sa || (ra >= seg1_lo && ra < seg1_hi)) ? 2u : 0u) << (4 * i);
+    vis |= (vb && h0 < p.G && (sb || (rb >= seg0_lo && rb < seg0_hi)) ? 4u : 0u) << (4 * i);
+    vis |= (vb && h1 < p.G && (sb || (rb >= seg1_lo && rb < seg1_hi)) ? 8u : 0u) << (4 * i);
+  }
+  // (2) fragment addresses: K rows for the first product (ldmatrix), V for the second (transposing ldmatrix), the
+  //     weight words this lane writes and reads
   const int mi = lane >> 3, l8 = lane & 7;
   const int arow = 2 * l8 + (((mi & 1) != 0) != (l8 >= 4) ? 1 : 0);
-  uint32_t k_off[8];                                     // k-step ks of a tile: tile base + k_off[ks]
+  uint32_t k_off[8];                                     // k-step ks of a tile: slot base + k_off[ks]
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) k_off[ks] = tile_offset(arow, 2 * ks + (mi >> 1));
   const uint16_t *q_lane = p.q + ((int64_t)b * p.H_q + kvh * p.G + min(g, p.G - 1)) * kHeadDim + 2 * c;   // this lane's first query element
-  uint32_t v_off = 2 * kHalfBytes + tile_offset((mi >> 1) * 8 + l8, 2 * cg8 + (mi & 1));
+  uint32_t v_off = tile_offset((mi >> 1) * 8 + l8, 2 * warp + (mi & 1));
   uint32_t pw_addr = smem_u32(sh.P) + (uint32_t)((h0 * kPHeadWords + g) * 4);   // + tile * kPTileWords * 4; head h1: + kPHeadWords * 4
   uint32_t pr_addr = smem_u32(sh.P) + (uint32_t)((g * kPHeadWords + c) * 4);    // + tile * kPTileWords * 4; rows 2c+8, 2c+9: + 16
   // (3) where this lane's results go: the owners of its two columns, as addresses in their shared memory
-  const int col_a = 16 * cg8 + g, col_b = col_a + 8;
+  const int col_a = 16 * warp + g, col_b = col_a + 8;
   const int own_a = col_a / cols, own_b = col_b / cols;
-  const int src_me = kRowHalves * rank + half;                    // this warp's place among the sources of an inbox
   uint32_t dst_a, dst_b, bar_a, bar_b, dst_ml = 0, bar_ml = 0;
   {
     const uint32_t inbox = smem_u32(sh.inbox_o);
-    const uint32_t la = inbox + (uint32_t)(((src_me * cols + (col_a - own_a * cols)) * kMaxGroup + h0) * 4);
-    const uint32_t lb = inbox + (uint32_t)(((src_me * cols + (col_b - own_b * cols)) * kMaxGroup + h0) * 4);
+    const uint32_t la = inbox + (uint32_t)(((rank * cols + (col_a - own_a * cols)) * kMaxGroup + h0) * 4);
+    const uint32_t lb = inbox + (uint32_t)(((rank * cols + (col_b - own_b * cols)) * kMaxGroup + h0) * 4);
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst_a) : "r"(la), "r"(own_a));
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst_b) : "r"(lb), "r"(own_b));
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_a) : "r"(inbox_bar), "r"(own_a));
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_b) : "r"(inbox_bar), "r"(own_b));
-    if (cg8 == 0 && g < cs) {                            // lane (g, c) of a half's first warp tells CTA g the (max, sum) of heads 2c, 2c+1
-      const uint32_t lm = smem_u32(&sh.inbox_ml[src_me][h0]);
+    if (warp == 0 && g < cs) {                           // lane (g, c) of warp 0 tells CTA g the (max, sum) of heads 2c, 2c+1
+      const uint32_t lm = smem_u32(&sh.inbox_ml[rank][h0]);
       asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst_ml) : "r"(lm), "r"(g));
       asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_ml) : "r"(inbox_bar), "r"(g));
     }
   }
   // (4) the finishing stage: one thread per output value (own column lc, head fh)
-  const int fin_items = my_cols * p.G, n_src = kRowHalves * cs;
+  const int fin_items = my_cols * p.G, n_src = cs;
   int fin_lc = tid / p.G, fin_h = tid - fin_lc * p.G;
   uint16_t *fin_out = p.out + ((int64_t)b * p.H_q + kvh * p.G + fin_h) * kHeadDim + rank * cols + fin_lc;
 #pragma unroll
@@ -330,69 +338,67 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     // One ticket per CTA, taken once the counter has been read (release: the load is ordered before it), by a
     // thread of the warp with the fewest tiles.  The answer is looked at only when the CTA is done, long after
     // it has come back.
-    if (tid == kDecodeThreads - 1)
+    if (tid == kConsumerThreads - 1)
       asm volatile("atom.add.release.gpu.global.s32 %0, [%1], 1;" : "=r"(my_ticket) : "l"(p.tickets + p.B * p.H_kv) : "memory");
   }
 
-  float M0 = -INFINITY, M1 = -INFINITY;   // running maxima of heads 2c, 2c+1 over the CTA's rows (log2 units)
-  float L0 = 0.f, L1 = 0.f;               // sums of the (bf16-rounded) weights over this warp's rows of the second product
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};    // O^T: (col_a, h0) (col_a, h1) (col_b, h0) (col_b, h1) over this warp's rows
   bool timed_out = false;                 // a copy never arrived: reported through the status word; the CTA runs on (its output is then meaningless)
-  int slot = -1, slot_tile = -1;          // the replaced window row and its CTA-local tile, worked out at first use
+  if (n > 0 && !mbar_wait(kbar, 0u)) timed_out = true;
+  SAGEKV_STAMP(3);
 
-  for (int r = 0; r < n_rounds; ++r) {
-    const int buf = kMulti ? (r & 1) : 0;
-    const uint32_t par = kMulti ? (uint32_t)((r >> 1) & 1) : 0u;
-    const int t0 = kMulti ? r * kDecodeRoundTiles : 0;
-    const int nt = kMulti ? min(kDecodeRoundTiles, my_tiles - t0) : my_tiles;
-    const uint32_t kbar = bar0 + 8 * buf, vbar = bar0 + 16 + 8 * buf;
-    const uint32_t buf_base = stage + (uint32_t)(buf * kDecodeRoundTiles * kTileBytes);
-    if (kMulti && r > 0) vis = visibility(t0);
-    if (nt > 0 && !mbar_wait(kbar, par)) timed_out = true;
-    if (r == 0) SAGEKV_STAMP(3);
-
-    // the staged copy of the replaced row is stale: the warp that works on its tile patches K and V
-    if (append && r == 0) {
-      slot = p.S + p.n_sel + step % p.ring_len;
-      slot_tile = (slot >> 4) - first_tile;
+  // the staged copy of the replaced row is stale: the warp that works on its tile patches K now, and V as soon as
+  // the tile's V copy is here (now, for an early tile; after the first product, for a late one)
+  int slot = -1, st = -1;                 // the replaced window row and its CTA-local tile (if 0 <= st < n)
+  if (append) {
+    slot = p.S + p.n_sel + step % p.ring_len;
+    st = (slot >> 4) - first_tile;
+  }
+  const bool patcher = append && st >= 0 && st < n && (st & (kDecodeWarps - 1)) == warp;
+  auto patch = [&](bool is_v) {           // lanes 0-15 hold the new K row, lanes 16-31 the new V row
+    if ((lane >= 16) == is_v) {
+      const int row = slot & 15, piece = lane & 15;
+      const uint32_t dst = stage + (uint32_t)((is_v ? v_slot(st) : st) * kSlotBytes) + tile_offset(row, piece);
+      asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(new_row.x), "r"(new_row.y), "r"(new_row.z), "r"(new_row.w) : "memory");
     }
-    const int st = slot_tile - t0;                       // tile of this round holding the replaced row, if in [0, nt)
-    if (append && st >= 0 && st < nt && (st & (kDecodeWarps - 1)) == warp) {
-      if (!mbar_wait(vbar, par)) timed_out = true;
-      {
-        const int row = slot & 15, piece = lane & 15;
-        const uint32_t dst = buf_base + (uint32_t)(st * kTileBytes + (lane < 16 ? 0 : 2 * kHalfBytes)) + tile_offset(row, piece);
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(new_row.x), "r"(new_row.y), "r"(new_row.z), "r"(new_row.w) : "memory");
-        if (SAGEKV_OK_INDEX(p.status, slot >= 0 && slot < p.L)) {
-          uint16_t *gdst = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
-                           (int64_t)slot * p.cs.token_stride + piece * 8;
-          st_v4(gdst, new_row);
-        }
-      }
-      __syncwarp();
+  };
+  if (patcher) {
+    patch(false);
+    if (st < n_early) {
+      if (!mbar_wait(vbar_e, 0u)) timed_out = true;
+      patch(true);
     }
+    if (SAGEKV_OK_INDEX(p.status, slot >= 0 && slot < p.L)) {
+      uint16_t *gdst = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
+                       (int64_t)slot * p.cs.token_stride + (lane & 15) * 8;
+      st_v4(gdst, new_row);
+    }
+    __syncwarp();
+  }
 
-    // ---- S = K Q^T: this warp's tiles of the round are warp, warp + kDecodeWarps, ... ----
-    // An mma takes far longer than its issue slot, so the work is laid out as short independent chains: per
-    // tile four accumulators (k-steps j and j + 4), the fragments requested ahead of the mmas.
-    float sv[kQkTiles][4];
-    float wm0 = -INFINITY, wm1 = -INFINITY;
-    {
-      float ch[kQkTiles][4][4];
-      uint32_t fa[kQkTiles][4][4];
+  // ---- S = K Q^T: this warp's tiles are warp, warp + 8, ...; three at a time ----
+  // An mma takes far longer than its issue slot, so the work is laid out as short independent chains: per
+  // tile four accumulators (k-steps j and j + 4), the fragments requested ahead of the mmas.
+  float sv[kQk][4];
+  float wm0 = -INFINITY, wm1 = -INFINITY;
+#pragma unroll
+  for (int grp = 0; grp < kQk / kQkGroup; ++grp) {
+    if (warp + kDecodeWarps * kQkGroup * grp < n) {
+      float ch[kQkGroup][4][4];
+      uint32_t fa[kQkGroup][4][4];
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {                   // k-steps 0..3, then 4..7
 #pragma unroll
-        for (int i = 0; i < kQkTiles; ++i) {
-          if (warp + kDecodeWarps * i < nt) {
-            const uint32_t tb = buf_base + (uint32_t)((warp + kDecodeWarps * i) * kTileBytes);
+        for (int i = 0; i < kQkGroup; ++i) {
+          const int t = warp + kDecodeWarps * (kQkGroup * grp + i);
+          if (t < n) {
+            const uint32_t tb = stage + (uint32_t)(t * kSlotBytes);
 #pragma unroll
             for (int j = 0; j < 4; ++j) ldmatrix_x4(tb + k_off[4 * hf + j], fa[i][j][0], fa[i][j][1], fa[i][j][2], fa[i][j][3]);
           }
         }
 #pragma unroll
-        for (int i = 0; i < kQkTiles; ++i) {
-          if (warp + kDecodeWarps * i < nt) {
+        for (int i = 0; i < kQkGroup; ++i) {
+          if (warp + kDecodeWarps * (kQkGroup * grp + i) < n) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               if (hf == 0)
@@ -406,105 +412,104 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
         }
       }
 #pragma unroll
-      for (int i = 0; i < kQkTiles; ++i) {
-        const bool have = warp + kDecodeWarps * i < nt;
-        const uint32_t vb4 = have ? (vis >> (4 * i)) & 15u : 0u;
+      for (int i = 0; i < kQkGroup; ++i) {
+        const int ti = kQkGroup * grp + i;
+        const bool have = warp + kDecodeWarps * ti < n;
+        const uint32_t vb4 = have ? (vis >> (4 * ti)) & 15u : 0u;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const float x = have ? (ch[i][0][e] + ch[i][1][e]) + (ch[i][2][e] + ch[i][3][e]) : 0.f;
-          sv[i][e] = ((vb4 >> e) & 1u) ? x * p.scale_log2 : -INFINITY;
+          sv[ti][e] = ((vb4 >> e) & 1u) ? x * p.scale_log2 : -INFINITY;
         }
-        wm0 = fmaxf(wm0, fmaxf(sv[i][0], sv[i][2]));
-        wm1 = fmaxf(wm1, fmaxf(sv[i][1], sv[i][3]));
+        wm0 = fmaxf(wm0, fmaxf(sv[ti][0], sv[ti][2]));
+        wm1 = fmaxf(wm1, fmaxf(sv[ti][1], sv[ti][3]));
       }
-    }
-    // over the eight lanes that hold the same heads (equal c): one warp-wide reduction per head
-    asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(wm0) : "f"(wm0), "r"(0x11111111u << c));
-    asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(wm1) : "f"(wm1), "r"(0x11111111u << c));
-    if (g == 0) { sh.warp_m[warp][h0] = wm0; sh.warp_m[warp][h1] = wm1; }
-    if (kMulti) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads and patches of the other buffer precede its refill
-    __syncthreads();   // A: the round's maxima are complete; every warp is past the round before
-
-    if (kMulti && warp == kIssueWarp && r >= 1 && r + 1 < n_rounds) issue_round(r + 1);   // into the buffer of round r - 1
-
-    float R0, R1;
-    {
-      float a0[kDecodeWarps], a1[kDecodeWarps];
+    } else {
 #pragma unroll
-      for (int w = 0; w < kDecodeWarps; ++w) { a0[w] = sh.warp_m[w][h0]; a1[w] = sh.warp_m[w][h1]; }
-#pragma unroll
-      for (int s2 = kDecodeWarps / 2; s2 > 0; s2 >>= 1)   // a tree, not a chain
-#pragma unroll
-        for (int w = 0; w < s2; ++w) { a0[w] = fmaxf(a0[w], a0[w + s2]); a1[w] = fmaxf(a1[w], a1[w + s2]); }
-      R0 = a0[0]; R1 = a1[0];
-    }
-    const float N0 = fmaxf(M0, R0), N1 = fmaxf(M1, R1);
-    if (r == 0) SAGEKV_STAMP_AFTER(4, N0 + N1);
-    const float s0 = N0 == -INFINITY ? 0.f : N0, s1 = N1 == -INFINITY ? 0.f : N1;
-    if (kMulti && r > 0) {                                 // bring sums and accumulators to the new maxima
-      const float f0 = fast_exp2(M0 - s0), f1 = fast_exp2(M1 - s1);
-      L0 *= f0; L1 *= f1;
-      acc[0] *= f0; acc[2] *= f0; acc[1] *= f1; acc[3] *= f1;
-    }
-    M0 = N0; M1 = N1;
-    // the weights enter the second product as bf16: one word per (tile, head, row pair g: rows 2g and 2g + 1)
-#pragma unroll
-    for (int i = 0; i < kQkTiles; ++i) {
-      const int t = warp + kDecodeWarps * i;
-      if (t < nt) {
-        const float x0 = fast_exp2(sv[i][0] - s0), x2 = fast_exp2(sv[i][2] - s0);              // head h0: elements 0 and 2
-        const float x1 = fast_exp2(sv[i][1] - s1), x3 = fast_exp2(sv[i][3] - s1);              // head h1: elements 1 and 3
-        const uint32_t p0 = g < 4 ? pack_bf16x2(x0, x2) : pack_bf16x2(x2, x0);                 // (row 2g in the low half)
-        const uint32_t p1 = g < 4 ? pack_bf16x2(x1, x3) : pack_bf16x2(x3, x1);
-        const uint32_t wa = pw_addr + (uint32_t)(t * kPTileWords * 4);
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(wa), "r"(p0) : "memory");
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(wa + kPHeadWords * 4), "r"(p1) : "memory");
-      }
-    }
-    __syncthreads();   // B: the weights of the round are in shared memory (and a patched V row is visible)
-    if (r == 0) SAGEKV_STAMP(5);
-    if (nt > 0 && !mbar_wait(vbar, par)) timed_out = true;
-
-    // ---- O^T += V^T P: columns 16*cg8 .. +15 over this warp's half of the round's rows ----
-    // A B fragment is two of the weight words (rows 2c, 2c+1 and 2c+8, 2c+9 of head g).  Six tiles per step, each on an
-    // accumulator chain of its own, all fragments requested before the mmas.  The same weights times a fragment
-    // of ones give the sums of the rounded weights per head, in every lane, in the accumulator layout (numerator
-    // and denominator agree; no shuffle or shared-memory exchange is needed for them).
-    {
-      const int nh = kRowHalves == 2 ? (nt + 1) >> 1 : nt;
-      const int t_lo = half ? nh : 0, t_hi = half ? nt : nh;
-      float xc[5][4], lc0[4] = {0.f, 0.f, 0.f, 0.f}, lc1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int u = 0; u < 5; ++u) xc[u][0] = xc[u][1] = xc[u][2] = xc[u][3] = 0.f;
-      const uint32_t vbase = buf_base + v_off;
-      const uint32_t ones = 0x3f803f80u;
-      for (int t6 = t_lo; t6 < t_hi; t6 += 6) {
-        uint32_t va[6][4], pb[6][2];
-#pragma unroll
-        for (int u = 0; u < 6; ++u) {
-          if (t6 + u < t_hi) {
-            ldmatrix_x4_trans(vbase + (uint32_t)((t6 + u) * kTileBytes), va[u][0], va[u][1], va[u][2], va[u][3]);
-            const uint32_t ra = pr_addr + (uint32_t)((t6 + u) * kPTileWords * 4);
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(pb[u][0]) : "r"(ra));
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(pb[u][1]) : "r"(ra + 16));
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 6; ++u) {
-          if (t6 + u < t_hi) {
-            if (u == 0) mma_bf16_16816(acc[0], acc[1], acc[2], acc[3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
-            else mma_bf16_16816(xc[u - 1][0], xc[u - 1][1], xc[u - 1][2], xc[u - 1][3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
-            if (u & 1) mma_bf16_16816(lc1[0], lc1[1], lc1[2], lc1[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
-            else mma_bf16_16816(lc0[0], lc0[1], lc0[2], lc0[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
-          }
-        }
-      }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[e] += ((xc[0][e] + xc[1][e]) + (xc[2][e] + xc[3][e])) + xc[4][e];
-      L0 += lc0[0] + lc1[0];
-      L1 += lc0[1] + lc1[1];
+      for (int i = 0; i < kQkGroup; ++i)
+        sv[kQkGroup * grp + i][0] = sv[kQkGroup * grp + i][1] = sv[kQkGroup * grp + i][2] = sv[kQkGroup * grp + i][3] = -INFINITY;
     }
   }
+  // over the eight lanes that hold the same heads (equal c): one warp-wide reduction per head
+  asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(wm0) : "f"(wm0), "r"(0x11111111u << c));
+  asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(wm1) : "f"(wm1), "r"(0x11111111u << c));
+  if (g == 0) { sh.warp_m[warp][h0] = wm0; sh.warp_m[warp][h1] = wm1; }
+  bar_sync(1, kDecodeThreads);   // A: the maxima are complete, and nobody reads a K slot any more (the copy warp refills them)
+
+  float M0, M1;                  // maxima of heads 2c, 2c+1 over the CTA's rows (log2 units)
+  {
+    float a0[kDecodeWarps], a1[kDecodeWarps];
+#pragma unroll
+    for (int w = 0; w < kDecodeWarps; ++w) { a0[w] = sh.warp_m[w][h0]; a1[w] = sh.warp_m[w][h1]; }
+#pragma unroll
+    for (int s2 = kDecodeWarps / 2; s2 > 0; s2 >>= 1)   // a tree, not a chain
+#pragma unroll
+      for (int w = 0; w < s2; ++w) { a0[w] = fmaxf(a0[w], a0[w + s2]); a1[w] = fmaxf(a1[w], a1[w + s2]); }
+    M0 = a0[0]; M1 = a1[0];
+  }
+  SAGEKV_STAMP_AFTER(4, M0 + M1);
+  const float s0 = M0 == -INFINITY ? 0.f : M0, s1 = M1 == -INFINITY ? 0.f : M1;
+  // the weights enter the second product as bf16: one word per (tile, head, row pair g: rows 2g and 2g + 1)
+#pragma unroll
+  for (int i = 0; i < kQk; ++i) {
+    const int t = warp + kDecodeWarps * i;
+    if (t < n) {
+      const float x0 = fast_exp2(sv[i][0] - s0), x2 = fast_exp2(sv[i][2] - s0);              // head h0: elements 0 and 2
+      const float x1 = fast_exp2(sv[i][1] - s1), x3 = fast_exp2(sv[i][3] - s1);              // head h1: elements 1 and 3
+      const uint32_t p0 = g < 4 ? pack_bf16x2(x0, x2) : pack_bf16x2(x2, x0);                 // (row 2g in the low half)
+      const uint32_t p1 = g < 4 ? pack_bf16x2(x1, x3) : pack_bf16x2(x3, x1);
+      const uint32_t wa = pw_addr + (uint32_t)(t * kPTileWords * 4);
+      asm volatile("st.shared.u32 [%0], %1;" ::"r"(wa), "r"(p0) : "memory");
+      asm volatile("st.shared.u32 [%0], %1;" ::"r"(wa + kPHeadWords * 4), "r"(p1) : "memory");
+    }
+  }
+  bar_sync(2, kConsumerThreads);   // B: the weights are in shared memory (and a patched early V row is visible)
+  SAGEKV_STAMP(5);
+
+  // ---- O^T = V^T P: columns 16*warp .. +15 over all rows, the early V tiles first ----
+  // A B fragment is two of the weight words (rows 2c, 2c+1 and 2c+8, 2c+9 of head g).  Six tiles per step, each on an
+  // accumulator chain of its own, all fragments requested before the mmas.  The same weights times a fragment
+  // of ones give the sums of the rounded weights per head, in every lane, in the accumulator layout (numerator
+  // and denominator agree; no shuffle or shared-memory exchange is needed for them).
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};    // O^T: (col_a, h0) (col_a, h1) (col_b, h0) (col_b, h1)
+  float xc[5][4], lc0[4] = {0.f, 0.f, 0.f, 0.f}, lc1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int u = 0; u < 5; ++u) xc[u][0] = xc[u][1] = xc[u][2] = xc[u][3] = 0.f;
+  auto second_product = [&](int t_lo, int t_hi) {
+    const uint32_t ones = 0x3f803f80u;
+    for (int t6 = t_lo; t6 < t_hi; t6 += 6) {
+      uint32_t va[6][4], pb[6][2];
+#pragma unroll
+      for (int u = 0; u < 6; ++u) {
+        if (t6 + u < t_hi) {
+          ldmatrix_x4_trans(stage + (uint32_t)(v_slot(t6 + u) * kSlotBytes) + v_off, va[u][0], va[u][1], va[u][2], va[u][3]);
+          const uint32_t ra = pr_addr + (uint32_t)((t6 + u) * kPTileWords * 4);
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(pb[u][0]) : "r"(ra));
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(pb[u][1]) : "r"(ra + 16));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 6; ++u) {
+        if (t6 + u < t_hi) {
+          if (u == 0) mma_bf16_16816(acc[0], acc[1], acc[2], acc[3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
+          else mma_bf16_16816(xc[u - 1][0], xc[u - 1][1], xc[u - 1][2], xc[u - 1][3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
+          if (u & 1) mma_bf16_16816(lc1[0], lc1[1], lc1[2], lc1[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
+          else mma_bf16_16816(lc0[0], lc0[1], lc0[2], lc0[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
+        }
+      }
+    }
+  };
+  if (n_early > 0 && !mbar_wait(vbar_e, 0u)) timed_out = true;
+  second_product(0, n_early);
+  if (kLong && n_late > 0) {                             // (the same for every thread of the CTA)
+    if (!mbar_wait(vbar_l, 0u)) timed_out = true;
+    if (patcher && st >= n_early) patch(true);
+    bar_sync(2, kConsumerThreads);                       // a patched late V row is visible
+    second_product(n_early, n);
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) acc[e] += ((xc[0][e] + xc[1][e]) + (xc[2][e] + xc[3][e])) + xc[4][e];
+  const float L0 = lc0[0] + lc1[0], L1 = lc0[1] + lc1[1];   // sums of the (bf16-rounded) weights of heads 2c, 2c+1 over the CTA's rows
   if (timed_out) atomicOr(p.status, kStatusWaitTimeout);
   SAGEKV_STAMP_AFTER(6, acc[0] + acc[1] + acc[2] + acc[3]);
 
@@ -522,7 +527,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       send2(dst_a, bar_a, acc[0], acc[1]);
       send2(dst_b, bar_b, acc[2], acc[3]);
     }
-    if (cg8 == 0 && g < cs) {
+    if (warp == 0 && g < cs) {
       send2(dst_ml, bar_ml, M0, L0);
       send2(dst_ml + 8u, bar_ml, M1, L1);
     }
@@ -535,35 +540,35 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   const int bk = b * p.H_kv + kvh;
   const int n_clusters = (int)gridDim.x / cs, cl = ci / cs;
   float *part = p.partials + ((int64_t)bk * n_clusters + cl) * kPartialStride;
-  for (int item = tid; item < fin_items; item += kDecodeThreads) {
+  for (int item = tid; item < fin_items; item += kConsumerThreads) {
     if (item != tid) {
       fin_lc = item / p.G;
       fin_h = item - fin_lc * p.G;
       fin_out = p.out + ((int64_t)b * p.H_q + kvh * p.G + fin_h) * kHeadDim + rank * cols + fin_lc;
     }
     const int lc = fin_lc, h = fin_h, col = rank * cols + lc;
-    float mx[kRowHalves * kDecodeMaxCluster], ls[kRowHalves * kDecodeMaxCluster], ov[kRowHalves * kDecodeMaxCluster];
+    float mx[kDecodeMaxCluster], ls[kDecodeMaxCluster], ov[kDecodeMaxCluster];
 #pragma unroll
-    for (int sI = 0; sI < kRowHalves * kDecodeMaxCluster; ++sI) {   // the loads of all sources are in flight together
+    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) {   // the loads of all sources are in flight together
       const float2 ml = sI < n_src ? sh.inbox_ml[sI][h] : make_float2(-INFINITY, 0.f);
       mx[sI] = ml.x; ls[sI] = ml.y;
       ov[sI] = sI < n_src ? sh.inbox_o[(sI * cols + lc) * kMaxGroup + h] : 0.f;
     }
-    float tm[kRowHalves * kDecodeMaxCluster];
+    float tm[kDecodeMaxCluster];
 #pragma unroll
-    for (int sI = 0; sI < kRowHalves * kDecodeMaxCluster; ++sI) tm[sI] = mx[sI];
+    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) tm[sI] = mx[sI];
 #pragma unroll
-    for (int w2 = kRowHalves * kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
+    for (int w2 = kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
 #pragma unroll
       for (int sI = 0; sI < w2; ++sI) tm[sI] = fmaxf(tm[sI], tm[sI + w2]);
     const float M = tm[0];
 #pragma unroll
-    for (int sI = 0; sI < kRowHalves * kDecodeMaxCluster; ++sI) {
+    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) {
       const float wgt = M == -INFINITY ? 0.f : fast_exp2(mx[sI] - M);
       ov[sI] *= wgt; ls[sI] *= wgt;
     }
 #pragma unroll
-    for (int w2 = kRowHalves * kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
+    for (int w2 = kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
 #pragma unroll
       for (int sI = 0; sI < w2; ++sI) { ov[sI] += ov[sI + w2]; ls[sI] += ls[sI + w2]; }
     const float o = ov[0], l = ls[0];
@@ -586,13 +591,13 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   if (n_clusters > 1) {
     // ---- several clusters per head: the last CTA to arrive merges the cluster results ----
     __threadfence();
-    __syncthreads();
+    bar_sync(2, kConsumerThreads);
     if (tid == 0) sh.last = atomicAdd(&p.tickets[bk], 1) == (int)gridDim.x - 1;
-    __syncthreads();
+    bar_sync(2, kConsumerThreads);
     if (sh.last != 0) {
       __threadfence();
       const float *all = p.partials + (int64_t)bk * n_clusters * kPartialStride;
-      for (int item = tid; item < p.G * kHeadDim; item += kDecodeThreads) {
+      for (int item = tid; item < p.G * kHeadDim; item += kConsumerThreads) {
         const int h = item >> 7, col = item & 127;
         float M = -INFINITY;
         for (int i = 0; i < n_clusters; ++i) M = fmaxf(M, __ldcg(all + i * kPartialStride + kMaxGroup * kHeadDim + h));
@@ -612,7 +617,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     }
   }
   // ---- the step counter: whoever took the last ticket of the launch knows that every CTA has read it ----
-  if (append && tid == kDecodeThreads - 1 && my_ticket == (int)(gridDim.x * gridDim.y * gridDim.z) - 1) {
+  if (append && tid == kConsumerThreads - 1 && my_ticket == (int)(gridDim.x * gridDim.y * gridDim.z) - 1) {
     p.tickets[p.B * p.H_kv] = 0;
     *p.d_step = step + 1;
   }
@@ -620,19 +625,19 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   SAGEKV_TRACE_END;
 }
 
-
-static size_t decode_smem_bytes(int resident_tiles) {
-  return 1024 + (size_t)resident_tiles * kTileBytes + sizeof(DecShared);
+static int decode_slots(int per_cta) { return 2 * per_cta < kDecodeSlots ? 2 * per_cta : kDecodeSlots; }
+static size_t decode_smem_bytes(int per_cta) {
+  return 1024 + (size_t)decode_slots(per_cta) * kSlotBytes + sizeof(DecShared);
 }
 
-// How many clusters of `c` CTAs with `tiles` resident tiles each can be on the device at once (a cluster must fit
+// How many clusters of `c` CTAs that take `tiles` tiles each can be on the device at once (a cluster must fit
 // into one GPC, so this is not n_sm / c: on this part 15 clusters of 8 whole-SM CTAs but 22 of 6).  Asked of the
 // runtime once per (device, size, tiles) and remembered.  0: unknown.
-static int g_cluster_cap[64][kDecodeMaxCluster + 1][kDecodeMaxResident + 1];   // answer + 1; 0 = not asked yet
+static int g_cluster_cap[64][kDecodeMaxCluster + 1][kDecodeMaxTiles + 1];   // answer + 1; 0 = not asked yet
 static std::mutex g_cap_mutex;
 
 static int cluster_capacity(int device, int c, int tiles) {
-  if (device < 0 || device >= 64 || c < 1 || c > kDecodeMaxCluster || tiles < 0 || tiles > kDecodeMaxResident) return 0;
+  if (device < 0 || device >= 64 || c < 1 || c > kDecodeMaxCluster || tiles < 0 || tiles > kDecodeMaxTiles) return 0;
   std::lock_guard<std::mutex> lock(g_cap_mutex);
   int &slot = g_cluster_cap[device][c][tiles];
   if (slot == 0) {
@@ -647,69 +652,56 @@ static int cluster_capacity(int device, int c, int tiles) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, decode_attn_kernel<false>, &cfg) != cudaSuccess) {
+    int nn = 0;
+    if (cudaOccupancyMaxActiveClusters(&nn, decode_attn_kernel<true>, &cfg) != cudaSuccess) {
       (void)cudaGetLastError();
-      n = 0;
+      nn = 0;
     }
-    slot = n + 1;
+    slot = nn + 1;
   }
   return slot - 1;
 }
 
 cudaError_t decode_setup(DeviceInfo *dev) {
-  const int max_smem = (int)decode_smem_bytes(kDecodeMaxResident);
-  cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
   (void)dev;
-  return e;
+  const cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)decode_smem_bytes(kDecodeMaxTiles));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)decode_smem_bytes(kDecodeMaxTiles));
 }
 
-// Launch geometry for a reduced cache of L rows: nc clusters of c CTAs per KV head.  A CTA holds its whole range at
-// once when it fits (up to kDecodeMaxResident tiles) and goes through it in rounds otherwise; with nc > 1 the
-// clusters' results are merged through scratch by the last CTA to arrive.  heads = batch x KV heads of the launch
-// (0, or dev null: not known; then one cluster of 8 per head, more only beyond kDecodeMaxRounds rounds).
-// Back-to-back launches overlap (the next one fetches its rows while this one computes), which only works if the
-// clusters of two launches fit on the device together, so the candidates are compared by
-//     waves of (two launches' clusters) / 2  x  time of one cluster,
-// the latter, measured on this part, about 4 us + 0.07 us per tile of a round + 3.5 us per further round + 1.5 us
-// for the merge through scratch.  (15 clusters of 8 whole-SM CTAs fit at once, 22 of 6, 26 of 5, 33 of 4.)
-constexpr int kDecodeMaxClustersPerHead = 4;
-
-void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, int *cs, int *resident_tiles, int *smem_bytes) {
+// Launch geometry for a reduced cache of L rows: nc clusters of c CTAs per KV head, a CTA taking at most
+// kDecodeMaxTiles tiles (its K tiles must all be resident); nc > 1 only beyond that, the clusters' results then
+// merged through scratch by the last CTA to arrive.  heads = batch x KV heads of the launch (0, or dev null: not
+// known; then clusters of 8).  Back-to-back launches overlap (the next one fetches its rows while this one
+// computes), which only works if the clusters of two launches fit on the device together, so the cluster sizes
+// are compared by   waves of (two launches' clusters) / 2  x  time of one cluster,   the latter, on this part,
+// about 4 us + 0.1 us per tile of a CTA, + 0.8 us when part of V has to wait for the K slots.
+// (15 clusters of 8 whole-SM CTAs fit at once, 22 of 6, 26 of 5, 33 of 4.)
+void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, int *cs, int *per_cta_tiles, int *smem_bytes) {
   const int n_tiles = (L + 15) / 16;
   int c = 1;
   while (c < kDecodeBaseCluster && c * 2 <= n_tiles) c <<= 1;                   // cluster size 1, 2, 4 or 8
-  const int per_cluster_cta = kDecodeRoundTiles * kDecodeMaxRounds;              // most tiles a CTA goes through
-  int nc = (n_tiles + c * per_cluster_cta - 1) / (c * per_cluster_cta);
+  const int nc = (n_tiles + c * kDecodeMaxTiles - 1) / (c * kDecodeMaxTiles);
   if (dev != nullptr && heads > 0 && c == kDecodeBaseCluster) {
     float best = 0.f;
-    int best_c = c, best_nc = nc;
-    for (int cand_nc = nc; cand_nc <= nc; ++cand_nc) {   // (more clusters per head than needed were measured: the merge through scratch and the lost overlap cost more than the rounds saved)
-      for (int cand = kDecodeBaseCluster; cand >= 4; --cand) {
-        if (cand == 7) continue;                                                 // (no more of them fit than of 8)
-        const int per = (n_tiles + cand * cand_nc - 1) / (cand * cand_nc);
-        if (per > per_cluster_cta) continue;
-        if (per < 4 && cand_nc > 1) continue;                                    // too little work per CTA to pay for the merge
-        const int resident = per <= kDecodeMaxResident ? per : 2 * kDecodeRoundTiles;
-        const int rounds = per <= kDecodeMaxResident ? 1 : (per + kDecodeRoundTiles - 1) / kDecodeRoundTiles;
-        const int cap = cluster_capacity(dev->device, cand, resident);
-        if (cap <= 0) continue;
-        const float one = 4.0f + 0.07f * (float)(rounds == 1 ? per : kDecodeRoundTiles) + 3.5f * (float)(rounds - 1) +
-                          (cand_nc > 1 ? 1.5f : 0.f);
-        const float cost = 0.5f * (float)((2 * heads * cand_nc + cap - 1) / cap) * one;
-        if (best == 0.f || cost < best) { best = cost; best_c = cand; best_nc = cand_nc; }
-      }
+    int best_c = c;
+    for (int cand = kDecodeBaseCluster; cand >= 4; --cand) {
+      const int per = (n_tiles + cand * nc - 1) / (cand * nc);
+      if (per > kDecodeMaxTiles) continue;
+      const int cap = cluster_capacity(dev->device, cand, per);
+      if (cap <= 0) continue;
+      const float one = 4.0f + 0.1f * (float)per + (2 * per > kDecodeSlots ? 0.8f : 0.f);
+      const float cost = 0.5f * (float)((2 * heads * nc + cap - 1) / cap) * one;
+      if (best == 0.f || cost < best) { best = cost; best_c = cand; }
     }
     c = best_c;
-    nc = best_nc;
   }
   const int per_cta = (n_tiles + c * nc - 1) / (c * nc);                         // most tiles a CTA gets
   *n_clusters = nc;
   *cs = c;
-  *resident_tiles = per_cta <= kDecodeMaxResident ? per_cta : 2 * kDecodeRoundTiles;
-  *smem_bytes = (int)decode_smem_bytes(*resident_tiles);
+  *per_cta_tiles = per_cta;
+  *smem_bytes = (int)decode_smem_bytes(per_cta);
 }
 
 // cuTensorMapEncodeTiled, looked up through the runtime (the library does not link against the driver)
@@ -747,8 +739,8 @@ static bool make_cache_map(CUtensorMap *map, const uint16_t *base, const DecodeP
 }
 
 cudaError_t launch_decode(const DecodeParams &p, const DeviceInfo &dev, cudaStream_t stream) {
-  int n_clusters, cs, resident, smem;
-  decode_geometry(p.L, p.B * p.H_kv, &dev, &n_clusters, &cs, &resident, &smem);
+  int n_clusters, cs, per_cta, smem;
+  decode_geometry(p.L, p.B * p.H_kv, &dev, &n_clusters, &cs, &per_cta, &smem);
   CUtensorMap map_k, map_v;
   if (!make_cache_map(&map_k, p.Kc, p) || !make_cache_map(&map_v, p.Vc, p)) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
@@ -765,10 +757,8 @@ cudaError_t launch_decode(const DecodeParams &p, const DeviceInfo &dev, cudaStre
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = p.pdl_mode > 0 ? 2 : 1;
-  const int n_tiles = (p.L + 15) / 16;
-  const int per_cta = (n_tiles + n_clusters * cs - 1) / (n_clusters * cs);
-  return per_cta > kDecodeMaxResident ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true>, p, map_k, map_v, resident)
-                                      : cudaLaunchKernelEx(&cfg, decode_attn_kernel<false>, p, map_k, map_v, resident);
+  return 2 * per_cta > kDecodeSlots ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true>, p, map_k, map_v, decode_slots(per_cta))
+                                    : cudaLaunchKernelEx(&cfg, decode_attn_kernel<false>, p, map_k, map_v, decode_slots(per_cta));
 }
 
 }  // namespace sagekv
