@@ -296,6 +296,7 @@ def side_workload(B, synth, torch, name, n_layers, dev, hint, check, O):
     w = synth.workload(name)
     st = Stack(B, synth, torch, w, n_layers, 4, dev, hint)
     st.sk.set_overlap(2)
+    st.sk.set_select_overlap(2)
     ga, gb, gc = st.graph(st.phase_a), st.graph(st.phase_b), st.graph(st.phase_c)
     a = st.time_graph(ga, 2, 3) * 1e3 / (2 * n_layers)
     b = st.time_graph(gb, 2, 3) * 1e3 / (2 * n_layers)
@@ -346,6 +347,10 @@ def run_cuda(args, w):
     # belongs to another layer, so the reduced cache may be fetched before the dependency wait
     overlap = args.overlap if args.overlap is not None else (2 if n_layers > 1 else 1)
     sk.set_overlap(overlap)
+    # the select calls of the layers are queued one after another (phase B follows the score calls of every layer),
+    # so no select launch's predecessor writes its inputs: the selection may run ahead of the dependency wait
+    sel_overlap = args.select_overlap if args.select_overlap is not None else (2 if n_layers > 1 else 1)
+    sk.set_select_overlap(sel_overlap)
     ga, gb, gc = st.graph(st.phase_a), st.graph(st.phase_b), st.graph(st.phase_c)
     c_replays = decode_steps // graph_steps
 
@@ -386,7 +391,7 @@ def run_cuda(args, w):
     a_us, b_us, c_us = (replicas.max_over_ranks(x, dev) for x in (a_us, b_us, c_us))
 
     # ---- beside the timed step (rank 0, one GPU): the other settings of the same calls, and the Qwen shape ----
-    by_hint, by_overlap, other, parity = {}, {}, [], None
+    by_hint, by_overlap, by_sel_overlap, other, parity = {}, {}, {}, [], None
     if rank == 0 and args.gpus == 1 and not args.quick:
         for mode in (0, 1, 2):
             st.set_hint(mode)
@@ -394,6 +399,12 @@ def run_cuda(args, w):
             by_hint[str(mode)] = {"score_us_per_layer": st.time_graph(g_a, 1, 3) * 1e3 / n_layers,
                                   "select_compact_us_per_layer": st.time_graph(g_b, 1, 3) * 1e3 / n_layers}
         st.set_hint(hint)
+        st.phase_a()
+        for mode in (0, 1, 2):
+            sk.set_select_overlap(mode)
+            g_b = gb if mode == sel_overlap else st.graph(st.phase_b)
+            by_sel_overlap[str(mode)] = st.time_graph(g_b, 1, 3) * 1e3 / n_layers
+        sk.set_select_overlap(sel_overlap)
         st.phase_a(); st.phase_b()                   # leave the caches as the timed step left them
         for mode in (0, 1, 2):
             sk.set_overlap(mode)
@@ -430,6 +441,7 @@ def run_cuda(args, w):
     }
     if by_hint:
         kernels["select_compact"]["by_hint_mode"] = by_hint
+        kernels["select_compact"]["by_select_overlap_mode"] = by_sel_overlap
         kernels["select_compact"]["note"] = ("hint mode 2: sagekv_score leaves a candidate list behind each row and "
                                              "sagekv_select_compact ranks it instead of reading the row, so its DRAM "
                                              "traffic is below the algorithmic bytes (which count the scores); the work "
@@ -448,7 +460,7 @@ def run_cuda(args, w):
                            w.n_q_heads, w.n_kv_heads, w.head_dim),
                        "layers": n_layers, "batch": w.batch, "n_ctx": w.n_ctx, "budget": w.budget, "n_init": w.n_init,
                        "n_recent": w.n_recent, "k_per_kv_head": w.n_sel, "k_q": w.k_q,
-                       "decode_steps_per_step": decode_steps, "decode_overlap_mode": overlap, "select_hint_mode": hint,
+                       "decode_steps_per_step": decode_steps, "decode_overlap_mode": overlap, "select_overlap_mode": sel_overlap, "select_hint_mode": hint,
                        "parallelism": "replicas x%d" % args.gpus,
                        "l2": "inputs larger than L2: layers visited round-robin, %.0f MB of K per layer, %.0f MB of "
                              "reduced caches per decode step" % (ab["score"] / 1e6, ab["decode_attn"] * n_layers / 1e6)},
@@ -569,6 +581,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--overlap", type=int, default=None, help="sagekv_set_overlap mode for the decode phase")
+    ap.add_argument("--select-overlap", type=int, default=None, help="sagekv_set_select_overlap mode for the select phase")
     ap.add_argument("--hint", type=int, default=2, help="sagekv_set_select_hint mode for the score and select phases")
     ap.add_argument("--check", action="store_true", help="compare layer 0 of every timed workload with the CPU oracle")
     ap.add_argument("--quick", action="store_true", help="only the timed step: no other modes, no other workloads")

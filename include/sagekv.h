@@ -169,9 +169,8 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
 
 /* How sagekv_decode_attn launches overlap with the kernel before them on the
  * stream.  Step 4 runs once per layer and per generated token, so at batch 1 the
- * launch-to-launch gap is a large share of its cost.  (The score and
- * select+compact launches are always plain: measured, early scheduling of their
- * successors cost them more than the hidden launch latency gained.)
+ * launch-to-launch gap is a large share of its cost.  (The score launches are
+ * always plain; sagekv_set_select_overlap covers select+compact.)
  *   0  (default) plain launch: starts when the previous kernel has finished.
  *   1  programmatic dependent launch: the kernel may be scheduled while its
  *      predecessor drains, and waits on the device for the predecessor to
@@ -184,6 +183,24 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
  *      are still read after the wait.
  * Errors: INVALID for a null context or a mode outside 0..2. */
 int sagekv_set_overlap(sagekv_ctx *ctx, int mode);
+
+/* The same choice for the launches of sagekv_select_compact, sagekv_select_topk
+ * and the pooled selection (Section 2, Steps 2 and 3), which run once per layer
+ * after prefill and last a few microseconds each, so that with many layers queued
+ * on a stream the gaps between them weigh as much as the work.
+ *   0  (default) plain launch.
+ *   1  programmatic dependent launch; the kernel waits on the device for its
+ *      predecessor before it reads or writes anything a program can observe (it
+ *      may ask for the candidate list to be brought into L2 earlier).  Always safe.
+ *   2  as 1, but with a trusted candidate list (select hint mode 2) the wait is
+ *      put off until the kernel's first WRITE: the list, K and V are read, and
+ *      the selection is made, while the predecessor may still be running.  Only
+ *      for callers who guarantee that the kernel directly before the call on the
+ *      stream writes none of the call's inputs (scores with their lists, K, V):
+ *      for example the select call of another layer, when the score calls of all
+ *      layers were queued first.  Without a candidate list mode 2 acts as mode 1.
+ * Errors: INVALID for a null context or a mode outside 0..2. */
+int sagekv_set_select_overlap(sagekv_ctx *ctx, int mode);
 
 /* How the G query heads of a KV head share its selected slots.
  *   0  (default, the paper's reading: Step 2 selects per query head and the

@@ -23,6 +23,7 @@ struct sagekv_ctx {
   int32_t *status;          // one int32: kStatus* bits raised by the kernels
   int last_cuda_error;
   int overlap;              // 0, 1 or 2: see sagekv_set_overlap
+  int select_overlap;       // 0, 1 or 2: see sagekv_set_select_overlap
   int hint;                 // 0, 1, 2: see sagekv_set_select_hint
   int32_t hint_k;
   int group_mode;           // 0: a selection per query head (the paper's), 1: one per KV head from pooled scores
@@ -88,6 +89,7 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   ctx->scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.0f / sqrtf((float)shape->head_dim);
   ctx->last_cuda_error = 0;
   ctx->overlap = 0;
+  ctx->select_overlap = 0;
   ctx->hint = 0;
   ctx->hint_k = 0;
   ctx->group_mode = 0;
@@ -230,6 +232,7 @@ int sagekv_select_compact(sagekv_ctx *ctx, const float *scores, int64_t scores_r
   p.status = ctx->status;
   p.sketch = !pooled && ctx->hint == 1;
   p.list = !pooled && ctx->hint == 2 && k == ctx->hint_k;
+  p.pdl = ctx->select_overlap;
   const cudaError_t e = launch_select_compact(p, ctx->dev->n_sm, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   state->n_init = n_init;
@@ -289,6 +292,12 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
 int sagekv_set_overlap(sagekv_ctx *ctx, int mode) {
   if (ctx == nullptr || mode < 0 || mode > 2) return SAGEKV_ERR_INVALID;
   ctx->overlap = mode;
+  return SAGEKV_OK;
+}
+
+int sagekv_set_select_overlap(sagekv_ctx *ctx, int mode) {
+  if (ctx == nullptr || mode < 0 || mode > 2) return SAGEKV_ERR_INVALID;
+  ctx->select_overlap = mode;
   return SAGEKV_OK;
 }
 

@@ -91,6 +91,7 @@ struct SelectParams {
   int32_t *status = nullptr;   // status word of the context, or null
   bool sketch = false;         // the caller asked for the histograms behind the rows to be used (sagekv_set_select_hint)
   bool list = false;           // the caller vouches for the candidate lists behind the rows (hint mode 2)
+  int pdl = 0;                 // 0 plain launch; 1 programmatic dependent launch; 2 also select before the dependency wait
 };
 cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t stream);
 cudaError_t select_compact_setup();   // one-time function attributes

@@ -32,6 +32,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "trace.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -120,34 +121,6 @@ __device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
 // keeps a value that was worked out early in a register, so that the work is not redone (later) where it is used
 __device__ __forceinline__ void pin(uint32_t &x) { asm volatile("" : "+r"(x)); }
 __device__ __forceinline__ void pin(int &x) { asm volatile("" : "+r"(x)); }
-
-// ---- timeline of a launch (only in a build with -DSAGEKV_TRACE; the normal build contains none of it) ----------
-// Thread 0 of every CTA notes the global timer at ten points and leaves the record in a ring in device memory,
-// which sagekv_trace_read copies out.  A stamp that has to follow a computation carries a (never true) dependence on
-// its result, so that it cannot be scheduled ahead of it.
-#if defined(SAGEKV_TRACE)
-constexpr int kTraceSlots = 1 << 15, kTraceStamps = 12;
-__device__ unsigned long long g_trace[kTraceSlots][kTraceStamps];
-__device__ unsigned int g_trace_n;
-__device__ __forceinline__ unsigned long long trace_now() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-#define SAGEKV_TRACE_BEGIN unsigned long long trace_t[kTraceStamps] = {0ull};
-#define SAGEKV_STAMP(i) do { if (threadIdx.x == 0) trace_t[i] = trace_now(); } while (0)
-#define SAGEKV_STAMP_AFTER(i, val_) do { if (threadIdx.x == 0) trace_t[i] = trace_now() + (unsigned long long)((val_) == 1.2345e-33f); } while (0)
-#define SAGEKV_TRACE_END do { if (threadIdx.x == 0) { \
-    const unsigned int slot_ = atomicAdd(&g_trace_n, 1u) % kTraceSlots; \
-    trace_t[10] = ((unsigned long long)blockIdx.x << 32) | ((unsigned long long)blockIdx.y << 16) | blockIdx.z; \
-    trace_t[11] = gridDim.x; \
-    for (int i_ = 0; i_ < kTraceStamps; ++i_) g_trace[slot_][i_] = trace_t[i_]; } } while (0)
-#else
-#define SAGEKV_TRACE_BEGIN
-#define SAGEKV_STAMP(i) do { } while (0)
-#define SAGEKV_STAMP_AFTER(i, val_) do { } while (0)
-#define SAGEKV_TRACE_END do { } while (0)
-#endif
 
 __device__ __forceinline__ void bar_sync(int id, int n_threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
@@ -763,17 +736,4 @@ cudaError_t launch_decode(const DecodeParams &p, const DeviceInfo &dev, cudaStre
 
 }  // namespace sagekv
 
-#if defined(SAGEKV_TRACE)
-// Copies the records out (host buffer of 32768 x 12 64-bit words), returns how many launches' CTAs were recorded
-// since the last call, and starts a new recording.  Synchronises the device.
-extern "C" int sagekv_trace_read(unsigned long long *host, unsigned int *n_records) {
-  if (cudaDeviceSynchronize() != cudaSuccess) return SAGEKV_ERR_CUDA;
-  unsigned int n = 0, zero = 0;
-  if (cudaMemcpyFromSymbol(&n, sagekv::g_trace_n, sizeof(n)) != cudaSuccess) return SAGEKV_ERR_CUDA;
-  if (cudaMemcpyFromSymbol(host, sagekv::g_trace, sizeof(unsigned long long) * sagekv::kTraceSlots * sagekv::kTraceStamps) != cudaSuccess)
-    return SAGEKV_ERR_CUDA;
-  if (cudaMemcpyToSymbol(sagekv::g_trace_n, &zero, sizeof(zero)) != cudaSuccess) return SAGEKV_ERR_CUDA;
-  *n_records = n;
-  return SAGEKV_OK;
-}
-#endif
+SAGEKV_TRACE_READER(sagekv_trace_read)

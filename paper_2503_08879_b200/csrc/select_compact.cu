@@ -29,6 +29,7 @@
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "trace.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -467,9 +468,15 @@ __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const 
 
 // Steps 4 and 5 on a position-sorted candidate list that every CTA of the cluster holds in `cand_all` (at least
 // k_q entries, each >= T0; sh.hist_fast zero, sh.n_border zero).  arrived: the CTA has a cluster arrival pending
-// (from fast_candidates) that has to be waited for before another path may run.
+// (from fast_candidates) that has to be waited for before another path may run.  defer_idx: nothing is written to
+// global memory here; the CTA's (slot, position) list in shared memory is all that comes out.
+#if defined(SAGEKV_TRACE)
+#define SAGEKV_STAMP_AT(tr_, i_) do { if ((tr_) != nullptr && threadIdx.x == 0) (tr_)[i_] = trace_now(); } while (0)
+#else
+#define SAGEKV_STAMP_AT(tr_, i_) do { } while (0)
+#endif
 __device__ int fast_decide(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c, uint32_t T0,
-                           uint32_t kmax, int M, bool arrived) {
+                           uint32_t kmax, int M, bool arrived, bool defer_idx = false, unsigned long long *tr = nullptr) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned long long *cand_all = reinterpret_cast<unsigned long long *>(c.scratch) + c.cand_cap;
   unsigned char *flag = reinterpret_cast<unsigned char *>(cand_all + c.cand_cap + 2);
@@ -488,6 +495,7 @@ __device__ int fast_decide(cg::cluster_group &cluster, SelShared &sh, const Sele
   find_bin_from_top(sh.hist_fast, kSelThreads, p.k_q, sh);
   const uint32_t b1 = (uint32_t)sh.found[0];
   const int r1 = sh.found[1];                            // the k_q-th largest is the r1-th largest inside b1
+  SAGEKV_STAMP_AT(tr, 3);
   uint32_t *border = sh.gmax;                            // free: every peer is past step 2
   for (int i = tid; i < M; i += kSelThreads) {
     const uint32_t bin = min((uint32_t)(cand_all[i] >> (32 + shift2)) - base2, (uint32_t)kSelThreads - 1u);
@@ -498,6 +506,7 @@ __device__ int fast_decide(cg::cluster_group &cluster, SelShared &sh, const Sele
     }
   }
   __syncthreads();
+  SAGEKV_STAMP_AT(tr, 4);
   const int nb = sh.n_border;
   if (nb > kSelThreads) {                                // a large group of near-equal scores at the cut
     if (arrived) cluster.barrier_wait();
@@ -512,6 +521,7 @@ __device__ int fast_decide(cg::cluster_group &cluster, SelShared &sh, const Sele
     if (lane == 0) flag[i] = before < r1 ? 1 : 0;
   }
   __syncthreads();
+  SAGEKV_STAMP_AT(tr, 5);
 
   // 5. output slots: the list is in position order, so a kept candidate's slot is the number of kept ones
   //    before it.  The CTA writes and gathers an even share of the slots, wherever the rows come from.
@@ -529,7 +539,7 @@ __device__ int fast_decide(cg::cluster_group &cluster, SelShared &sh, const Sele
         if (slot >= slot_lo && slot < slot_hi) {
           const int pos = p.S + (int)(0xffffffffu - (uint32_t)(cand_all[i] & 0xffffffffull));
           (void)SAGEKV_OK_INDEX(p.status, pos >= p.S && pos < p.S + p.E && slot - slot_lo < c.list_cap);
-          idx_row[slot] = pos;
+          if (!defer_idx) idx_row[slot] = pos;            // deferred: the caller writes them from the list, later
           c.list[slot - slot_lo] = make_int2(slot, pos);
         }
         ++slot;
@@ -671,6 +681,26 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   const int cs = cluster.num_blocks();
   const int rank = cluster.block_rank();
   const int cid = blockIdx.x / cs;
+  SAGEKV_TRACE_BEGIN
+  SAGEKV_STAMP(0);
+  // Programmatic dependent launch (sagekv_set_select_overlap): the kernel may have been scheduled while its
+  // predecessor on the stream was still running.  Mode 1 reads and writes nothing before the predecessor is
+  // complete (a request to bring the candidate list into L2 changes nothing a program can observe).  Mode 2 (the
+  // caller vouches that the predecessor writes none of this call's inputs) puts the wait off until the first
+  // write: selection and the first round of row loads run ahead of it, on the candidate-list path.
+  bool waited = p.pdl == 0;
+  if (p.pdl) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (p.pdl == 1 || (p.pdl == 2 && (list_off < 0 || cid >= n_rows))) {
+    if (list_off >= 0 && cid < n_rows) {
+      const char *lines = reinterpret_cast<const char *>(p.scores + (int64_t)cid * p.row_stride + list_off);
+      const int n_lines = (kListTagWords * 4 + cand_cap * 8 + 127) >> 7;
+      const int mine = rank + (int)threadIdx.x * cs;
+      if (mine < n_lines) asm volatile("prefetch.global.L2 [%0];" ::"l"(lines + (int64_t)mine * 128));
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    waited = true;
+  }
+  SAGEKV_STAMP(1);
   if (cid >= n_rows) {   // whole cluster takes this branch together; it touches no peer's memory
     copy_static_rows(p, (cid - n_rows) * cs + rank, (gridDim.x / cs - n_rows) * cs);
     return;
@@ -748,6 +778,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
 
   // The gather list follows the buffers of the path that runs (see select_smem_bytes).
   bool done = false, exit_wait = false;   // exit_wait: a cluster arrival of the prefilter is still to be waited for
+  bool idx_deferred = false;              // the selection wrote no indices: they follow from the gather lists
   if (try_fast) {
     c.list = reinterpret_cast<int2 *>(c.scratch + (size_t)cand_cap * 16 + 16 + (((size_t)cand_cap + 15) & ~(size_t)15));
     int code = kFastRetry;
@@ -762,14 +793,23 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
       if (tid == 0) sh.n_border = 0;
       cluster.barrier_wait();                              // the arrive at kernel entry; no peer's memory is touched on this path
       __syncthreads();
-      code = fast_decide(cluster, sh, p, c, lt[4], lt[5], M, false);
+      SAGEKV_STAMP(2);
+#if defined(SAGEKV_TRACE)
+      code = fast_decide(cluster, sh, p, c, lt[4], lt[5], M, false, !waited, trace_t);
+#else
+      code = fast_decide(cluster, sh, p, c, lt[4], lt[5], M, false, !waited);
+#endif
+      SAGEKV_STAMP(6);
+      idx_deferred = !waited && code == kFastDone;
       if (code == kFastGeneral) {                          // (a large group of equal scores at the cut)
+        if (!waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited = true; }
         c.list = reinterpret_cast<int2 *>(c.scratch + kGeneralScratch);
         general_select(cluster, sh, p, c);
         code = kFastDone;
       }
       done = true;
     }
+    if (!done && !waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited = true; }   // the other paths write as they go
     if (!done && sketch_off >= 0 && tag0 == kSketchMagic && tag1 == (uint32_t)p.E)   // the same words in every CTA of the row
       code = resident ? fast_select<true, true>(cluster, sh, p, c, hint, false)
                       : fast_select<false, true>(cluster, sh, p, c, hint, false);
@@ -784,6 +824,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     cluster.barrier_wait();
   }
   if (!done) {
+    if (!waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited = true; }
     c.list = reinterpret_cast<int2 *>(c.scratch + kGeneralScratch);
     general_select(cluster, sh, p, c);
   }
@@ -791,7 +832,9 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   // gather the rows on this CTA's list into head j's segment of the reduced cache: a warp moves four rows at a
   // time (K in lanes 0-15, V in lanes 16-31), all loads issued before the stores
   const bool gather = p.Kc != nullptr;                   // null: the caller wants the indices only
-  const int n_list = gather ? min(sh.list_count, list_cap) : 0;
+  int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
+  const int n_list_all = min(sh.list_count, list_cap);
+  const int n_list = gather ? n_list_all : 0;
   const uint16_t *src_base = (lane < 16 ? p.K : p.V) + (int64_t)b * p.ks.batch_stride + (int64_t)kvh * p.ks.head_stride +
                              (lane & 15) * 8;
   uint16_t *dst_base = (lane < 16 ? p.Kc : p.Vc) + (int64_t)b * p.cs.batch_stride + (int64_t)kvh * p.cs.head_stride +
@@ -803,7 +846,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   int sr = (j * cs + rank) * kSelWarps + warp;           // this warp's first static row
   for (int e0 = warp * 4; e0 < n_list || sr < n_static; e0 += kSelWarps * 4) {
     uint4 v[4], vs = make_uint4(0u, 0u, 0u, 0u);
-    int slot[4];
+    int slot[4], pos[4];
     const bool has_static = sr < n_static;
     if (has_static) {
       const int64_t src_tok = sr < p.S ? sr : (int64_t)p.E + sr;                 // S + E + (sr - S)
@@ -816,8 +859,18 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
         int2 sp = c.list[min(e0 + u, n_list - 1)];
         if (!SAGEKV_OK_INDEX(p.status, sp.x >= 0 && sp.x < p.k_q && sp.y >= p.S && sp.y < p.S + p.E)) sp = make_int2(0, p.S);
         slot[u] = sp.x;
+        pos[u] = sp.y;
         v[u] = ld_stream_v4(src_base + (int64_t)sp.y * p.ks.token_stride);
       }
+    }
+    if (!waited) {                                         // the first write of this warp
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      waited = true;
+    }
+    if (idx_deferred) {                                    // the indices of the rows this warp moves
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (lane == u && e0 + u < n_list) idx_row[slot[u]] = pos[u];
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
@@ -829,7 +882,14 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
       sr += static_stride;
     }
   }
+  if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");   // a warp without a round of the loop
+  if (idx_deferred && !gather)                             // indices only: nothing was moved, every thread is here
+    for (int i = tid; i < n_list_all; i += kSelThreads) idx_row[c.list[i].x] = c.list[i].y;
+  SAGEKV_STAMP(7);
   if (cid == 0 && rank == 0 && tid == 0 && p.d_step != nullptr) *p.d_step = 0;
+  SAGEKV_STAMP(8);
+  SAGEKV_STAMP(9);
+  SAGEKV_TRACE_END;
   if (exit_wait) cluster.barrier_wait();   // prefilter path: a peer may still have been copying this CTA's candidates
 }
 
@@ -985,7 +1045,9 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   const bool sketch = list || (select && p.sketch && sketch_fits(p.E, p.row_stride));   // both read the row unstaged, if at all
   // cluster size: slices of at least 2048 scores, at most 8 CTAs (the portable limit)
   int cs = 1;
-  while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E && (!sketch || (int64_t)n_rows * cs * 2 <= 2 * (int64_t)n_sm)) cs <<= 1;
+  // (from a candidate list nothing but the gather scales with the cluster, and two CTAs share an SM well)
+  const int64_t cta_room = list ? 2 * (int64_t)n_sm : (int64_t)n_sm;
+  while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E && (!sketch || (int64_t)n_rows * cs * 2 <= cta_room)) cs <<= 1;
   int chunk = (p.E + cs - 1) / cs;
   chunk = (chunk + 3) & ~3;
   if (chunk < 4) chunk = 4;
@@ -1015,13 +1077,15 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   cfg.blockDim = dim3(kSelThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = cs;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = p.pdl ? 2 : 1;
   const int64_t sketch_off = try_fast && sketch && !list ? sketch_offset(p.E) : (int64_t)-1;
   const int64_t list_off = try_fast && list ? sketch_offset(p.E) : (int64_t)-1;
   return cudaLaunchKernelEx(&cfg, select_compact_kernel, p, n_rows, chunk, (int)resident, list_cap, cand_cap,
@@ -1029,3 +1093,5 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
 }
 
 }  // namespace sagekv
+
+SAGEKV_TRACE_READER(sagekv_trace_read_select)

@@ -1,11 +1,11 @@
-"""Timeline of the decode-attention launches: where the time of a launch goes, CTA by CTA.
+"""Timeline of the decode-attention (or select+compact) launches: where the time of a launch goes, CTA by CTA.
 
-Builds the library with -DSAGEKV_TRACE (thread 0 of every CTA of sagekv_decode_attn's kernel notes the global timer
-at ten points; the normal build has none of that), replays a CUDA graph of decode calls over the layers of a
-workload, and prints the phases of a launch as medians over CTAs and launches.  The stamps cost a few per cent, so
-the microseconds per launch printed here are a little above the benchmark's.
+Builds the library with -DSAGEKV_TRACE (thread 0 of every CTA of the kernel notes the global timer at ten points;
+the normal build has none of that), replays a CUDA graph of decode calls (select calls in hint mode 2 with
+`--select`) over the layers of a workload, and prints the phases of a launch as medians over CTAs and launches.
+The stamps cost a few per cent, so the microseconds per launch printed here are a little above the benchmark's.
 
-    python -m paper_2503_08879_b200.trace [workload] [overlap mode] [layers]
+    python -m paper_2503_08879_b200.trace [workload] [overlap mode] [layers] [--select]
 """
 
 from __future__ import annotations
@@ -16,8 +16,85 @@ import sys
 
 import numpy as np
 
+SELECT_NAMES = ["CTA starts", "dependency wait over", "candidate list in shared memory", "cut bin found",
+                "candidates flagged", "border ranked", "slots written", "gather issued", "step word", "CTA ends"]
 NAMES = ["CTA starts", "copies issued", "dependency wait over", "K landed", "maxima exchanged", "weights stored",
          "second product done", "results sent", "inbox full", "CTA ends"]
+
+
+def report(buf_reader, names, ctas_of, run, label):
+    """Records one run and prints the phases; ctas_of(first record) = CTAs per launch."""
+    import torch
+    buf = np.zeros((1 << 15, 12), dtype=np.uint64)
+    n = C.c_uint(0)
+    buf_reader(buf.ctypes.data_as(C.c_void_p), C.byref(n))                         # starts a fresh recording
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); n_calls = run(); e1.record(); torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n_calls
+    buf_reader(buf.ctypes.data_as(C.c_void_p), C.byref(n))
+    t = buf[: min(n.value, 1 << 15)].astype(np.int64)
+    ctas = ctas_of(t[0])
+    n_launch = t.shape[0] // ctas
+    t = t[np.argsort(t[:, 9])][: n_launch * ctas].reshape(n_launch, ctas, 12)       # launches end one after another
+    ends = t[:, :, 9].max(axis=1)
+    lo, hi = n_launch // 4, n_launch - n_launch // 4
+    mid, prev = t[lo:hi], ends[lo - 1: hi - 1]
+    print("%s: %d CTAs per launch, %.2f us per launch with the stamps; launch ends %.0f ns apart (median)" % (
+        label, ctas, us, np.median(np.diff(ends))))
+    print("| phase of a CTA | median ns | 10 % | 90 % |")
+    print("|---|---|---|---|")
+    for i in range(9):
+        d = mid[:, :, i + 1] - mid[:, :, i]
+        print("| %s -> %s | %.0f | %.0f | %.0f |" % (names[i], names[i + 1], np.median(d), np.percentile(d, 10), np.percentile(d, 90)))
+    print("| previous launch's last CTA ends -> dependency wait over | %.0f | | |" % np.median(mid[:, :, names.index("dependency wait over")] - prev[:, None]))
+    print("| CTA starts, relative to the previous launch's end | %.0f | | |" % np.median(mid[:, :, 0] - prev[:, None]))
+    rel = mid[:, :, 9] - ends[lo:hi, None]
+    print("| CTA ends, relative to its launch's last CTA | %.0f | %.0f | %.0f |" % (np.median(rel), np.percentile(rel, 10), 0))
+
+
+def trace_select(argv):
+    """Select+compact launches in hint mode 2 over the layers of a workload (scores and lists from sagekv_score)."""
+    import torch
+    from . import binding as B, synth
+    name = argv[0] if len(argv) > 0 else "C3-2048"
+    overlap = int(argv[1]) if len(argv) > 1 else 1
+    w = synth.workload(name)
+    n_layers = int(argv[2]) if len(argv) > 2 else min(16, w.n_layers)
+    dev = torch.device("cuda:0")
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L, device=dev)
+    sk.set_select_hint(2, w.n_sel)
+    stride = sk.score_stride(w.n_ctx, w.n_init, w.n_recent)
+    layers = []
+    for l in range(n_layers):
+        lay = synth.make_layer(w, l, dev)
+        lay["scores"] = torch.empty(w.batch * w.n_q_heads, stride, dtype=torch.float32, device=dev)
+        lay["cache"] = sk.new_layer(w.n_init, w.n_recent, w.n_sel)
+        B.sagekv_score(sk.ctx, lay["q_last"], lay["K"], w.n_ctx, w.n_init, w.n_recent, lay["scores"], stride)
+        layers.append(lay)
+    sk.set_overlap(overlap)
+    rounds = 4
+
+    def phase():
+        for _ in range(rounds):
+            for lay in layers:
+                c = lay["cache"]
+                B.sagekv_select_compact(sk.ctx, lay["scores"], stride, lay["K"], lay["V"], w.n_ctx, w.n_init, w.n_recent,
+                                        w.n_sel, c.idx, c.Kc, c.Vc, c.state)
+
+    phase(); torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        phase()
+    for _ in range(3):
+        g.replay()
+
+    def run():
+        g.replay()
+        return rounds * n_layers
+
+    report(B.lib.sagekv_trace_read_select, SELECT_NAMES, lambda r: int(r[11]), run,
+           "%s select+compact, hint mode 2, overlap mode %d, %d layers" % (name, overlap, n_layers))
+    sk.close()
 
 
 def main(argv):
@@ -25,6 +102,8 @@ def main(argv):
     os.environ["SAGEKV_LIB"] = build.build(trace=True)
     import torch
     from . import binding as B, synth
+    if "--select" in argv:
+        return trace_select([a for a in argv if a != "--select"])
     name = argv[0] if len(argv) > 0 else "C3-2048"
     overlap = int(argv[1]) if len(argv) > 1 else 2
     w = synth.workload(name)
@@ -52,32 +131,13 @@ def main(argv):
         phase()
     for _ in range(3):
         g.replay()
-    buf = np.zeros((1 << 15, 12), dtype=np.uint64)
-    n = C.c_uint(0)
-    B.lib.sagekv_trace_read(buf.ctypes.data_as(C.c_void_p), C.byref(n))           # starts a fresh recording
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(); g.replay(); e1.record(); torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) * 1e3 / (steps * n_layers)
-    B.lib.sagekv_trace_read(buf.ctypes.data_as(C.c_void_p), C.byref(n))
-    t = buf[: min(n.value, 1 << 15)].astype(np.int64)
-    ctas = int(t[0, 11]) * w.n_kv_heads * w.batch
-    n_launch = t.shape[0] // ctas
-    t = t[np.argsort(t[:, 9])][: n_launch * ctas].reshape(n_launch, ctas, 12)       # launches end one after another
-    ends = t[:, :, 9].max(axis=1)
-    mid = t[n_launch // 4: n_launch - n_launch // 4]
-    prev = ends[n_launch // 4 - 1: n_launch - n_launch // 4 - 1]
-    print("%s, overlap mode %d, %d layers: %d CTAs per launch (cluster size %d), %.2f us per launch with the stamps; "
-          "launch ends %.0f ns apart (median)" % (name, overlap, n_layers, ctas, int(t[0, 0, 11]), us, np.median(np.diff(ends))))
-    print("| phase of a CTA | median ns | 10 % | 90 % |")
-    print("|---|---|---|---|")
-    for i in range(9):
-        d = mid[:, :, i + 1] - mid[:, :, i]
-        print("| %s -> %s | %.0f | %.0f | %.0f |" % (NAMES[i], NAMES[i + 1], np.median(d), np.percentile(d, 10), np.percentile(d, 90)))
-    print("| previous launch's last CTA ends -> dependency wait over | %.0f | | |" % np.median(mid[:, :, 2] - prev[:, None]))
-    print("| CTA starts, relative to the previous launch's end | %.0f | | |" % np.median(mid[:, :, 0] - prev[:, None]))
-    print("| CTA ends, relative to its launch's last CTA | %.0f | %.0f | %.0f |" % (
-        np.median(mid[:, :, 9] - ends[n_launch // 4: n_launch - n_launch // 4, None]),
-        np.percentile(mid[:, :, 9] - ends[n_launch // 4: n_launch - n_launch // 4, None], 10), 0))
+
+    def run():
+        g.replay()
+        return steps * n_layers
+
+    report(B.lib.sagekv_trace_read, NAMES, lambda r: int(r[11]) * w.n_kv_heads * w.batch, run,
+           "%s decode, overlap mode %d, %d layers (cluster size %s)" % (name, overlap, n_layers, "= CTAs / (KV heads x batch)"))
     sk.close()
 
 

@@ -355,6 +355,47 @@ def test_dependent_launch_same_layer_back_to_back(B):
     sk.close()
 
 
+@pytest.mark.parametrize("mode,hint", [(1, 0), (1, 2), (2, 2), (2, 1), (2, 0)])
+def test_select_overlap_across_layers(B, mode, hint):
+    """sagekv_set_select_overlap: the select calls of three layers follow one another on the stream, several rounds
+    without host synchronisation, after the score calls of all layers (so no call's predecessor writes its inputs,
+    which is what mode 2 asks for; with hint 2 the selection then runs ahead of the dependency wait).  Indices are
+    those of the oracle's select on the GPU's scores, caches are the oracle's gather, the step words are reset."""
+    w = synth.workload("C3-2048").with_(n_ctx=20011, n_layers=3)
+    dev = "cuda"
+    sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L)
+    sk.set_select_hint(hint, w.n_sel)
+    stride = sk.score_stride(w.n_ctx, w.n_init, w.n_recent)
+    lays, caches, scores = [], [], []
+    for l in range(3):
+        lay = synth.make_layer(w, l, dev)
+        sc = sk.new_scores(w.n_ctx, w.n_init, w.n_recent)
+        B.sagekv_score(sk.ctx, lay["q_last"], lay["K"], w.n_ctx, w.n_init, w.n_recent, sc, stride)
+        c = sk.new_layer(w.n_init, w.n_recent, w.n_sel, spare_rows=GUARD_ROWS)
+        lays.append(lay); scores.append(sc); caches.append(c)
+    sk.set_select_overlap(mode)
+    for rnd in range(3):
+        for c in caches:
+            c.Kc.view(torch.int16).fill_(CANARY)
+            c.Vc.view(torch.int16).fill_(CANARY)
+            c.idx.fill_(-1)
+            c.step.fill_(99)
+        for l in range(3):                                # back to back: nothing between the three launches
+            sk.select_compact(scores[l], lays[l]["K"], lays[l]["V"], w.n_init, w.n_recent, w.n_sel, caches[l])
+    torch.cuda.synchronize()
+    assert sk.status() == 0
+    for l in range(3):
+        got = scores[l].view(w.batch, w.n_q_heads, -1)[0, :, : w.E].cpu().numpy()
+        idx = caches[l].indices()[0].cpu().numpy()
+        assert np.array_equal(idx, O.select(got, w.k_q, w.n_init))
+        Kc_ref, Vc_ref = O.compact(bits(lays[l]["K"][0]), bits(lays[l]["V"][0]), idx, w.n_init, w.n_recent)
+        Kc, Vc = caches[l].cache()
+        assert np.array_equal(bits(Kc[0]), Kc_ref) and np.array_equal(bits(Vc[0]), Vc_ref)
+        assert (caches[l].Kc.view(torch.int16)[:, :, w.L:] == CANARY).all()
+        assert int(caches[l].step.item()) == 0
+    sk.close()
+
+
 def test_prefetch_overlap_across_layers(B):
     """Overlap mode 2: decode calls of different layers alternate on one stream, so the kernel before each
     call never writes that call's cache, which is what the mode asks the caller to guarantee."""
