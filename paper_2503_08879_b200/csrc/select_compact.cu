@@ -829,7 +829,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     general_select(cluster, sh, p, c);
   }
 
-  // gather the rows on this CTA's list into head j's segment of the reduced cache: a warp moves four rows at a
+  // gather the rows on this CTA's list into head j's segment of the reduced cache: a warp moves eight rows at a
   // time (K in lanes 0-15, V in lanes 16-31), all loads issued before the stores
   const bool gather = p.Kc != nullptr;                   // null: the caller wants the indices only
   int32_t *idx_row = p.idx + (int64_t)c.row * p.k_q;
@@ -844,9 +844,9 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   const int n_static = gather ? p.S + p.R + 1 : 0;
   const int static_stride = p.G * cs * kSelWarps;
   int sr = (j * cs + rank) * kSelWarps + warp;           // this warp's first static row
-  for (int e0 = warp * 4; e0 < n_list || sr < n_static; e0 += kSelWarps * 4) {
-    uint4 v[4], vs = make_uint4(0u, 0u, 0u, 0u);
-    int slot[4], pos[4];
+  constexpr int kRows = 8;                                 // rows a warp has in flight: all loads issued before the stores
+  for (int e0 = warp * kRows; e0 < n_list || sr < n_static; e0 += kSelWarps * kRows) {
+    uint4 v[kRows], vs = make_uint4(0u, 0u, 0u, 0u);
     const bool has_static = sr < n_static;
     if (has_static) {
       const int64_t src_tok = sr < p.S ? sr : (int64_t)p.E + sr;                 // S + E + (sr - S)
@@ -854,27 +854,25 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
       vs = ld_stream_v4(src_base + src_tok * p.ks.token_stride);
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (e0 < n_list) {
-        int2 sp = c.list[min(e0 + u, n_list - 1)];
-        if (!SAGEKV_OK_INDEX(p.status, sp.x >= 0 && sp.x < p.k_q && sp.y >= p.S && sp.y < p.S + p.E)) sp = make_int2(0, p.S);
-        slot[u] = sp.x;
-        pos[u] = sp.y;
-        v[u] = ld_stream_v4(src_base + (int64_t)sp.y * p.ks.token_stride);
+    for (int u = 0; u < kRows; ++u) {
+      if (e0 + u < n_list) {
+        int pos = c.list[e0 + u].y;
+        if (!SAGEKV_OK_INDEX(p.status, pos >= p.S && pos < p.S + p.E)) pos = p.S;
+        v[u] = ld_stream_v4(src_base + (int64_t)pos * p.ks.token_stride);
       }
     }
     if (!waited) {                                         // the first write of this warp
       asm volatile("griddepcontrol.wait;" ::: "memory");
       waited = true;
     }
-    if (idx_deferred) {                                    // the indices of the rows this warp moves
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (lane == u && e0 + u < n_list) idx_row[slot[u]] = pos[u];
+    for (int u = 0; u < kRows; ++u) {
+      if (e0 + u < n_list) {
+        int slot = c.list[e0 + u].x;
+        if (!SAGEKV_OK_INDEX(p.status, slot >= 0 && slot < p.k_q)) slot = 0;
+        st_v4(dst_base + (int64_t)slot * p.cs.token_stride, v[u]);
+      }
     }
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (e0 + u < n_list) st_v4(dst_base + (int64_t)slot[u] * p.cs.token_stride, v[u]);
     if (has_static) {
       // dst_base points at the head's segment S + j*k_q; static rows are addressed from row 0 of the KV head
       const int64_t dst_row = sr < p.S ? sr : (int64_t)p.G * p.k_q + sr;         // S + G*k_q + (sr - S)
@@ -883,8 +881,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     }
   }
   if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");   // a warp without a round of the loop
-  if (idx_deferred && !gather)                             // indices only: nothing was moved, every thread is here
-    for (int i = tid; i < n_list_all; i += kSelThreads) idx_row[c.list[i].x] = c.list[i].y;
+  if (idx_deferred)                                        // every thread is here, and past the wait
+    for (int i = tid; i < n_list_all; i += kSelThreads) {
+      const int2 sp = c.list[i];
+      if (SAGEKV_OK_INDEX(p.status, sp.x >= 0 && sp.x < p.k_q)) idx_row[sp.x] = sp.y;
+    }
   SAGEKV_STAMP(7);
   if (cid == 0 && rank == 0 && tid == 0 && p.d_step != nullptr) *p.d_step = 0;
   SAGEKV_STAMP(8);
@@ -1045,9 +1046,10 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   const bool sketch = list || (select && p.sketch && sketch_fits(p.E, p.row_stride));   // both read the row unstaged, if at all
   // cluster size: slices of at least 2048 scores, at most 8 CTAs (the portable limit)
   int cs = 1;
-  // (from a candidate list nothing but the gather scales with the cluster, and two CTAs share an SM well)
-  const int64_t cta_room = list ? 2 * (int64_t)n_sm : (int64_t)n_sm;
-  while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E && (!sketch || (int64_t)n_rows * cs * 2 <= cta_room)) cs <<= 1;
+  // From a candidate list nothing but the gather scales with the cluster: a CTA takes up to 128 rows (one round of
+  // its 16 warps), and small launches leave room for the next launch's CTAs to run ahead (sagekv_set_select_overlap).
+  while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E &&
+         (list ? (p.k_q + cs - 1) / cs > 128 : (!sketch || (int64_t)n_rows * cs * 2 <= 2 * (int64_t)n_sm))) cs <<= 1;
   int chunk = (p.E + cs - 1) / cs;
   chunk = (chunk + 3) & ~3;
   if (chunk < 4) chunk = 4;
