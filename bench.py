@@ -434,11 +434,18 @@ def run_cuda(args, w):
                 "algorithmic_bytes": ab[name], "traffic": ncu_traffic(kernel, files)}
     score_kernel = ("score_logits_kernel+score_finalize_candidates_kernel" if hint == 2
                     else "score_logits_kernel+score_finalize_kernel")
+    hf = ["common.cuh", "trace.cuh"]
     kernels = {
-        "score": roof("score", a_us, score_kernel, ["score.cu", "select_compact.cu", "common.cuh"]),
-        "select_compact": roof("select_compact", b_us, "select_compact_kernel", ["select_compact.cu", "common.cuh"]),
-        "decode_attn": roof("decode_attn", c_us, "decode_attn_kernel", ["decode_attn.cu", "common.cuh"]),
+        "score": roof("score", a_us, score_kernel, ["score.cu", "select_compact.cu"] + hf),
+        "select_compact": roof("select_compact", b_us, "select_compact_kernel", ["select_compact.cu"] + hf),
+        "decode_attn": roof("decode_attn", c_us, "decode_attn_kernel", ["decode_attn.cu"] + hf),
     }
+    if hint == 2 and w.E >= 14337 and w.k_q > 0:
+        # what this mode's select call moves: the candidate lists instead of the score rows (8 tag words and
+        # 1.5 k_q + 256 entries of 8 bytes per row at most), the kept rows in and out, the indices
+        moved = ab["select_compact"] - w.batch * w.n_q_heads * (w.E * 4 - (32 + 8 * (w.k_q + w.k_q // 2 + 256)))
+        kernels["select_compact"]["bytes_moved_in_hint_mode_2"] = moved
+        kernels["select_compact"]["frac_of_bytes_moved"] = moved / (b_us * 1e-6) / 1e9 / peak
     if by_hint:
         kernels["select_compact"]["by_hint_mode"] = by_hint
         kernels["select_compact"]["by_select_overlap_mode"] = by_sel_overlap

@@ -198,7 +198,9 @@ int sagekv_set_overlap(sagekv_ctx *ctx, int mode);
  *      for callers who guarantee that the kernel directly before the call on the
  *      stream writes none of the call's inputs (scores with their lists, K, V):
  *      for example the select call of another layer, when the score calls of all
- *      layers were queued first.  Without a candidate list mode 2 acts as mode 1.
+ *      layers were queued first.
+ * Launches that do not start from a candidate list (select hint modes 0 and 1)
+ * pass over the score rows and are always plain, whatever the mode.
  * Errors: INVALID for a null context or a mode outside 0..2. */
 int sagekv_set_select_overlap(sagekv_ctx *ctx, int mode);
 

@@ -595,7 +595,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     *p.d_step = step + 1;
   }
   SAGEKV_STAMP(9);
-  SAGEKV_TRACE_END;
+  SAGEKV_TRACE_END(p.out);
 }
 
 static int decode_slots(int per_cta) { return 2 * per_cta < kDecodeSlots ? 2 * per_cta : kDecodeSlots; }

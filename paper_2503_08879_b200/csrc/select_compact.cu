@@ -673,6 +673,9 @@ __device__ void general_select(cg::cluster_group &cluster, SelShared &sh, const 
   cluster.sync();   // no CTA moves on (and may exit) while a peer still reads its shared memory
 }
 
+// kAhead: the instance for launches that start from a trusted candidate list with the dependency wait put off
+// (eight rows in flight per warp, which the other instance has no registers for).
+template <bool kAhead>
 __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const SelectParams p, int n_rows, int chunk,
                                                                       int resident, int list_cap, int cand_cap,
                                                                       int try_fast, int64_t sketch_off, int64_t list_off) {
@@ -844,8 +847,9 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   const int n_static = gather ? p.S + p.R + 1 : 0;
   const int static_stride = p.G * cs * kSelWarps;
   int sr = (j * cs + rank) * kSelWarps + warp;           // this warp's first static row
-  constexpr int kRows = 8;                                 // rows a warp has in flight: all loads issued before the stores
-  for (int e0 = warp * kRows; e0 < n_list || sr < n_static; e0 += kSelWarps * kRows) {
+  constexpr int kRows = kAhead ? 8 : 4;                    // rows a warp has in flight: all loads issued before the stores
+  const int per_warp = n_list > kSelWarps * 4 ? kRows : 4;   // a short list is spread over all the warps
+  for (int e0 = warp * per_warp; e0 < n_list || sr < n_static; e0 += kSelWarps * per_warp) {
     uint4 v[kRows], vs = make_uint4(0u, 0u, 0u, 0u);
     const bool has_static = sr < n_static;
     if (has_static) {
@@ -855,7 +859,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     }
 #pragma unroll
     for (int u = 0; u < kRows; ++u) {
-      if (e0 + u < n_list) {
+      if (u < per_warp && e0 + u < n_list) {
         int pos = c.list[e0 + u].y;
         if (!SAGEKV_OK_INDEX(p.status, pos >= p.S && pos < p.S + p.E)) pos = p.S;
         v[u] = ld_stream_v4(src_base + (int64_t)pos * p.ks.token_stride);
@@ -867,7 +871,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
     }
 #pragma unroll
     for (int u = 0; u < kRows; ++u) {
-      if (e0 + u < n_list) {
+      if (u < per_warp && e0 + u < n_list) {
         int slot = c.list[e0 + u].x;
         if (!SAGEKV_OK_INDEX(p.status, slot >= 0 && slot < p.k_q)) slot = 0;
         st_v4(dst_base + (int64_t)slot * p.cs.token_stride, v[u]);
@@ -890,7 +894,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_compact_kernel(const Se
   if (cid == 0 && rank == 0 && tid == 0 && p.d_step != nullptr) *p.d_step = 0;
   SAGEKV_STAMP(8);
   SAGEKV_STAMP(9);
-  SAGEKV_TRACE_END;
+  SAGEKV_TRACE_END(p.idx);
   if (exit_wait) cluster.barrier_wait();   // prefilter path: a peer may still have been copying this CTA's candidates
 }
 
@@ -1004,7 +1008,9 @@ static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, int share
 }
 
 cudaError_t select_compact_setup() {
-  cudaError_t e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSmemLimit);
+  cudaError_t e = cudaFuncSetAttribute(select_compact_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSmemLimit);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(select_compact_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSmemLimit);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(score_finalize_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSmemLimit);
 }
@@ -1048,8 +1054,9 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   int cs = 1;
   // From a candidate list nothing but the gather scales with the cluster: a CTA takes up to 128 rows (one round of
   // its 16 warps), and small launches leave room for the next launch's CTAs to run ahead (sagekv_set_select_overlap).
+  const bool ahead = list && p.pdl == 2;
   while (cs < kMaxCluster && (int64_t)cs * 2048 < p.E &&
-         (list ? (p.k_q + cs - 1) / cs > 128 : (!sketch || (int64_t)n_rows * cs * 2 <= 2 * (int64_t)n_sm))) cs <<= 1;
+         (ahead ? (p.k_q + cs - 1) / cs > 128 : (!sketch || (int64_t)n_rows * cs * 2 <= 2 * (int64_t)n_sm))) cs <<= 1;
   int chunk = (p.E + cs - 1) / cs;
   chunk = (chunk + 3) & ~3;
   if (chunk < 4) chunk = 4;
@@ -1087,11 +1094,17 @@ cudaError_t launch_select_compact(const SelectParams &p, int n_sm, cudaStream_t 
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = p.pdl ? 2 : 1;
+  // Only launches that start from a candidate list are short enough to gain from early scheduling: the others
+  // pass over the row, and successors scheduled early take bandwidth and SM room from that.
+  SelectParams pl = p;
+  if (!list) pl.pdl = 0;
+  cfg.numAttrs = pl.pdl ? 2 : 1;
   const int64_t sketch_off = try_fast && sketch && !list ? sketch_offset(p.E) : (int64_t)-1;
   const int64_t list_off = try_fast && list ? sketch_offset(p.E) : (int64_t)-1;
-  return cudaLaunchKernelEx(&cfg, select_compact_kernel, p, n_rows, chunk, (int)resident, list_cap, cand_cap,
-                            try_fast, sketch_off, list_off);
+  return ahead ? cudaLaunchKernelEx(&cfg, select_compact_kernel<true>, pl, n_rows, chunk, (int)resident, list_cap, cand_cap,
+                                    try_fast, sketch_off, list_off)
+               : cudaLaunchKernelEx(&cfg, select_compact_kernel<false>, pl, n_rows, chunk, (int)resident, list_cap, cand_cap,
+                                    try_fast, sketch_off, list_off);
 }
 
 }  // namespace sagekv

@@ -16,8 +16,9 @@ import sys
 
 import numpy as np
 
-SELECT_NAMES = ["CTA starts", "dependency wait over", "candidate list in shared memory", "cut bin found",
-                "candidates flagged", "border ranked", "slots written", "gather issued", "step word", "CTA ends"]
+# (in select overlap mode 2 the dependency wait sits between "slots written" and "rows moved", not at the entry)
+SELECT_NAMES = ["CTA starts", "entry done", "candidate list in shared memory", "cut bin found",
+                "candidates flagged", "border ranked", "slots written", "rows moved", "step word", "CTA ends"]
 NAMES = ["CTA starts", "copies issued", "dependency wait over", "K landed", "maxima exchanged", "weights stored",
          "second product done", "results sent", "inbox full", "CTA ends"]
 
@@ -33,9 +34,18 @@ def report(buf_reader, names, ctas_of, run, label):
     us = e0.elapsed_time(e1) * 1e3 / n_calls
     buf_reader(buf.ctypes.data_as(C.c_void_p), C.byref(n))
     t = buf[: min(n.value, 1 << 15)].astype(np.int64)
-    ctas = ctas_of(t[0])
-    n_launch = t.shape[0] // ctas
-    t = t[np.argsort(t[:, 9])][: n_launch * ctas].reshape(n_launch, ctas, 12)       # launches end one after another
+    grid = t[:, 11] & 0xffffffff
+    tags = t[:, 11] >> 32                          # which buffer the launch wrote: one value per layer
+    ctas = ctas_of(np.concatenate([t[0, :11], grid[:1]]))
+    groups = []                                    # launches may overlap in time: told apart by tag, then by start
+    for tag in np.unique(tags):
+        r = t[tags == tag]
+        r = r[np.argsort(r[:, 0])]
+        for k in range(r.shape[0] // ctas):
+            groups.append(r[k * ctas: (k + 1) * ctas])
+    groups.sort(key=lambda g_: g_[:, 9].max())
+    t = np.stack(groups)
+    n_launch = t.shape[0]
     ends = t[:, :, 9].max(axis=1)
     lo, hi = n_launch // 4, n_launch - n_launch // 4
     mid, prev = t[lo:hi], ends[lo - 1: hi - 1]
@@ -46,7 +56,8 @@ def report(buf_reader, names, ctas_of, run, label):
     for i in range(9):
         d = mid[:, :, i + 1] - mid[:, :, i]
         print("| %s -> %s | %.0f | %.0f | %.0f |" % (names[i], names[i + 1], np.median(d), np.percentile(d, 10), np.percentile(d, 90)))
-    print("| previous launch's last CTA ends -> dependency wait over | %.0f | | |" % np.median(mid[:, :, names.index("dependency wait over")] - prev[:, None]))
+    if "dependency wait over" in names:
+        print("| previous launch's last CTA ends -> dependency wait over | %.0f | | |" % np.median(mid[:, :, names.index("dependency wait over")] - prev[:, None]))
     print("| CTA starts, relative to the previous launch's end | %.0f | | |" % np.median(mid[:, :, 0] - prev[:, None]))
     rel = mid[:, :, 9] - ends[lo:hi, None]
     print("| CTA ends, relative to its launch's last CTA | %.0f | %.0f | %.0f |" % (np.median(rel), np.percentile(rel, 10), 0))
@@ -57,7 +68,7 @@ def trace_select(argv):
     import torch
     from . import binding as B, synth
     name = argv[0] if len(argv) > 0 else "C3-2048"
-    overlap = int(argv[1]) if len(argv) > 1 else 1
+    overlap = int(argv[1]) if len(argv) > 1 else 2
     w = synth.workload(name)
     n_layers = int(argv[2]) if len(argv) > 2 else min(16, w.n_layers)
     dev = torch.device("cuda:0")
@@ -71,7 +82,7 @@ def trace_select(argv):
         lay["cache"] = sk.new_layer(w.n_init, w.n_recent, w.n_sel)
         B.sagekv_score(sk.ctx, lay["q_last"], lay["K"], w.n_ctx, w.n_init, w.n_recent, lay["scores"], stride)
         layers.append(lay)
-    sk.set_overlap(overlap)
+    sk.set_select_overlap(overlap)
     rounds = 4
 
     def phase():
