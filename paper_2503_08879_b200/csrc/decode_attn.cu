@@ -308,11 +308,13 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   if (append) {
     new_row = ld_v4((lane < 16 ? kn : vn) + (lane & 15) * 8);
     asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(step) : "l"(p.d_step));
-    // One ticket per CTA, taken once the counter has been read (release: the load is ordered before it), by a
-    // thread of the warp with the fewest tiles.  The answer is looked at only when the CTA is done, long after
-    // it has come back.
+    // One ticket per CTA, taken once the counter has been read, by a thread of the warp with the fewest tiles.
+    // The increment is computed from the value read (its sign bit, never set, plus one), so the atomic cannot
+    // be issued before the load has returned; a release fence in its place held the warp for 0.5 us, and the
+    // block barrier after the first product with it.  The answer is looked at only when the CTA is done.
     if (tid == kConsumerThreads - 1)
-      asm volatile("atom.add.release.gpu.global.s32 %0, [%1], 1;" : "=r"(my_ticket) : "l"(p.tickets + p.B * p.H_kv) : "memory");
+      asm volatile("{ .reg .b32 inc; shr.u32 inc, %2, 31; add.u32 inc, inc, 1; atom.add.relaxed.gpu.global.s32 %0, [%1], inc; }"
+                   : "=r"(my_ticket) : "l"(p.tickets + p.B * p.H_kv), "r"(step) : "memory");
   }
 
   bool timed_out = false;                 // a copy never arrived: reported through the status word; the CTA runs on (its output is then meaningless)
