@@ -55,6 +55,7 @@ struct DecShared {
   int last;
   int pad_[3];
   float warp_m[kDecodeWarps][kMaxGroup];                       // maxima of the warps' rows
+  float warp_l[kDecodeWarps][kMaxGroup];                       // sums of the warps' (rounded) weights
   float2 inbox_ml[kDecodeMaxCluster][kMaxGroup];               // [source CTA][head] (max, sum)
   uint32_t P[kDecodeMaxTiles * kPTileWords];                   // softmax weights: [tile][head][row pair g: rows 2g, 2g + 1]
   float inbox_o[(kHeadDim + 4 * kDecodeMaxCluster) * kMaxGroup];   // [source CTA][my column][head]; cluster size x columns <= 160
@@ -405,9 +406,13 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
         sv[kQkGroup * grp + i][0] = sv[kQkGroup * grp + i][1] = sv[kQkGroup * grp + i][2] = sv[kQkGroup * grp + i][3] = -INFINITY;
     }
   }
-  // over the eight lanes that hold the same heads (equal c): one warp-wide reduction per head
-  asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(wm0) : "f"(wm0), "r"(0x11111111u << c));
-  asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(wm1) : "f"(wm1), "r"(0x11111111u << c));
+  // over the eight lanes that hold the same heads (equal c)
+  // (three exchange steps: measured, redux.sync.max.f32 over such a partial lane mask took 0.2 us apiece)
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    wm0 = fmaxf(wm0, __shfl_xor_sync(0xffffffffu, wm0, o));
+    wm1 = fmaxf(wm1, __shfl_xor_sync(0xffffffffu, wm1, o));
+  }
   if (g == 0) { sh.warp_m[warp][h0] = wm0; sh.warp_m[warp][h1] = wm1; }
   bar_sync(1, kDecodeThreads);   // A: the maxima are complete, and nobody reads a K slot any more (the copy warp refills them)
 
@@ -424,7 +429,9 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   }
   SAGEKV_STAMP_AFTER(4, M0 + M1);
   const float s0 = M0 == -INFINITY ? 0.f : M0, s1 = M1 == -INFINITY ? 0.f : M1;
-  // the weights enter the second product as bf16: one word per (tile, head, row pair g: rows 2g and 2g + 1)
+  // the weights enter the second product as bf16: one word per (tile, head, row pair g: rows 2g and 2g + 1);
+  // their sums per head are taken from the rounded values, so that numerator and denominator agree
+  float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
   for (int i = 0; i < kQk; ++i) {
     const int t = warp + kDecodeWarps * i;
@@ -433,25 +440,32 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       const float x1 = fast_exp2(sv[i][1] - s1), x3 = fast_exp2(sv[i][3] - s1);              // head h1: elements 1 and 3
       const uint32_t p0 = g < 4 ? pack_bf16x2(x0, x2) : pack_bf16x2(x2, x0);                 // (row 2g in the low half)
       const uint32_t p1 = g < 4 ? pack_bf16x2(x1, x3) : pack_bf16x2(x3, x1);
+      ls0 += __uint_as_float(p0 << 16) + __uint_as_float(p0 & 0xffff0000u);                  // the weights as rounded
+      ls1 += __uint_as_float(p1 << 16) + __uint_as_float(p1 & 0xffff0000u);
       const uint32_t wa = pw_addr + (uint32_t)(t * kPTileWords * 4);
       asm volatile("st.shared.u32 [%0], %1;" ::"r"(wa), "r"(p0) : "memory");
       asm volatile("st.shared.u32 [%0], %1;" ::"r"(wa + kPHeadWords * 4), "r"(p1) : "memory");
     }
   }
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    ls0 += __shfl_xor_sync(0xffffffffu, ls0, o);
+    ls1 += __shfl_xor_sync(0xffffffffu, ls1, o);
+  }
+  if (g == 0) { sh.warp_l[warp][h0] = ls0; sh.warp_l[warp][h1] = ls1; }
   bar_sync(2, kConsumerThreads);   // B: the weights are in shared memory (and a patched early V row is visible)
   SAGEKV_STAMP(5);
 
   // ---- O^T = V^T P: columns 16*warp .. +15 over all rows, the early V tiles first ----
   // A B fragment is two of the weight words (rows 2c, 2c+1 and 2c+8, 2c+9 of head g).  Six tiles per step, each on an
-  // accumulator chain of its own, all fragments requested before the mmas.  The same weights times a fragment
-  // of ones give the sums of the rounded weights per head, in every lane, in the accumulator layout (numerator
-  // and denominator agree; no shuffle or shared-memory exchange is needed for them).
+  // accumulator chain of its own, all fragments requested before the mmas.  (An mma's result takes about 130
+  // cycles: the sums of the weights used to come from a second mma per tile against a fragment of ones, on two
+  // chains eleven links long, and those chains alone took 0.75 us; they are summed in registers now.)
   float acc[4] = {0.f, 0.f, 0.f, 0.f};    // O^T: (col_a, h0) (col_a, h1) (col_b, h0) (col_b, h1)
-  float xc[5][4], lc0[4] = {0.f, 0.f, 0.f, 0.f}, lc1[4] = {0.f, 0.f, 0.f, 0.f};
+  float xc[5][4];
 #pragma unroll
   for (int u = 0; u < 5; ++u) xc[u][0] = xc[u][1] = xc[u][2] = xc[u][3] = 0.f;
   auto second_product = [&](int t_lo, int t_hi) {
-    const uint32_t ones = 0x3f803f80u;
     for (int t6 = t_lo; t6 < t_hi; t6 += 6) {
       uint32_t va[6][4], pb[6][2];
 #pragma unroll
@@ -468,8 +482,6 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
         if (t6 + u < t_hi) {
           if (u == 0) mma_bf16_16816(acc[0], acc[1], acc[2], acc[3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
           else mma_bf16_16816(xc[u - 1][0], xc[u - 1][1], xc[u - 1][2], xc[u - 1][3], va[u][0], va[u][1], va[u][2], va[u][3], pb[u][0], pb[u][1]);
-          if (u & 1) mma_bf16_16816(lc1[0], lc1[1], lc1[2], lc1[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
-          else mma_bf16_16816(lc0[0], lc0[1], lc0[2], lc0[3], ones, ones, ones, ones, pb[u][0], pb[u][1]);
         }
       }
     }
@@ -484,7 +496,11 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   }
 #pragma unroll
   for (int e = 0; e < 4; ++e) acc[e] += ((xc[0][e] + xc[1][e]) + (xc[2][e] + xc[3][e])) + xc[4][e];
-  const float L0 = lc0[0] + lc1[0], L1 = lc0[1] + lc1[1];   // sums of the (bf16-rounded) weights of heads 2c, 2c+1 over the CTA's rows
+  float L0 = 0.f, L1 = 0.f;              // sums of the (bf16-rounded) weights of heads 2c, 2c+1 over the CTA's rows
+  if (warp == 0 && g < cs) {
+#pragma unroll
+    for (int w = 0; w < kDecodeWarps; ++w) { L0 += sh.warp_l[w][h0]; L1 += sh.warp_l[w][h1]; }
+  }
   if (timed_out) atomicOr(p.status, kStatusWaitTimeout);
   SAGEKV_STAMP_AFTER(6, acc[0] + acc[1] + acc[2] + acc[3]);
 
