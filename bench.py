@@ -347,6 +347,7 @@ def run_cuda(args, w):
     # belongs to another layer, so the reduced cache may be fetched before the dependency wait
     overlap = args.overlap if args.overlap is not None else (2 if n_layers > 1 else 1)
     sk.set_overlap(overlap)
+    sk.set_decode_variant(args.decode_variant)
     # the select calls of the layers are queued one after another (phase B follows the score calls of every layer),
     # so no select launch's predecessor writes its inputs: the selection may run ahead of the dependency wait
     sel_overlap = args.select_overlap if args.select_overlap is not None else (2 if n_layers > 1 else 1)
@@ -467,7 +468,7 @@ def run_cuda(args, w):
                            w.n_q_heads, w.n_kv_heads, w.head_dim),
                        "layers": n_layers, "batch": w.batch, "n_ctx": w.n_ctx, "budget": w.budget, "n_init": w.n_init,
                        "n_recent": w.n_recent, "k_per_kv_head": w.n_sel, "k_q": w.k_q,
-                       "decode_steps_per_step": decode_steps, "decode_overlap_mode": overlap, "select_overlap_mode": sel_overlap, "select_hint_mode": hint,
+                       "decode_steps_per_step": decode_steps, "decode_overlap_mode": overlap, "decode_variant": args.decode_variant, "select_overlap_mode": sel_overlap, "select_hint_mode": hint,
                        "parallelism": "replicas x%d" % args.gpus,
                        "l2": "inputs larger than L2: layers visited round-robin, %.0f MB of K per layer, %.0f MB of "
                              "reduced caches per decode step" % (ab["score"] / 1e6, ab["decode_attn"] * n_layers / 1e6)},
@@ -588,6 +589,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--overlap", type=int, default=None, help="sagekv_set_overlap mode for the decode phase")
+    ap.add_argument("--decode-variant", type=int, default=0, help="sagekv_set_decode_variant: 0 library's choice, 1 mma.sync, 2 tcgen05")
     ap.add_argument("--select-overlap", type=int, default=None, help="sagekv_set_select_overlap mode for the select phase")
     ap.add_argument("--hint", type=int, default=2, help="sagekv_set_select_hint mode for the score and select phases")
     ap.add_argument("--check", action="store_true", help="compare layer 0 of every timed workload with the CPU oracle")

@@ -184,6 +184,21 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
  * Errors: INVALID for a null context or a mode outside 0..2. */
 int sagekv_set_overlap(sagekv_ctx *ctx, int mode);
 
+/* Which kernel sagekv_decode_attn launches.  Both compute the same thing to the
+ * same tolerance (Section 2, Step 4).
+ *   0  (default) the library's choice: 1.
+ *   1  warp-level tensor-core instructions fed through shared-memory loads; every
+ *      cache length.
+ *   2  the tensor cores' own path (operands read from shared memory by the tensor
+ *      core, accumulators in tensor memory) where it applies: one cluster per KV
+ *      head and at most 22 tiles of 16 rows per CTA (reduced caches up to 2816
+ *      rows with clusters of 8); longer caches run as 1.  With the 4 to 8 query
+ *      heads of a KV head as the only useful columns it is the slower one
+ *      (measured: the tensor core spends one clock per operand row and k-step
+ *      however few columns there are), and it is kept as a checked alternative.
+ * Errors: INVALID for a null context or a variant outside 0..2. */
+int sagekv_set_decode_variant(sagekv_ctx *ctx, int variant);
+
 /* The same choice for the launches of sagekv_select_compact, sagekv_select_topk
  * and the pooled selection (Section 2, Steps 2 and 3), which run once per layer
  * after prefill and last a few microseconds each, so that with many layers queued

@@ -53,6 +53,8 @@ lib.sagekv_score_static.argtypes = [C.POINTER(Shape), _vp, _vp, Strides, _i64, _
 lib.sagekv_score_static.restype = C.c_int
 lib.sagekv_set_overlap.argtypes = [_vp, C.c_int]
 lib.sagekv_set_overlap.restype = C.c_int
+lib.sagekv_set_decode_variant.argtypes = [_vp, C.c_int]
+lib.sagekv_set_decode_variant.restype = C.c_int
 lib.sagekv_set_select_overlap.argtypes = [_vp, C.c_int]
 lib.sagekv_set_select_overlap.restype = C.c_int
 lib.sagekv_set_select_hint.argtypes = [_vp, C.c_int, _i32]
@@ -140,6 +142,10 @@ def sagekv_score(ctx, q_last, K, n_ctx: int, n_init: int, n_recent: int, scores,
 
 def sagekv_set_overlap(ctx, mode: int):
     _check(lib.sagekv_set_overlap(ctx, mode), "sagekv_set_overlap", ctx)
+
+
+def sagekv_set_decode_variant(ctx, variant: int):
+    _check(lib.sagekv_set_decode_variant(ctx, variant), "sagekv_set_decode_variant", ctx)
 
 
 def sagekv_set_select_overlap(ctx, mode: int):
@@ -253,6 +259,9 @@ class SageKV:
 
     def set_overlap(self, mode: int):
         sagekv_set_overlap(self.ctx, mode)
+
+    def set_decode_variant(self, variant: int):
+        sagekv_set_decode_variant(self.ctx, variant)
 
     def set_select_overlap(self, mode: int):
         sagekv_set_select_overlap(self.ctx, mode)

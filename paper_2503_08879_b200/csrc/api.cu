@@ -24,6 +24,7 @@ struct sagekv_ctx {
   int last_cuda_error;
   int overlap;              // 0, 1 or 2: see sagekv_set_overlap
   int select_overlap;       // 0, 1 or 2: see sagekv_set_select_overlap
+  int decode_variant;       // 0, 1 or 2: see sagekv_set_decode_variant
   int hint;                 // 0, 1, 2: see sagekv_set_select_hint
   int32_t hint_k;
   int group_mode;           // 0: a selection per query head (the paper's), 1: one per KV head from pooled scores
@@ -90,6 +91,7 @@ int sagekv_create(sagekv_ctx **out, const sagekv_shape *shape, int64_t max_ctx, 
   ctx->last_cuda_error = 0;
   ctx->overlap = 0;
   ctx->select_overlap = 0;
+  ctx->decode_variant = 0;
   ctx->hint = 0;
   ctx->hint_k = 0;
   ctx->group_mode = 0;
@@ -284,6 +286,7 @@ int sagekv_decode_attn(sagekv_ctx *ctx, const void *q, const void *k_new, const 
   p.B = ctx->shape.batch;
   p.scale_log2 = ctx->scale * kLog2e;
   p.pdl_mode = ctx->overlap;
+  p.variant = ctx->decode_variant == 0 ? kDecodeDefaultVariant : ctx->decode_variant;
   p.pooled = pooled ? 1 : 0;
   const cudaError_t e = launch_decode(p, *ctx->dev, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? SAGEKV_OK : cuda_fail(ctx, e);
@@ -298,6 +301,12 @@ int sagekv_set_overlap(sagekv_ctx *ctx, int mode) {
 int sagekv_set_select_overlap(sagekv_ctx *ctx, int mode) {
   if (ctx == nullptr || mode < 0 || mode > 2) return SAGEKV_ERR_INVALID;
   ctx->select_overlap = mode;
+  return SAGEKV_OK;
+}
+
+int sagekv_set_decode_variant(sagekv_ctx *ctx, int variant) {
+  if (ctx == nullptr || variant < 0 || variant > 2) return SAGEKV_ERR_INVALID;
+  ctx->decode_variant = variant;
   return SAGEKV_OK;
 }
 

@@ -113,6 +113,7 @@ cudaError_t launch_compact_window_rope(const WindowRopeParams &p, int n_sm, cuda
 cudaError_t launch_pool_scores(const float *scores, int64_t row_stride, float *pooled, int64_t pooled_stride, int E, int G,
                                int n_groups, int n_sm, cudaStream_t stream);
 
+constexpr int kDecodeDefaultVariant = 1;   // what sagekv_set_decode_variant(ctx, 0) stands for
 constexpr int kQuestBlock = 16;   // tokens per block of the Quest-style summaries (SAGEKV_QUEST_BLOCK)
 cudaError_t launch_quest_build(const uint16_t *K, sagekv_strides ks, uint16_t *kmin, uint16_t *kmax, int S, int E, int H_kv,
                                int B, int n_sm, cudaStream_t stream);
@@ -141,6 +142,7 @@ struct DecodeParams {
   int S, k_q, n_sel, ring_len, L, G, H_q, H_kv, B;
   float scale_log2;
   int pdl_mode;            // 0 plain launch, 1 programmatic dependent launch, 2 also fetch the cache before the wait
+  int variant;             // 1 warp-level mma kernel; 2 tensor-memory kernel where it applies
   int pooled;              // 1: every query head sees all selected rows of its KV head (k_q = n_sel), 0: its own segment
 };
 

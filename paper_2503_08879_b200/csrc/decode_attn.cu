@@ -50,14 +50,18 @@ constexpr int kQkTiles = (kDecodeMaxTiles + kDecodeWarps - 1) / kDecodeWarps;   
 constexpr uint32_t kWaitLimit = 1u << 22;      // polls of a copy barrier before giving up (each poll already blocks for a while)
 
 struct DecShared {
-  unsigned long long bar[3];                                   // K landed, early V landed, late V landed
+  // softmax weights: [tile][head][row pair g: rows 2g, 2g + 1]; the tensor-memory variant keeps its two small
+  // operands here instead (12 KB of weights, 4 KB of queries, both in the 128-byte-swizzled operand layout, which
+  // wants 1024-byte alignment: the struct sits behind the staging area, on such a boundary)
+  alignas(1024) uint32_t P[kDecodeMaxTiles * kPTileWords];
+  unsigned long long bar[5];                                   // K landed, early V landed, late V landed; scores ready, outputs ready (tensor-memory variant)
   unsigned long long inbox_bar;                                // every CTA's share for this CTA's columns has landed
   int last;
-  int pad_[3];
+  uint32_t tmem_base;                                          // tensor-memory variant: first column of the CTA's allocation
+  int pad_[2];
   float warp_m[kDecodeWarps][kMaxGroup];                       // maxima of the warps' rows
   float warp_l[kDecodeWarps][kMaxGroup];                       // sums of the warps' (rounded) weights
   float2 inbox_ml[kDecodeMaxCluster][kMaxGroup];               // [source CTA][head] (max, sum)
-  uint32_t P[kDecodeMaxTiles * kPTileWords];                   // softmax weights: [tile][head][row pair g: rows 2g, 2g + 1]
   float inbox_o[(kHeadDim + 4 * kDecodeMaxCluster) * kMaxGroup];   // [source CTA][my column][head]; cluster size x columns <= 160
 };
 
@@ -616,6 +620,16 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   SAGEKV_TRACE_END(p.out);
 }
 
+}  // namespace sagekv
+
+#include "decode_attn_tc.cuh"
+
+namespace sagekv {
+
+static size_t decode_tc_smem_bytes(int per_cta) {
+  return 1024 + (size_t)((per_cta + 7) / 8) * kTcBlockBytes + (size_t)per_cta * kSlotBytes + sizeof(DecShared);
+}
+
 static int decode_slots(int per_cta) { return 2 * per_cta < kDecodeSlots ? 2 * per_cta : kDecodeSlots; }
 static size_t decode_smem_bytes(int per_cta) {
   return 1024 + (size_t)decode_slots(per_cta) * kSlotBytes + sizeof(DecShared);
@@ -658,7 +672,10 @@ cudaError_t decode_setup(DeviceInfo *dev) {
   const cudaError_t e = cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)decode_smem_bytes(kDecodeMaxTiles));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)decode_smem_bytes(kDecodeMaxTiles));
+  const cudaError_t e2 = cudaFuncSetAttribute(decode_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)decode_smem_bytes(kDecodeMaxTiles));
+  if (e2 != cudaSuccess) return e2;
+  return cudaFuncSetAttribute(decode_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)decode_tc_smem_bytes(kTcMaxTiles));
 }
 
 // Launch geometry for a reduced cache of L rows: nc clusters of c CTAs per KV head, a CTA taking at most
@@ -748,6 +765,11 @@ cudaError_t launch_decode(const DecodeParams &p, const DeviceInfo &dev, cudaStre
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = p.pdl_mode > 0 ? 2 : 1;
+  // the tensor-memory variant where it applies: one cluster per head, every tile resident twice over
+  if (p.variant == 2 && n_clusters == 1 && per_cta <= kTcMaxTiles) {
+    cfg.dynamicSmemBytes = decode_tc_smem_bytes(per_cta);
+    return cudaLaunchKernelEx(&cfg, decode_attn_tc_kernel, p, map_k, map_v, per_cta);
+  }
   return 2 * per_cta > kDecodeSlots ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true>, p, map_k, map_v, decode_slots(per_cta))
                                     : cudaLaunchKernelEx(&cfg, decode_attn_kernel<false>, p, map_k, map_v, decode_slots(per_cta));
 }

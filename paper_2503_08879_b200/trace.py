@@ -5,7 +5,7 @@ the normal build has none of that), replays a CUDA graph of decode calls (select
 `--select`) over the layers of a workload, and prints the phases of a launch as medians over CTAs and launches.
 The stamps cost a few per cent, so the microseconds per launch printed here are a little above the benchmark's.
 
-    python -m paper_2503_08879_b200.trace [workload] [overlap mode] [layers] [--select]
+    python -m paper_2503_08879_b200.trace [workload] [overlap mode] [layers] [decode variant] [--select]
 """
 
 from __future__ import annotations
@@ -129,6 +129,7 @@ def main(argv):
         d = synth.make_decode_inputs(w, l, 0, dev)
         layers.append((cache, d, torch.empty_like(d["q"])))
     sk.set_overlap(overlap)
+    sk.set_decode_variant(int(argv[3]) if len(argv) > 3 else 0)
     steps = 4
 
     def phase():

@@ -73,7 +73,7 @@ CANARY = 0x5A5A           # bf16 bit pattern in the guard rows of the reduced ca
 GUARD_ROWS = 2
 
 
-def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0, hint=0, scale=0.0, sampled_heads=None):
+def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0, hint=0, scale=0.0, sampled_heads=None, variant=0):
     """All four steps on one layer of workload `w`, every result checked against the oracle.
 
     Every output buffer carries a guard band (rows behind the reduced cache, floats behind each score row, an
@@ -93,6 +93,7 @@ def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0, hint=0
         K, V = Kp[:, :, : w.n_ctx, :128], Vp[:, :, : w.n_ctx, :128]
     sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max_ctx=w.n_ctx, max_len=w.L, softmax_scale=scale)
     sk.set_overlap(overlap)
+    sk.set_decode_variant(variant)
     sk.set_select_hint(hint if (hint < 2 or w.n_sel > 0) else 0, w.n_sel)
     stride = sk.score_stride(w.n_ctx, w.n_init, w.n_recent)
     n_rows = w.batch * w.n_q_heads
@@ -208,6 +209,24 @@ def test_c1_full_config(B):
 def test_scaled_configs(B, name, kw, n_decode, hint):
     w = synth.workload(name).with_(n_layers=1, **kw)
     run_pipeline(B, w, n_decode, hint=hint)
+
+
+@pytest.mark.parametrize("name,kw,n_decode,overlap", [
+    ("C1", dict(), 8, 0),                                                   # 33 tiles: five per CTA, one score block
+    ("C1", dict(n_ctx=3001, budget=128, n_recent_min=8), 21, 1),            # the ring wraps twice
+    ("C3-2048", dict(n_ctx=20011), 4, 0),                                    # 129 tiles: the benchmark's geometry, three blocks
+    ("C2", dict(n_ctx=20011), 5, 2),
+    ("C4-b1", dict(n_ctx=9000, batch=2), 4, 0),                              # G = 7
+    ("C4-b1", dict(n_ctx=6000, batch=5), 2, 0),                              # clusters of 6: unequal column shares
+    ("C1", dict(n_ctx=300, budget=24, n_init=4, n_recent_min=20), 3, 0),     # k = 0: sink + recent only
+    ("C1", dict(n_ctx=2, budget=1, n_init=0, n_recent_min=1), 3, 0),         # two tokens: a single tile
+    ("C3-4096", dict(n_ctx=40000), 3, 0),                                    # beyond the variant's reach: runs as variant 1
+])
+def test_decode_tensor_memory_variant(B, name, kw, n_decode, overlap):
+    """sagekv_set_decode_variant(2): both products on tcgen05 with accumulators in tensor memory; same oracle,
+    same tolerance."""
+    w = synth.workload(name).with_(n_layers=1, **kw)
+    run_pipeline(B, w, n_decode, overlap=overlap, variant=2)
 
 
 def test_strided_cache(B):
