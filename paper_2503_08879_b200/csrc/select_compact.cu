@@ -207,10 +207,15 @@ struct SketchHint {
 // list, the bound T0 and the row maximum) and fast_decide (steps 4 and 5).  The score step can run the first
 // half itself while it normalises a row (kOwnMax: the caller hands in the maximum of the thread's own elements,
 // which it has just written to `c.data`) and leave the list behind the row for the select step to start from.
+#if defined(SAGEKV_TRACE)
+#define SAGEKV_STAMP_AT(tr_, i_) do { if ((tr_) != nullptr && threadIdx.x == 0) (tr_)[i_] = trace_now(); } while (0)
+#else
+#define SAGEKV_STAMP_AT(tr_, i_) do { } while (0)
+#endif
 template <bool kStaged, bool kSketch, bool kOwnMax = false>
 __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c,
                                const SketchHint &hint, bool entered, float own_max, uint32_t &T0_out, uint32_t &kmax_out,
-                               int &M_out, int &my_start) {
+                               int &M_out, int &my_start, unsigned long long *tr = nullptr) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned long long *cand_local = reinterpret_cast<unsigned long long *>(c.scratch);
   unsigned long long *cand_all = cand_local + c.cand_cap;            // 16-byte aligned: cand_cap is even
@@ -305,6 +310,7 @@ __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const 
     }
   }
   cluster.sync();
+  SAGEKV_STAMP_AT(tr, 5);
 
   // 2. all maxima of the cluster -> T0 (512 bins laid over [kmin, kmax])
   uint32_t gm[kMaxCluster];
@@ -331,6 +337,7 @@ __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const 
   sh.hist_fast[tid] = 0;                                 // reused in step 4 (barriers in between)
   }
   const float T0f = key_to_score(T0);
+  SAGEKV_STAMP_AT(tr, 6);
 
   // 3. candidates: scores >= T0 as (key, position), packed so that a larger value precedes in
   //    (score desc, position asc), written in position order.  A thread's hits of one iteration are a 32-bit
@@ -369,11 +376,15 @@ __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const 
   }
   __syncthreads();
   auto byte_sum = [](uint32_t w) { return (w & 0xffu) + ((w >> 8) & 0xffu) + ((w >> 16) & 0xffu) + (w >> 24); };
+  SAGEKV_STAMP_AT(tr, 7);
   int n_loc = sh.wsum[0];
   for (int it = 0; it < n_it; ++it)                      // lane l holds row l/4, warps 4*(l%4) .. +3 of the iteration's table
     n_loc += (int)__reduce_add_sync(0xffffffffu, byte_sum(reinterpret_cast<const uint32_t *>(table)[it * 32 + lane]));
   if (kSketch) cluster.barrier_wait();                   // pairs with the arrive at kernel entry: every peer runs
   if (tid < c.cs) cluster.map_shared_rank(sh.cand_cnt, tid)[c.rank] = n_loc;
+  // The score step needs only the peers' counts, not their candidates: it arrives here (release: the count is
+  // written) and waits after its own second pass, so that nobody waits for a peer's second pass.
+  if (kOwnMax) cluster.barrier_arrive();
   if (n_loc <= c.cand_cap) {
     int run_base = 0;                                    // hits of the iterations before this one
     for (int it = 0; it < n_it; ++it) {
@@ -430,7 +441,13 @@ __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const 
             ((unsigned long long)score_key(c.data[tail_i]) << 32) | (0xffffffffu - (uint32_t)(c.lo + tail_i));
     }
   }
-  cluster.sync();
+  SAGEKV_STAMP_AT(tr, 8);
+  if (kOwnMax) {
+    __syncthreads();                                     // the CTA's candidates are complete: other threads copy them out
+    cluster.barrier_wait();
+  } else {
+    cluster.sync();
+  }
   int start[kMaxCluster + 1];
   bool overflow = false;
   start[0] = 0;
@@ -470,11 +487,6 @@ __device__ int fast_candidates(cg::cluster_group &cluster, SelShared &sh, const 
 // k_q entries, each >= T0; sh.hist_fast zero, sh.n_border zero).  arrived: the CTA has a cluster arrival pending
 // (from fast_candidates) that has to be waited for before another path may run.  defer_idx: nothing is written to
 // global memory here; the CTA's (slot, position) list in shared memory is all that comes out.
-#if defined(SAGEKV_TRACE)
-#define SAGEKV_STAMP_AT(tr_, i_) do { if ((tr_) != nullptr && threadIdx.x == 0) (tr_)[i_] = trace_now(); } while (0)
-#else
-#define SAGEKV_STAMP_AT(tr_, i_) do { } while (0)
-#endif
 __device__ int fast_decide(cg::cluster_group &cluster, SelShared &sh, const SelectParams &p, const SelCtx &c, uint32_t T0,
                            uint32_t kmax, int M, bool arrived, bool defer_idx = false, unsigned long long *tr = nullptr) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -914,6 +926,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) score_finalize_candidates_kern
   const int row = blockIdx.x / cs;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   cluster.barrier_arrive();   // completed in fast_candidates: every CTA of the cluster runs before anyone writes into a peer
+  SAGEKV_TRACE_BEGIN
+  SAGEKV_STAMP(0);
   SelShared &sh = *reinterpret_cast<SelShared *>(smem_raw);
   float *staged = reinterpret_cast<float *>(smem_raw + sizeof(SelShared));
   SelCtx c;
@@ -934,16 +948,28 @@ __global__ void __launch_bounds__(kSelThreads, 2) score_finalize_candidates_kern
     const float2 v = part[i];
     merge_ml(m, l, v.x, v.y);
   }
+  {   // the maximum first, then the sums rescaled to it: independent exponentials instead of a chain of merges
+    float wm = m;
 #pragma unroll
-  for (int off = 1; off < 32; off <<= 1)
-    merge_ml(m, l, __shfl_xor_sync(0xffffffffu, m, off), __shfl_xor_sync(0xffffffffu, l, off));
-  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
-  __syncthreads();
-  m = sm_m[0]; l = sm_l[0];
+    for (int off = 1; off < 32; off <<= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
+    l = wm == -INFINITY ? 0.f : l * fast_exp2(m - wm);
 #pragma unroll
-  for (int w = 1; w < kSelWarps; ++w) merge_ml(m, l, sm_m[w], sm_l[w]);
+    for (int off = 1; off < 32; off <<= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+    if (lane == 0) { sm_m[warp] = wm; sm_l[warp] = l; }
+    __syncthreads();
+    float mm[kSelWarps], ll[kSelWarps];
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) { mm[w] = sm_m[w]; ll[w] = sm_l[w]; }
+    m = mm[0];
+#pragma unroll
+    for (int w = 1; w < kSelWarps; ++w) m = fmaxf(m, mm[w]);
+    l = 0.f;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) l += mm[w] == -INFINITY ? 0.f : ll[w] * fast_exp2(mm[w] - m);
+  }
   const float inv = 1.f / l;
   __syncthreads();   // the prefilter reuses the words the pairs were exchanged in
+  SAGEKV_STAMP(1);
 
   // normalise this thread's vectors (the ones it works on in the prefilter: see n_iterations)
   float *grow = sp.scores + (int64_t)row * sp.row_stride + c.lo;
@@ -976,12 +1002,19 @@ __global__ void __launch_bounds__(kSelThreads, 2) score_finalize_candidates_kern
     fm = fmaxf(fm, y);
   }
   c.data = resident ? staged : grow;
+  SAGEKV_STAMP_AFTER(2, fm);
 
   SketchHint none = {0u, 0u, 0u};
   uint32_t T0 = 0u, kmax = 0u;
   int M = 0, my_start = 0;
-  const int code = resident ? fast_candidates<true, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M, my_start)
-                            : fast_candidates<false, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M, my_start);
+#if defined(SAGEKV_TRACE)
+  unsigned long long *tr = trace_t;
+#else
+  unsigned long long *tr = nullptr;
+#endif
+  const int code = resident ? fast_candidates<true, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M, my_start, tr)
+                            : fast_candidates<false, false, true>(cluster, sh, p, c, none, false, fm, T0, kmax, M, my_start, tr);
+  SAGEKV_STAMP(3);
   uint32_t *tag = reinterpret_cast<uint32_t *>(sp.scores + (int64_t)row * sp.row_stride + list_off);
   if (code == kFastDone) {   // the CTAs' lists, one behind the other, are the row's list in position order
     const unsigned long long *cand_local = reinterpret_cast<const unsigned long long *>(c.scratch);
@@ -995,6 +1028,9 @@ __global__ void __launch_bounds__(kSelThreads, 2) score_finalize_candidates_kern
     tag[0] = kListMagic; tag[1] = (uint32_t)p.E; tag[2] = (uint32_t)p.k_q; tag[3] = (uint32_t)M;
     tag[4] = T0; tag[5] = kmax; tag[6] = 0u; tag[7] = 0u;
   }
+  SAGEKV_STAMP(4);
+  SAGEKV_STAMP(9);
+  SAGEKV_TRACE_END(sp.scores);
 }
 
 static size_t select_smem_bytes(int chunk, int list_cap, int cand_cap, int share, bool resident) {
