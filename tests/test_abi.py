@@ -87,4 +87,6 @@ def test_budget_split_host_function_matches_paper_and_oracle(lib):
 
 def test_null_context_is_rejected_before_any_cuda_call(lib):
     assert lib.sagekv_destroy(None) == -1
+    for setter in (lib.sagekv_set_overlap, lib.sagekv_set_select_overlap, lib.sagekv_set_decode_variant, lib.sagekv_set_group_mode):
+        assert setter(None, 0) == -1
     assert lib.sagekv_create(None, None, ctypes.c_int64(1), 1) == -1

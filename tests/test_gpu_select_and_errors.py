@@ -306,6 +306,10 @@ def test_argument_errors_are_reported_before_launch(B):
     assert code(B.sagekv_decode_attn, sk.ctx, q, None, None, layer.Kc, layer.Vc, bad, out) == B.ERR_INVALID
     B.sagekv_decode_attn(sk.ctx, q, None, None, layer.Kc, layer.Vc, layer.state, out)
     torch.cuda.synchronize()                                                                   # context still healthy
+    # the mode setters take 0..2 (the group mode 0..1) and nothing else
+    for setter in (lib.sagekv_set_overlap, lib.sagekv_set_select_overlap, lib.sagekv_set_decode_variant):
+        assert setter(sk.ctx, 3) == B.ERR_INVALID and setter(sk.ctx, -1) == B.ERR_INVALID and setter(sk.ctx, 2) == 0 and setter(sk.ctx, 0) == 0
+    assert lib.sagekv_set_group_mode(sk.ctx, 2) == B.ERR_INVALID
     # create
     h = C.c_void_p()
     shp = B.Shape(8, 2, 64, 1, 0.0)
