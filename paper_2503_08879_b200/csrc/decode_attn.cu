@@ -277,7 +277,12 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_ml) : "r"(inbox_bar), "r"(g));
     }
   }
-  // (4) the finishing stage: one thread per output value (own column lc, head fh)
+  // (4) integer divisions cost a hundred instructions apiece: the ones the tail needs are done here, and the step
+  //     counter is reduced modulo the ring length with a reciprocal worked out here
+  int n_clusters = (int)gridDim.x / cs, cl = ci / cs;
+  uint32_t ring_magic = 0xffffffffu / (uint32_t)max(p.ring_len, 1);
+  pin(n_clusters); pin(cl); pin(ring_magic);
+  // (5) the finishing stage: one thread per output value (own column lc, head fh)
   const int fin_items = my_cols * p.G, n_src = cs;
   int fin_lc = tid / p.G, fin_h = tid - fin_lc * p.G;
   uint16_t *fin_out = p.out + ((int64_t)b * p.H_q + kvh * p.G + fin_h) * kHeadDim + rank * cols + fin_lc;
@@ -330,7 +335,9 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   // the tile's V copy is here (now, for an early tile; after the first product, for a late one)
   int slot = -1, st = -1;                 // the replaced window row and its CTA-local tile (if 0 <= st < n)
   if (append) {
-    slot = p.S + p.n_sel + step % p.ring_len;
+    uint32_t r = (uint32_t)step - __umulhi((uint32_t)step, ring_magic) * (uint32_t)p.ring_len;   // the quotient may be one short
+    while (r >= (uint32_t)p.ring_len) r -= (uint32_t)p.ring_len;
+    slot = p.S + p.n_sel + (int)r;
     st = (slot >> 4) - first_tile;
   }
   const bool patcher = append && st >= 0 && st < n && (st & (kDecodeWarps - 1)) == warp;
@@ -533,7 +540,6 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
 
   // ---- finish columns [rank*cols, rank*cols + my_cols) of every head from the inbox ----
   const int bk = b * p.H_kv + kvh;
-  const int n_clusters = (int)gridDim.x / cs, cl = ci / cs;
   float *part = p.partials + ((int64_t)bk * n_clusters + cl) * kPartialStride;
   for (int item = tid; item < fin_items; item += kConsumerThreads) {
     if (item != tid) {
