@@ -281,7 +281,8 @@ def test_every_workload_at_full_size_one_layer(B, name, hint):
     run_pipeline(B, w, 2, hint=hint)
 
 
-def test_candidate_lists_with_a_large_group_of_equal_scores_at_the_cut(B):
+@pytest.mark.parametrize("sel_overlap", [0, 2])
+def test_candidate_lists_with_a_large_group_of_equal_scores_at_the_cut(B, sel_overlap):
     """Hint mode 2 on rows in which several hundred tokens share one key, placed so that the k-th score falls
     inside that group: the select step starts from the score step's list, finds too many equal scores at the cut
     for its exact ranking and hands the row to the radix path.  The lowest positions of the group must be kept."""
@@ -295,15 +296,21 @@ def test_candidate_lists_with_a_large_group_of_equal_scores_at_the_cut(B):
         q_hat = q_hat / q_hat.norm()
         lay["K"][0, kvh, pos] = (3.0 * q_hat).to(torch.bfloat16)
     sk = B.SageKV(w.n_q_heads, w.n_kv_heads, w.head_dim, 1, max_ctx=w.n_ctx, max_len=w.L)
-    for hint in (2, 0):
+    sk.set_select_overlap(sel_overlap)                    # 2: the launch whose wait is put off, falling back after it
+    for hint, spoil in ((2, False), (2, True), (0, False)):
         sk.set_select_hint(hint, w.n_sel)
         scores = sk.score(lay["q_last"], lay["K"], w.n_init, w.n_recent)
+        if spoil:                                        # rows without a usable list: the tag's first word says so
+            E4 = (w.E + 3) // 4 * 4
+            scores[::3, E4:E4 + 1] = 0.0
         layer = sk.select_compact(scores, lay["K"], lay["V"], w.n_init, w.n_recent, w.n_sel)
+        layer2 = sk.select_compact(scores, lay["K"], lay["V"], w.n_init, w.n_recent, w.n_sel)   # back to back
         torch.cuda.synchronize()
         got = scores[:, : w.E].cpu().numpy()
-        idx = layer.indices()[0].cpu().numpy()
-        assert np.array_equal(idx, O.select(got, w.k_q, w.n_init)), hint
-        check_compact(layer, lay, idx, w, 0)
+        for lyr in (layer, layer2):
+            idx = lyr.indices()[0].cpu().numpy()
+            assert np.array_equal(idx, O.select(got, w.k_q, w.n_init)), (hint, spoil)
+            check_compact(lyr, lay, idx, w, 0)
     assert sk.status() == 0
     sk.close()
 
