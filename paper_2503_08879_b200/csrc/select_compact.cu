@@ -75,8 +75,8 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *tmp) {
   __syncthreads();                     // tmp may still be read from an earlier call
   if (lane == 31) tmp[warp] = inc;
   __syncthreads();
-  int base = 0;
-  for (int w = 0; w < warp; ++w) base += tmp[w];
+  // the totals of the warps before this one: one load per lane and one warp-wide sum (not a chain of loads)
+  const int base = __reduce_add_sync(0xffffffffu, lane < warp ? tmp[lane] : 0);
   return base + inc - v;
 }
 
