@@ -392,7 +392,7 @@ def run_cuda(args, w):
     a_us, b_us, c_us = (replicas.max_over_ranks(x, dev) for x in (a_us, b_us, c_us))
 
     # ---- beside the timed step (rank 0, one GPU): the other settings of the same calls, and the Qwen shape ----
-    by_hint, by_overlap, by_sel_overlap, other, parity = {}, {}, {}, [], None
+    by_hint, by_overlap, by_sel_overlap, by_variant, other, parity = {}, {}, {}, {}, [], None
     if rank == 0 and args.gpus == 1 and not args.quick:
         for mode in (0, 1, 2):
             st.set_hint(mode)
@@ -412,6 +412,10 @@ def run_cuda(args, w):
             g_c = gc if mode == overlap else st.graph(st.phase_c)
             by_overlap[str(mode)] = st.time_graph(g_c, 8, 3) * 1e3 / (8 * graph_steps * n_layers)
         sk.set_overlap(overlap)
+        for variant in (1, 2):                       # 1: mma.sync kernel, 2: tcgen05 kernel (where it applies)
+            sk.set_decode_variant(variant)
+            by_variant[str(variant)] = st.time_graph(st.graph(st.phase_c), 8, 3) * 1e3 / (8 * graph_steps * n_layers)
+        sk.set_decode_variant(args.decode_variant)
     if args.check and rank == 0:
         parity = st.check(O)
 
@@ -456,6 +460,7 @@ def run_cuda(args, w):
                                              "moved shows in score_us_per_layer of the same mode")
     if by_overlap:
         kernels["decode_attn"]["by_overlap_mode"] = by_overlap
+        kernels["decode_attn"]["by_variant"] = by_variant
     share = {"score": a_us * n_layers, "select_compact": b_us * n_layers, "decode_attn": c_us * c_launches}
     dominant = max(share, key=share.get)
 
