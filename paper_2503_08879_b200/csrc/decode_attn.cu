@@ -56,6 +56,7 @@ struct DecShared {
   alignas(1024) uint32_t P[kDecodeMaxTiles * kPTileWords];
   unsigned long long bar[5];                                   // K landed, early V landed, late V landed; scores ready, outputs ready (tensor-memory variant)
   unsigned long long inbox_bar;                                // every CTA's share for this CTA's columns has landed
+  unsigned long long ml_bar;                                   // every CTA's (max, sum) pairs have landed (they travel ahead of the columns)
   int last;
   uint32_t tmem_base;                                          // tensor-memory variant: first column of the CTA's allocation
   int pad_[2];
@@ -173,17 +174,20 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
 
   const uint32_t kbar = smem_u32(&sh.bar[0]), vbar_e = smem_u32(&sh.bar[1]), vbar_l = smem_u32(&sh.bar[2]);
   const uint32_t inbox_bar = smem_u32(&sh.inbox_bar);
+  const uint32_t ml_bar = smem_u32(&sh.ml_bar);
   if (tid == 0) {
     mbar_init(kbar, 1);
     mbar_init(vbar_e, 1);
     mbar_init(vbar_l, 1);
     mbar_init(inbox_bar, 1);
+    mbar_init(ml_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
     // from every CTA of the cluster: 8 bytes per (own column, head pair in use) and 64 bytes of (max, sum) pairs
-    mbar_expect_tx(inbox_bar, (uint32_t)(cs * (my_cols * n_pairs * 8 + 64)));
+    mbar_expect_tx(inbox_bar, (uint32_t)(cs * my_cols * n_pairs * 8));
+    mbar_expect_tx(ml_bar, (uint32_t)(cs * 64));
   }
   __syncthreads();
   cluster.barrier_arrive();                              // waited for just before the first store into a peer: its barrier is set up
@@ -274,7 +278,7 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
     if (warp == 0 && g < cs) {                           // lane (g, c) of warp 0 tells CTA g the (max, sum) of heads 2c, 2c+1
       const uint32_t lm = smem_u32(&sh.inbox_ml[rank][h0]);
       asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst_ml) : "r"(lm), "r"(g));
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_ml) : "r"(inbox_bar), "r"(g));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar_ml) : "r"(ml_bar), "r"(g));
     }
   }
   // (4) integer divisions cost a hundred instructions apiece: the ones the tail needs are done here, and the step
@@ -466,6 +470,21 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   if (g == 0) { sh.warp_l[warp][h0] = ls0; sh.warp_l[warp][h1] = ls1; }
   bar_sync(2, kConsumerThreads);   // B: the weights are in shared memory (and a patched early V row is visible)
   SAGEKV_STAMP(5);
+  // The (max, sum) pairs of the CTA go to every CTA of the cluster now, ahead of the second product, with
+  // asynchronous stores that count their bytes on a barrier of their own at the receiver: the finishing stage
+  // has its weights ready before the columns arrive.
+  cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs, its barriers are set up
+  auto send2 = [&](uint32_t addr, uint32_t rbar, float x, float y) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+                 ::"r"(addr), "f"(x), "f"(y), "r"(rbar) : "memory");
+  };
+  if (warp == 0 && g < cs) {
+    float L0 = 0.f, L1 = 0.f;            // sums of the (bf16-rounded) weights of heads 2c, 2c+1 over the CTA's rows
+#pragma unroll
+    for (int w = 0; w < kDecodeWarps; ++w) { L0 += sh.warp_l[w][h0]; L1 += sh.warp_l[w][h1]; }
+    send2(dst_ml, bar_ml, M0, L0);
+    send2(dst_ml + 8u, bar_ml, M1, L1);
+  }
 
   // ---- O^T = V^T P: columns 16*warp .. +15 over all rows, the early V tiles first ----
   // A B fragment is two of the weight words (rows 2c, 2c+1 and 2c+8, 2c+9 of head g).  Six tiles per step, each on an
@@ -507,11 +526,6 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   }
 #pragma unroll
   for (int e = 0; e < 4; ++e) acc[e] += ((xc[0][e] + xc[1][e]) + (xc[2][e] + xc[3][e])) + xc[4][e];
-  float L0 = 0.f, L1 = 0.f;              // sums of the (bf16-rounded) weights of heads 2c, 2c+1 over the CTA's rows
-  if (warp == 0 && g < cs) {
-#pragma unroll
-    for (int w = 0; w < kDecodeWarps; ++w) { L0 += sh.warp_l[w][h0]; L1 += sh.warp_l[w][h1]; }
-  }
   if (timed_out) atomicOr(p.status, kStatusWaitTimeout);
   SAGEKV_STAMP_AFTER(6, acc[0] + acc[1] + acc[2] + acc[3]);
 
@@ -519,22 +533,42 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   // Every warp sends its 16 columns straight from registers into the owners' inboxes with asynchronous stores
   // that count their bytes on the owner's barrier: data and signal travel together and nobody waits for an
   // acknowledgement or for a cluster-wide barrier; a CTA only waits for its own inbox to fill.
-  cluster.barrier_wait();                                // pairs with the arrive at kernel entry: every peer runs, its barrier is set up
-  {
-    auto send2 = [&](uint32_t addr, uint32_t rbar, float x, float y) {
-      asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
-                   ::"r"(addr), "f"(x), "f"(y), "r"(rbar) : "memory");
-    };
-    if (h0 < p.G) {
-      send2(dst_a, bar_a, acc[0], acc[1]);
-      send2(dst_b, bar_b, acc[2], acc[3]);
-    }
-    if (warp == 0 && g < cs) {
-      send2(dst_ml, bar_ml, M0, L0);
-      send2(dst_ml + 8u, bar_ml, M1, L1);
-    }
+  if (h0 < p.G) {
+    send2(dst_a, bar_a, acc[0], acc[1]);
+    send2(dst_b, bar_b, acc[2], acc[3]);
   }
   SAGEKV_STAMP(7);
+  // the weights of the sources for this thread's first output: worked out while the columns are still on their way
+  float fin_w[kDecodeMaxCluster], fin_M = -INFINITY, fin_inv = 0.f, fin_l = 0.f;
+  auto source_weights = [&](int h) {
+    float mx[kDecodeMaxCluster], lsum[kDecodeMaxCluster];
+#pragma unroll
+    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) {
+      const float2 ml = sI < n_src ? sh.inbox_ml[sI][h] : make_float2(-INFINITY, 0.f);
+      mx[sI] = ml.x; lsum[sI] = ml.y;
+    }
+    float tm[kDecodeMaxCluster];
+#pragma unroll
+    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) tm[sI] = mx[sI];
+#pragma unroll
+    for (int w2 = kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
+#pragma unroll
+      for (int sI = 0; sI < w2; ++sI) tm[sI] = fmaxf(tm[sI], tm[sI + w2]);
+    fin_M = tm[0];
+#pragma unroll
+    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) {
+      fin_w[sI] = fin_M == -INFINITY ? 0.f : fast_exp2(mx[sI] - fin_M);
+      lsum[sI] *= fin_w[sI];
+    }
+#pragma unroll
+    for (int w2 = kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
+#pragma unroll
+      for (int sI = 0; sI < w2; ++sI) lsum[sI] += lsum[sI + w2];
+    fin_l = lsum[0];
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(fin_inv) : "f"(fin_l));   // the output is rounded to bf16: an approximate reciprocal is ample
+  };
+  if (!mbar_wait(ml_bar, 0u) && tid == 0) atomicOr(p.status, kStatusWaitTimeout);
+  if (tid < fin_items) source_weights(fin_h);
   if (!mbar_wait(inbox_bar, 0u) && tid == 0) atomicOr(p.status, kStatusWaitTimeout);
   SAGEKV_STAMP(8);
 
@@ -547,36 +581,19 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       fin_h = item - fin_lc * p.G;
       fin_out = p.out + ((int64_t)b * p.H_q + kvh * p.G + fin_h) * kHeadDim + rank * cols + fin_lc;
     }
+    if (item != tid) source_weights(fin_h);
     const int lc = fin_lc, h = fin_h, col = rank * cols + lc;
-    float mx[kDecodeMaxCluster], ls[kDecodeMaxCluster], ov[kDecodeMaxCluster];
+    float ov[kDecodeMaxCluster];
 #pragma unroll
-    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) {   // the loads of all sources are in flight together
-      const float2 ml = sI < n_src ? sh.inbox_ml[sI][h] : make_float2(-INFINITY, 0.f);
-      mx[sI] = ml.x; ls[sI] = ml.y;
-      ov[sI] = sI < n_src ? sh.inbox_o[(sI * cols + lc) * kMaxGroup + h] : 0.f;
-    }
-    float tm[kDecodeMaxCluster];
-#pragma unroll
-    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) tm[sI] = mx[sI];
+    for (int sI = 0; sI < kDecodeMaxCluster; ++sI)       // the loads of all sources are in flight together
+      ov[sI] = sI < n_src ? sh.inbox_o[(sI * cols + lc) * kMaxGroup + h] * fin_w[sI] : 0.f;
 #pragma unroll
     for (int w2 = kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
 #pragma unroll
-      for (int sI = 0; sI < w2; ++sI) tm[sI] = fmaxf(tm[sI], tm[sI + w2]);
-    const float M = tm[0];
-#pragma unroll
-    for (int sI = 0; sI < kDecodeMaxCluster; ++sI) {
-      const float wgt = M == -INFINITY ? 0.f : fast_exp2(mx[sI] - M);
-      ov[sI] *= wgt; ls[sI] *= wgt;
-    }
-#pragma unroll
-    for (int w2 = kDecodeMaxCluster / 2; w2 > 0; w2 >>= 1)
-#pragma unroll
-      for (int sI = 0; sI < w2; ++sI) { ov[sI] += ov[sI + w2]; ls[sI] += ls[sI + w2]; }
-    const float o = ov[0], l = ls[0];
+      for (int sI = 0; sI < w2; ++sI) ov[sI] += ov[sI + w2];
+    const float o = ov[0], l = fin_l, M = fin_M;
     if (n_clusters == 1) {
-      float inv;                                           // the output is rounded to bf16: an approximate reciprocal is ample
-      asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(l));
-      const float outv = l > 0.f ? o * inv : 0.f;
+      const float outv = l > 0.f ? o * fin_inv : 0.f;
       *fin_out = (uint16_t)(pack_bf16x2(outv, 0.f) & 0xffffu);
       if (p.lse != nullptr && col == 0)
         p.lse[(int64_t)b * p.H_q + kvh * p.G + h] = l > 0.f ? (M + log2f(l)) * kLn2 : -INFINITY;
