@@ -106,6 +106,15 @@ def run_pipeline(B, w, n_decode, device="cuda", strided=False, overlap=0, hint=0
     layer.Kc.view(torch.int16).fill_(CANARY)
     layer.Vc.view(torch.int16).fill_(CANARY)
     sk.select_compact(scores, K, V, w.n_init, w.n_recent, w.n_sel, layer)
+    if hint == 2:                                                     # the same call as a launch whose wait is put off
+        sk.set_select_overlap(2)
+        ahead = sk.new_layer(w.n_init, w.n_recent, w.n_sel, spare_rows=GUARD_ROWS)
+        ahead.Kc.view(torch.int16).fill_(CANARY)
+        ahead.Vc.view(torch.int16).fill_(CANARY)
+        sk.select_compact(scores, K, V, w.n_init, w.n_recent, w.n_sel, ahead)
+        sk.set_select_overlap(0)
+        torch.cuda.synchronize()
+        assert torch.equal(ahead.idx, layer.idx) and torch.equal(ahead.Kc, layer.Kc) and torch.equal(ahead.Vc, layer.Vc)
     torch.cuda.synchronize()
     assert torch.equal(first, scores[:, : w.E])                       # the score step repeats bit for bit
     if hint == 2 and w.E >= 14337 and 0 < w.k_q <= 2048:                # the lists are there and were usable
