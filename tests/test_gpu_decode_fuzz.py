@@ -47,6 +47,7 @@ def test_random_cases_match_the_oracle(B, seed):
         sm_scale = float(rng.choice([0.0, 0.0, 0.05, 0.2]))      # softmax scale of the context; 0: the default 1/sqrt(d)
         sk = B.SageKV(H, Hkv, 128, Bt, max_ctx=N, max_len=L, softmax_scale=sm_scale)
         sk.set_overlap(int(rng.integers(0, 2)))
+        sk.set_decode_variant(2 if case % 3 == 2 else 0)          # every third case on the tensor-memory kernel (where it applies)
         layer = sk.select_compact(buf if k_q else None, K, V, S, R, G * k_q)
         torch.cuda.synchronize()
         what = dict(case=case, G=G, Hkv=Hkv, batch=Bt, S=S, R=R, k_q=k_q, E=E, L=L, softmax_scale=sm_scale)
