@@ -372,15 +372,16 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
   float sv[kQk][4];
   float wm0 = -INFINITY, wm1 = -INFINITY;
 #pragma unroll
-  for (int grp = 0; grp < kQk / kQkGroup; ++grp) {
-    if (warp + kDecodeWarps * kQkGroup * grp < n) {
-      float ch[kQkGroup][4][4];
-      uint32_t fa[kQkGroup][4][4];
+  constexpr int kGrp = kLong ? 2 : kQkGroup;                // tiles at once: two where the scores of six tiles stay in registers
+  for (int grp = 0; grp < kQk / kGrp; ++grp) {
+    if (warp + kDecodeWarps * kGrp * grp < n) {
+      float ch[kGrp][4][4];
+      uint32_t fa[kGrp][4][4];
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {                   // k-steps 0..3, then 4..7
 #pragma unroll
-        for (int i = 0; i < kQkGroup; ++i) {
-          const int t = warp + kDecodeWarps * (kQkGroup * grp + i);
+        for (int i = 0; i < kGrp; ++i) {
+          const int t = warp + kDecodeWarps * (kGrp * grp + i);
           if (t < n) {
             const uint32_t tb = stage + (uint32_t)(t * kSlotBytes);
 #pragma unroll
@@ -388,8 +389,8 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
           }
         }
 #pragma unroll
-        for (int i = 0; i < kQkGroup; ++i) {
-          if (warp + kDecodeWarps * (kQkGroup * grp + i) < n) {
+        for (int i = 0; i < kGrp; ++i) {
+          if (warp + kDecodeWarps * (kGrp * grp + i) < n) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               if (hf == 0)
@@ -403,8 +404,8 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
         }
       }
 #pragma unroll
-      for (int i = 0; i < kQkGroup; ++i) {
-        const int ti = kQkGroup * grp + i;
+      for (int i = 0; i < kGrp; ++i) {
+        const int ti = kGrp * grp + i;
         const bool have = warp + kDecodeWarps * ti < n;
         const uint32_t vb4 = have ? (vis >> (4 * ti)) & 15u : 0u;
 #pragma unroll
@@ -417,8 +418,8 @@ decode_attn_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map
       }
     } else {
 #pragma unroll
-      for (int i = 0; i < kQkGroup; ++i)
-        sv[kQkGroup * grp + i][0] = sv[kQkGroup * grp + i][1] = sv[kQkGroup * grp + i][2] = sv[kQkGroup * grp + i][3] = -INFINITY;
+      for (int i = 0; i < kGrp; ++i)
+        sv[kGrp * grp + i][0] = sv[kGrp * grp + i][1] = sv[kGrp * grp + i][2] = sv[kGrp * grp + i][3] = -INFINITY;
     }
   }
   // over the eight lanes that hold the same heads (equal c)
