@@ -707,8 +707,7 @@ cudaError_t decode_setup(DeviceInfo *dev) {
 // merged through scratch by the last CTA to arrive.  heads = batch x KV heads of the launch (0, or dev null: not
 // known; then clusters of 8).  Back-to-back launches overlap (the next one fetches its rows while this one
 // computes), which only works if the clusters of two launches fit on the device together, so the cluster sizes
-// are compared by   waves of (two launches' clusters) / 2  x  time of one cluster,   the latter, on this part,
-// about 4 us + 0.1 us per tile of a CTA, + 0.8 us when part of V has to wait for the K slots.
+// are compared by a cost fitted to measurements (below).
 // (15 clusters of 8 whole-SM CTAs fit at once, 22 of 6, 26 of 5, 33 of 4.)
 void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, int *cs, int *per_cta_tiles, int *smem_bytes) {
   const int n_tiles = (L + 15) / 16;
@@ -723,8 +722,13 @@ void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, i
       if (per > kDecodeMaxTiles) continue;
       const int cap = cluster_capacity(dev->device, cand, per);
       if (cap <= 0) continue;
-      const float one = 4.0f + 0.1f * (float)per + (2 * per > kDecodeSlots ? 0.8f : 0.f);
-      const float cost = 0.5f * (float)((2 * heads * nc + cap - 1) / cap) * one;
+      // measured on this part (us per launch, batch 1 x 8 heads, L = 1025 / 2049 / 4097, clusters of 5 to 8):
+      // 2.97 + 0.0445 per tile of a CTA; the same again per tile when the clusters of two launches do not fit
+      // together (the copies are then issued on the critical path); 0.084 per V tile that has to wait for a K slot
+      const int late = 2 * per > kDecodeSlots ? 2 * per - kDecodeSlots : 0;
+      const int waves = (heads * nc + cap - 1) / cap;                          // of one launch
+      const float one = 2.97f + 0.0445f * (float)per * (2 * heads * nc <= cap ? 1.f : 2.f) + 0.084f * (float)late;
+      const float cost = (float)waves * one;
       if (best == 0.f || cost < best) { best = cost; best_c = cand; }
     }
     c = best_c;
