@@ -4,7 +4,7 @@
 // Flash-decoding on thread-block clusters.  The L rows of one KV head are cut into 16-row tiles that are
 // dealt evenly, as contiguous ranges, to the CTAs of one cluster.  A CTA brings its K and V tiles into shared
 // memory with tensor copies (one 16-row x 64-column box per request, 128-byte swizzle, completion counted on
-// an mbarrier), issued by a ninth warp that does nothing else.  The staging area has 44 slots of one tile
+// an mbarrier), issued by a ninth warp that does nothing else.  The staging area has 50 slots of one tile
 // (K or V) each.  All K tiles of the range are resident from the start; so are the V tiles while slots last,
 // and the remaining V tiles take over the K slots as soon as the first product is done.  There is one pass:
 //   S = K Q^T     16 rows x 8 heads per mma, a tile per warp in turn (the scores of all its tiles stay in
@@ -19,7 +19,7 @@
 // distributed shared memory: each warp sends its 16 columns straight from registers into the inbox of the
 // CTA that finishes those columns with asynchronous stores counted on that CTA's barrier (one way, no
 // cluster barrier), and each CTA writes its slice of the 128 output columns.  With several clusters per
-// head (caches beyond 44 tiles per CTA) the cluster results go to scratch and the CTA that arrives last
+// head (caches beyond 44 tiles per CTA: a warp keeps the scores of at most six) the cluster results go to scratch and the CTA that arrives last
 // (one atomic ticket, no waiting) merges them.
 // The staged copy of the window row that the new token replaces is overwritten in shared memory from
 // k_new / v_new once it has landed, and the CTA owning that row stores the new token into the cache.
@@ -654,6 +654,7 @@ static size_t decode_tc_smem_bytes(int per_cta) {
   return 1024 + (size_t)((per_cta + 7) / 8) * kTcBlockBytes + (size_t)per_cta * kSlotBytes + sizeof(DecShared);
 }
 
+static_assert(1024 + (size_t)kDecodeSlots * kSlotBytes + sizeof(DecShared) <= 232448, "the staging area and the rest fit into 227 KB");
 static int decode_slots(int per_cta) { return 2 * per_cta < kDecodeSlots ? 2 * per_cta : kDecodeSlots; }
 static size_t decode_smem_bytes(int per_cta) {
   return 1024 + (size_t)decode_slots(per_cta) * kSlotBytes + sizeof(DecShared);
@@ -798,7 +799,9 @@ cudaError_t launch_decode(const DecodeParams &p, const DeviceInfo &dev, cudaStre
     cfg.dynamicSmemBytes = decode_tc_smem_bytes(per_cta);
     return cudaLaunchKernelEx(&cfg, decode_attn_tc_kernel, p, map_k, map_v, per_cta);
   }
-  return 2 * per_cta > kDecodeSlots ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true>, p, map_k, map_v, decode_slots(per_cta))
+  // the short instance keeps three tiles' scores per warp and has every V tile resident from the start
+  const bool is_long = 2 * per_cta > kDecodeSlots || per_cta > kQkGroup * kDecodeWarps;
+  return is_long ? cudaLaunchKernelEx(&cfg, decode_attn_kernel<true>, p, map_k, map_v, decode_slots(per_cta))
                                     : cudaLaunchKernelEx(&cfg, decode_attn_kernel<false>, p, map_k, map_v, decode_slots(per_cta));
 }
 

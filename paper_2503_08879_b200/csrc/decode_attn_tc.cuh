@@ -29,7 +29,7 @@ namespace sagekv {
 
 constexpr int kTcBlockBytes = 8 * kSlotBytes;        // eight K tiles: 128 rows x 256 bytes, as two column halves
 constexpr int kTcHalfBytes = 8 * kHalfBytes;         // 128 rows x 128 bytes
-constexpr int kTcMaxTiles = kDecodeSlots / 2;        // 22 tiles per CTA: three blocks
+constexpr int kTcMaxTiles = 22;                      // tiles per CTA: three blocks (their K blocks and V tiles fit the staging area)
 constexpr int kTcMaxBlocks = (kTcMaxTiles + 7) / 8;
 constexpr int kTcColumns = 64;                       // tensor-memory columns: 16 per score block, 16 for the output
 constexpr int kTcOutColumn = 16 * kTcMaxBlocks;
