@@ -124,6 +124,7 @@ cudaError_t launch_quest_bounds(const uint16_t *q, const uint16_t *kmin, const u
 constexpr int kDecodeWarps = 8;                                        // consumer warps per CTA (one more warp issues the copies)
 constexpr int kDecodeMaxCluster = 8;                                   // CTAs per cluster (the portable limit)
 constexpr int kDecodeSlots = 50;                                       // 4 KB slots of a CTA's staging area, one K or one V tile each: 200 KB (what fits beside the rest)
+constexpr int kDecodeExtraClusters = 2;                                // clusters per head a launch may use beyond the fewest possible
 constexpr int kDecodeMaxTiles = 44;                                    // most 16-row tiles a CTA takes: its K tiles must all be resident, and a warp keeps the scores of six
 constexpr int kPartialStride = kMaxGroup * kHeadDim + 2 * kMaxGroup;   // floats per cluster result: O[8][128], m[8], l[8]
 

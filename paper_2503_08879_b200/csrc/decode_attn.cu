@@ -714,25 +714,34 @@ void decode_geometry(int L, int heads, const DeviceInfo *dev, int *n_clusters, i
   const int n_tiles = (L + 15) / 16;
   int c = 1;
   while (c < kDecodeBaseCluster && c * 2 <= n_tiles) c <<= 1;                   // cluster size 1, 2, 4 or 8
-  const int nc = (n_tiles + c * kDecodeMaxTiles - 1) / (c * kDecodeMaxTiles);
+  int nc = (n_tiles + c * kDecodeMaxTiles - 1) / (c * kDecodeMaxTiles);          // the fewest clusters per head
   if (dev != nullptr && heads > 0 && c == kDecodeBaseCluster) {
     float best = 0.f;
-    int best_c = c;
-    for (int cand = kDecodeBaseCluster; cand >= 4; --cand) {
-      const int per = (n_tiles + cand * nc - 1) / (cand * nc);
-      if (per > kDecodeMaxTiles) continue;
-      const int cap = cluster_capacity(dev->device, cand, per);
-      if (cap <= 0) continue;
-      // measured on this part (us per launch, batch 1 x 8 heads, L = 1025 / 2049 / 4097, clusters of 5 to 8):
-      // 2.97 + 0.0445 per tile of a CTA; the same again per tile when the clusters of two launches do not fit
-      // together (the copies are then issued on the critical path); 0.084 per V tile that has to wait for a K slot
-      const int late = 2 * per > kDecodeSlots ? 2 * per - kDecodeSlots : 0;
-      const int waves = (heads * nc + cap - 1) / cap;                          // of one launch
-      const float one = 2.97f + 0.0445f * (float)per * (2 * heads * nc <= cap ? 1.f : 2.f) + 0.084f * (float)late;
-      const float cost = (float)waves * one;
-      if (best == 0.f || cost < best) { best = cost; best_c = cand; }
+    int best_c = c, best_nc = nc;
+    // up to kDecodeExtraClusters more clusters per head than needed: beyond one cluster the results are merged
+    // through scratch anyway, and more, smaller clusters leave fewer V tiles waiting for a K slot
+    for (int n_try = nc; n_try <= (nc > 1 ? nc + kDecodeExtraClusters : nc); ++n_try) {
+      for (int cand = kDecodeBaseCluster; cand >= 4; --cand) {
+        const int per = (n_tiles + cand * n_try - 1) / (cand * n_try);
+        if (per > kDecodeMaxTiles) continue;
+        const int cap = cluster_capacity(dev->device, cand, per);
+        if (cap <= 0) continue;
+        // measured on this part (us per launch, batch 1 x 8 heads, L = 1025 / 2049 / 4097, clusters of 5 to 8):
+        // 2.97 + 0.0445 per tile of a CTA; the same again per tile when the clusters of two launches do not fit
+        // together (the copies are then issued on the critical path); 0.084 per V tile that has to wait for a K
+        // slot; 2.6 for the merge through scratch (L = 8193)
+        const int late = 2 * per > kDecodeSlots ? 2 * per - kDecodeSlots : 0;
+        const int waves = (heads * n_try + cap - 1) / cap;                      // of one launch
+        const float one = 2.97f + 0.0445f * (float)per * (2 * heads * n_try <= cap ? 1.f : 2.f) + 0.084f * (float)late +
+                          (n_try > 1 ? 2.6f : 0.f);
+        const float cost = (float)waves * one;
+        if (best == 0.f || cost < best) { best = cost; best_c = cand; best_nc = n_try; }
+      }
     }
     c = best_c;
+    nc = best_nc;
+  } else if (nc > 1) {
+    nc += kDecodeExtraClusters;                          // (context set-up: the most clusters per head a launch may choose)
   }
   const int per_cta = (n_tiles + c * nc - 1) / (c * nc);                         // most tiles a CTA gets
   *n_clusters = nc;
